@@ -1,0 +1,179 @@
+/*
+ * xsv -- compressed-KV streaming attention step (XStreamVGGT hot path), C ABI.
+ *
+ * One cache object holds, per transformer layer, the pruned and quantised
+ * key/value cache of the frame-wise causal global-attention module
+ * (paper section 3.1, Eq. 1).  xsv_step() runs one streaming step of one
+ * layer: attention of the new frame's queries over [cache ; new frame]
+ * (Eq. 2, with the cache dequantised on the fly, Eq. 12), then -- once the
+ * total length exceeds the budget L_max -- importance scoring (Eq. 3-7),
+ * top-k pruning that always keeps the first and the current frame (Eq. 8),
+ * and dimension-adaptive quantisation of the resulting cache (Eq. 9-11:
+ * keys per channel over groups of 64 tokens, values per token over 64
+ * channels).  Every step of that path runs in CUDA kernels for sm_100a;
+ * there is no CPU fallback.
+ *
+ * Conventions
+ *  - Every call returns an xsv_status; nothing throws or aborts.  Argument,
+ *    shape and order errors are detected on the host before any launch and
+ *    leave the cache unchanged.
+ *  - Pointers named "device" are CUDA device pointers, owned by the caller,
+ *    and must stay valid until `stream` has passed the call's work.  Pointers
+ *    named "host" are ordinary host pointers.
+ *  - Q, K, V, out: [heads][n_tokens][head_dim], contiguous, 16-bit elements
+ *    (fp16 or bf16 as given by `dtype`), 16-byte aligned.  `out` must not
+ *    alias an input.
+ *  - xsv_step only enqueues work on `stream`; it does not synchronise and
+ *    does not allocate (all device memory is allocated by
+ *    xsv_cache_create / xsv_cache_set_options / the first step).
+ *  - All steps of one cache share scratch buffers: issue them on one stream
+ *    (or order them yourself).  Each layer is stepped once per frame, frames
+ *    in order; layers may be stepped in any order.
+ *  - Lengths never need a device read-back: the cache length after a step is
+ *    a closed-form function of the step count, n_tokens and the budget.
+ */
+#ifndef XSV_H
+#define XSV_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct xsv_cache xsv_cache; /* opaque, library-owned */
+
+typedef enum {
+    XSV_OK = 0,
+    XSV_ERR_ARG = 1,     /* null pointer, value out of range                          */
+    XSV_ERR_SHAPE = 2,   /* n_tokens / dtype differ from the first step, bad alignment */
+    XSV_ERR_ORDER = 3,   /* options changed after the first step, layer stepped twice  */
+    XSV_ERR_OOM = 4,     /* device or host allocation failed                          */
+    XSV_ERR_CUDA = 5,    /* a CUDA runtime call failed                                */
+    XSV_ERR_TIMEOUT = 6, /* a bounded device-side wait ran out (status word)          */
+    XSV_ERR_RANGE = 7,   /* a zero-point left the int32 range (status word)           */
+    XSV_ERR_CAPACITY = 8 /* unbounded cache grew past max_cache_tokens                */
+} xsv_status;
+
+typedef enum { XSV_F16 = 0, XSV_BF16 = 1 } xsv_dtype;
+
+/* Which attention kernel xsv_step launches. */
+typedef enum {
+    XSV_ATTN_AUTO = 0,   /* the tcgen05/TMEM kernel when available for the shape */
+    XSV_ATTN_MMA = 1,    /* warp-level mma.sync kernel (portable baseline)       */
+    XSV_ATTN_TC5 = 2     /* tcgen05 + TMEM kernel                                */
+} xsv_attn_impl;
+
+/* Phases timed by the optional profiling events (xsv_cache_set_profiling). */
+enum { XSV_PHASE_ATTN = 0, XSV_PHASE_SCORE = 1, XSV_PHASE_SELECT = 2, XSV_PHASE_QUANT = 3, XSV_PHASE_COUNT = 4 };
+
+/*
+ * Create a cache for `layers` independent layers (section 3.1, Eq. 1; the
+ * budget and bit width of sections 3.2-3.3).
+ *   heads, head_dim : attention geometry; head_dim must be 64.
+ *   budget_tokens   : L_max, the cache length bound in tokens; <= 0 means
+ *                     unbounded (no pruning; see max_cache_tokens below).
+ *   bits            : 2, 4 or 8 -> quantised cache; 16 -> quantisation off
+ *                     (the cache keeps the 16-bit inputs).
+ * No device memory is allocated until the first step (or set_options with
+ * max_frame_tokens > 0).  *out receives the handle.  Uses the current device.
+ */
+xsv_status xsv_cache_create(xsv_cache** out, int layers, int heads, int head_dim,
+                            long long budget_tokens, int bits);
+
+/*
+ * Optional settings; must precede the first step (XSV_ERR_ORDER otherwise).
+ *   n_special        : camera + register tokens at the head of each frame,
+ *                      kept un-pooled by the query pooling (Eq. 3).  Default 5.
+ *   pool_group       : g, patch tokens averaged per pooled query (Eq. 3).  Default 16.
+ *   quant_group      : G, quantisation group size (section 4.1).  Must be 64.
+ *   max_frame_tokens : tokens per frame F if known (allocates now); 0: learnt
+ *                      from the first step.
+ *   max_cache_tokens : capacity in tokens for an unbounded cache
+ *                      (budget_tokens <= 0); ignored otherwise.  Default 16 frames.
+ * A negative value leaves a setting unchanged.
+ */
+xsv_status xsv_cache_set_options(xsv_cache* c, int n_special, int pool_group, int quant_group,
+                                 int max_frame_tokens, long long max_cache_tokens);
+
+/* Select the attention kernel (default XSV_ATTN_AUTO). */
+xsv_status xsv_cache_set_attn_impl(xsv_cache* c, xsv_attn_impl impl);
+
+/*
+ * One streaming step of layer `layer` (Fig. 2; Eq. 2-12).
+ *   Q, K, V : device, the new frame's queries / keys / values.
+ *   n_tokens: F; must equal the first step's.
+ *   out     : device, receives softmax(Q [K~cache ; K]^T / sqrt(head_dim)) [V~cache ; V].
+ *   stream  : cudaStream_t (as void*); NULL is the default stream.
+ * Afterwards the layer's cache holds [first frame ; kept middle ; this frame],
+ * quantised, of length min-closed-form (see xsv_cache_len).
+ */
+xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const void* V,
+                    int n_tokens, xsv_dtype dtype, void* out, void* stream);
+
+/*
+ * Same step with HOST buffers: copies Q, K, V to device staging owned by the
+ * cache, runs xsv_step, copies `out` back, all on `stream`, and returns
+ * without synchronising.  Pinned host memory makes the copies asynchronous.
+ */
+xsv_status xsv_step_host(xsv_cache* c, int layer, const void* Q_host, const void* K_host,
+                         const void* V_host, int n_tokens, xsv_dtype dtype, void* out_host,
+                         void* stream);
+
+/* Device bytes held now: codes, scales, zero-points, origin ids of all layer
+ * buffers plus the spare buffer and scratch (section 4.6's memory figure). */
+size_t xsv_cache_bytes(const xsv_cache* c);
+
+/* Bytes of one layer's packed KV at its current length (codes + scales + zero-points). */
+size_t xsv_cache_layer_kv_bytes(const xsv_cache* c, int layer);
+
+void xsv_cache_destroy(xsv_cache* c);
+
+/* Tokens currently cached in `layer` (host-side closed form; no device read). */
+long long xsv_cache_len(const xsv_cache* c, int layer);
+
+/* Frames stepped so far in `layer`. */
+long long xsv_cache_frames(const xsv_cache* c, int layer);
+
+/*
+ * Copy one layer's logical state to HOST arrays (synchronises `stream`).
+ * Any pointer may be NULL to skip it.  With T = xsv_cache_len, H heads, d = head_dim:
+ *   k_codes, v_codes : unsigned char [H][T][d], one code per byte (bits < 16);
+ *   k_scale / k_zero : float / int [H][ceil(T/64)][d]  (Eq. 10, per channel per 64-token group);
+ *   v_scale / v_zero : float / int [H][T]              (per token);
+ *   origin           : long long [T], frame_index * F + token_index of each slot;
+ *   k_raw, v_raw     : unsigned short [H][T][d], the 16-bit cache when bits == 16.
+ */
+xsv_status xsv_cache_export_layer(xsv_cache* c, int layer, unsigned char* k_codes, float* k_scale,
+                                  int* k_zero, unsigned char* v_codes, float* v_scale, int* v_zero,
+                                  long long* origin, unsigned short* k_raw, unsigned short* v_raw,
+                                  void* stream);
+
+/*
+ * Importance scores (Eq. 7) of the last pruning step of any layer, copied to
+ * a HOST array of capacity `cap` floats; *n receives their count (the length
+ * of the prunable middle segment), 0 if the last step did not prune.
+ * Synchronises `stream`.
+ */
+xsv_status xsv_last_scores(xsv_cache* c, float* scores_host, long long cap, long long* n, void* stream);
+
+/* Read (and keep) the sticky device status word; synchronises `stream`.
+ * XSV_OK, XSV_ERR_TIMEOUT or XSV_ERR_RANGE. */
+xsv_status xsv_cache_status(xsv_cache* c, void* stream);
+
+/* Per-phase CUDA-event timing.  When on, every step records events around
+ * each phase on the step's stream.  xsv_cache_profile_read synchronises the
+ * recorded events, adds their durations to per-phase totals, and returns the
+ * totals (milliseconds) and launch counts accumulated since the last reset. */
+xsv_status xsv_cache_set_profiling(xsv_cache* c, int on);
+xsv_status xsv_cache_profile_read(xsv_cache* c, double ms[XSV_PHASE_COUNT], long long launches[XSV_PHASE_COUNT], int reset);
+
+/* Kernels launched by this library in the calling process since load. */
+long long xsv_kernel_launches(void);
+
+const char* xsv_strerror(xsv_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XSV_H */

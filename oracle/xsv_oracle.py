@@ -212,11 +212,16 @@ class LayerCache:
         c = self.Vc.reshape(H, T, d // G, G)
         return dequantize(c, self.Vs[..., None], self.Vz[..., None]).reshape(H, T, d)
 
-    def step(self, Q, K, V):
+    def step(self, Q, K, V, select_on=None):
         """One streaming step (Fig. 2): attention over [cache ; frame], then,
         if the total length exceeds the budget, scoring + top-k pruning, then
         quantisation of the resulting cache.  Q, K, V [H, F, d] hold values
-        exactly representable in the 16-bit input type.  Returns out float64."""
+        exactly representable in the 16-bit input type.  Returns out float64.
+
+        select_on: for step-locked comparisons only -- an externally supplied
+        score vector on which Eq. 8 is evaluated instead of this step's own
+        scores (which are still computed and kept in last_scores), so that the
+        cache update can be compared for one and the same keep set."""
         H, d, G = self.H, self.d, self.G
         Q = np.asarray(Q, dtype=F32)
         K = np.asarray(K, dtype=F32)
@@ -241,7 +246,7 @@ class LayerCache:
         self.last_scores = None
         if prune:
             S = importance_scores(Q, Kd[:, T_first:T_c, :], self.n_special, self.g)
-            keep = keep_positions(S, T_first, Fc, T, self.L_max)
+            keep = keep_positions(S if select_on is None else np.asarray(select_on), T_first, Fc, T, self.L_max)
             self.last_scores = S
         else:
             keep = np.arange(T, dtype=np.int64)

@@ -1,0 +1,567 @@
+// Bandwidth-bound kernels of the step: pooled-query reduction and importance
+// scores (Eq. 3-7), top-k selection (Eq. 8), quantise-and-pack of the new
+// cache order (Eq. 9-11).
+#include "xsv_kernels.h"
+
+namespace {
+
+// ---------------------------------------------------------------------------
+// Eq. 3-4 (+ the row mean of Eq. 7) by linearity:
+//   q~[c] = 1/(H*N_pooled) * sum_h sum_i w_i Q[h,i,c],
+//   w_i = 1 for special tokens, 1/|group| for a patch token in a pooling group.
+// This kernel writes the fixed-order partial sums per (head, token chunk).
+// ---------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) qtilde_partial_kernel(const T* __restrict__ Q, int F, int n_special,
+                                                             int g, float* __restrict__ qpart) {
+    const int h = blockIdx.y, chunk = blockIdx.x;
+    const int per = (F + XSV_QCHUNKS - 1) / XSV_QCHUNKS;
+    const int i0 = chunk * per, i1 = min(F, i0 + per);
+    const int c2 = threadIdx.x & 31, r = threadIdx.x >> 5;
+    const int n_patch = F - n_special;
+    float a0 = 0.f, a1 = 0.f;
+    for (int i = i0 + r; i < i1; i += 8) {
+        float w = 1.f;
+        if (i >= n_special) {
+            int gi = (i - n_special) / g;
+            int sz = min(g, n_patch - gi * g);
+            w = 1.f / (float)sz;
+        }
+        const T* row = Q + ((size_t)h * F + i) * XSV_D + 2 * c2;
+        a0 = fmaf(w, xsv_to_float<T>(row[0]), a0);
+        a1 = fmaf(w, xsv_to_float<T>(row[1]), a1);
+    }
+    __shared__ float red[8][64];
+    red[r][2 * c2] = a0;
+    red[r][2 * c2 + 1] = a1;
+    __syncthreads();
+    if (threadIdx.x < 64) {
+        float s = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) s += red[k][threadIdx.x];
+        qpart[((size_t)h * XSV_QCHUNKS + chunk) * 64 + threadIdx.x] = s;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Eq. 5-7: S[j] = (1/H) sum_h q~ . K~[h, T_first + j, :] over the middle segment.
+// One thread per token; the (scale, zero-point) rows of the key groups a block
+// touches are staged in shared memory.
+// ---------------------------------------------------------------------------
+constexpr int SCORE_TPB = 256;
+constexpr int SCORE_MAXG = SCORE_TPB / XSV_G + 1;   // groups a block can span
+
+template <int BITS>
+__global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, int T_first, int T_c,
+                                                          const float* __restrict__ qpart, float qnorm,
+                                                          float* __restrict__ scores) {
+    constexpr int ROWB = XSV_D * BITS / 8;
+    constexpr int NV = ROWB / 16;              // 16-byte loads per row
+    constexpr int CPW = 32 / BITS;             // codes per 32-bit word
+    extern __shared__ float sm[];
+    float* qt = sm;                             // [64]
+    float* sS = qt + 64;                        // [H][SCORE_MAXG][64]
+    float* sZ = sS + (size_t)H * SCORE_MAXG * 64;
+
+    const int j0 = blockIdx.x * SCORE_TPB;
+    const int p0 = T_first + j0;
+    const int g_lo = p0 >> 6;
+    const int p_last = min(T_c - 1, p0 + SCORE_TPB - 1);
+    const int ng = (p_last >> 6) - g_lo + 1;
+
+    if (threadIdx.x < 64) {
+        float s = 0.f;
+        for (int k = 0; k < H * XSV_QCHUNKS; ++k) s += qpart[(size_t)k * 64 + threadIdx.x];
+        qt[threadIdx.x] = s * qnorm;
+    }
+    for (int i = threadIdx.x; i < H * ng * 64; i += SCORE_TPB) {
+        int c = i & 63, gg = (i >> 6) % ng, h = (i >> 6) / ng;
+        size_t m = ((size_t)h * lv.capg + g_lo + gg) * 64 + c;
+        sS[(h * SCORE_MAXG + gg) * 64 + c] = lv.kscale[m];
+        sZ[(h * SCORE_MAXG + gg) * 64 + c] = (float)lv.kzero[m];
+    }
+    __syncthreads();
+
+    const int p = p0 + threadIdx.x;
+    if (p >= T_c) return;
+    const int gg = (p >> 6) - g_lo;
+    float acc = 0.f;
+    for (int h = 0; h < H; ++h) {
+        const uint4* row = reinterpret_cast<const uint4*>(lv.kcodes + ((size_t)h * lv.cap + p) * ROWB);
+        const float* s = sS + (h * SCORE_MAXG + gg) * 64;
+        const float* z = sZ + (h * SCORE_MAXG + gg) * 64;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            uint4 q = row[v];
+            uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+#pragma unroll
+                for (int e = 0; e < CPW; ++e) {
+                    int c = (v * 4 + k) * CPW + e;
+                    float code = (float)((w[k] >> (e * BITS)) & ((1u << BITS) - 1u));
+                    float kt = __fmul_rn(__fsub_rn(code, z[c]), s[c]);
+                    acc = fmaf(qt[c], kt, acc);
+                }
+            }
+        }
+    }
+    scores[j0 + threadIdx.x] = acc / (float)H;
+}
+
+// bits == 16: keys are raw 16-bit values.
+template <typename T>
+__global__ void __launch_bounds__(SCORE_TPB) score_raw_kernel(LayerView lv, int H, int T_first, int T_c,
+                                                              const float* __restrict__ qpart, float qnorm,
+                                                              float* __restrict__ scores) {
+    __shared__ float qt[64];
+    if (threadIdx.x < 64) {
+        float s = 0.f;
+        for (int k = 0; k < H * XSV_QCHUNKS; ++k) s += qpart[(size_t)k * 64 + threadIdx.x];
+        qt[threadIdx.x] = s * qnorm;
+    }
+    __syncthreads();
+    const int j = blockIdx.x * SCORE_TPB + threadIdx.x;
+    const int p = T_first + j;
+    if (p >= T_c) return;
+    float acc = 0.f;
+    for (int h = 0; h < H; ++h) {
+        const T* row = reinterpret_cast<const T*>(lv.kcodes + ((size_t)h * lv.cap + p) * (XSV_D * 2));
+#pragma unroll 8
+        for (int c = 0; c < XSV_D; ++c) acc = fmaf(qt[c], xsv_to_float<T>(row[c]), acc);
+    }
+    scores[j] = acc / (float)H;
+}
+
+// ---------------------------------------------------------------------------
+// Eq. 8: top-k by radix select on an order-preserving integer image of the
+// float32 scores, ties broken by position, then an ordered compaction.
+// One block of 1024 threads; n is at most a few tens of thousands.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t score_key(float s) {
+    if (s == 0.f) s = 0.f;   // -0 and +0 compare equal: give them one key
+    uint32_t u = __float_as_uint(s);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ scores, int n, int k,
+                                                      int T_first, int T_c, int* __restrict__ srcmap,
+                                                      int* __restrict__ dscal) {
+    __shared__ int hist[256];
+    __shared__ uint32_t s_prefix;
+    __shared__ int s_remaining;
+    __shared__ int w_gt[32], w_eq[32], w_off[32], w_eqb[32];
+    __shared__ int s_first_evicted;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    uint32_t thr = 0xFFFFFFFFu;
+    int need_eq = 0;
+    if (k > 0) {
+        uint32_t prefix = 0, mask = 0;
+        if (tid == 0) s_remaining = k;
+        for (int pass = 3; pass >= 0; --pass) {
+            const int shift = pass * 8;
+            if (tid < 256) hist[tid] = 0;
+            __syncthreads();
+            for (int j = tid; j < n; j += 1024) {
+                uint32_t key = score_key(scores[j]);
+                if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1);
+            }
+            __syncthreads();
+            if (tid == 0) {
+                int remaining = s_remaining, cum = 0, digit = 0;
+                for (int b = 255; b >= 0; --b) {
+                    if (cum + hist[b] >= remaining) { digit = b; break; }
+                    cum += hist[b];
+                }
+                s_remaining = remaining - cum;
+                s_prefix = prefix | ((uint32_t)digit << shift);
+            }
+            __syncthreads();
+            prefix = s_prefix;
+            mask |= 255u << shift;
+        }
+        thr = prefix;
+        need_eq = s_remaining;     // how many of the keys equal to thr are taken (lowest positions)
+    }
+    if (tid == 0) s_first_evicted = n;
+    // ordered compaction: warp w owns the contiguous range [w*seg, (w+1)*seg)
+    const int seg = ((n + 31) / 32 + 31) / 32 * 32;
+    const int a = min(n, warp * seg), b = min(n, a + seg);
+    const int bend = a + (b - a + 31) / 32 * 32;     // whole stripes, so every lane joins the ballots
+    int cgt = 0, ceq = 0;
+    for (int j = a + lane; j < bend; j += 32) {
+        uint32_t key = j < b ? score_key(scores[j]) : 0u;
+        bool gt = j < b && key > thr, eq = j < b && key == thr && k > 0;
+        cgt += __popc(__ballot_sync(0xFFFFFFFFu, gt));
+        ceq += __popc(__ballot_sync(0xFFFFFFFFu, eq));
+    }
+    if (lane == 0) { w_gt[warp] = cgt; w_eq[warp] = ceq; }
+    __syncthreads();
+    if (warp == 0) {
+        // exclusive scans over the 32 warps, in warp order
+        int eq = w_eq[lane], gt = w_gt[lane];
+        int eq_incl = eq;
+        for (int o = 1; o < 32; o <<= 1) { int t = __shfl_up_sync(0xFFFFFFFFu, eq_incl, o); if (lane >= o) eq_incl += t; }
+        int eq_before = eq_incl - eq;
+        int take_eq = max(0, min(eq, need_eq - eq_before));
+        int kept = gt + take_eq;
+        int k_incl = kept;
+        for (int o = 1; o < 32; o <<= 1) { int t = __shfl_up_sync(0xFFFFFFFFu, k_incl, o); if (lane >= o) k_incl += t; }
+        w_off[lane] = k_incl - kept;
+        w_eqb[lane] = eq_before;
+    }
+    __syncthreads();
+    int off = w_off[warp], eqb = w_eqb[warp];
+    int first_ev = n;
+    const uint32_t lt = (1u << lane) - 1u;
+    for (int j = a + lane; j < bend; j += 32) {
+        uint32_t key = j < b ? score_key(scores[j]) : 0u;
+        bool gt = j < b && key > thr, eq = j < b && key == thr && k > 0;
+        uint32_t beq = __ballot_sync(0xFFFFFFFFu, eq);
+        int rank = eqb + __popc(beq & lt);
+        bool keep = gt || (eq && rank < need_eq);
+        uint32_t bk = __ballot_sync(0xFFFFFFFFu, keep);
+        if (keep) srcmap[off + __popc(bk & lt)] = T_first + j;
+        if (j < b && !keep) first_ev = min(first_ev, j);
+        off += __popc(bk);
+        eqb += __popc(beq);
+    }
+    for (int o = 16; o > 0; o >>= 1) first_ev = min(first_ev, __shfl_xor_sync(0xFFFFFFFFu, first_ev, o));
+    if (lane == 0 && first_ev < n) atomicMin(&s_first_evicted, first_ev);
+    __syncthreads();
+    if (tid == 0) dscal[0] = min(T_first + s_first_evicted, T_c) >> 6;
+}
+
+// ---------------------------------------------------------------------------
+// Eq. 9-11 for keys.  One block per (new 64-token group, head): gather the
+// group's members as float32 (Eq. 12 for cached tokens, widening for fresh
+// ones), per-channel min/max over the tokens, parameters, codes, pack.
+// ---------------------------------------------------------------------------
+template <typename T, int BITS>
+__global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView dst, const T* __restrict__ Kf,
+                                                        int F, int n_old_new, int T_new, int T_first,
+                                                        const int* __restrict__ srcmap,
+                                                        const int* __restrict__ fz_dev, int fz_host,
+                                                        int g_base, int* __restrict__ status) {
+    constexpr int ROWB = XSV_D * BITS / 8;
+    constexpr int WPR = ROWB / 4;              // 32-bit words per row
+    constexpr int CPW = 32 / BITS;             // codes per word
+    constexpr int NMAX = (1 << BITS) - 1;
+    const int gi = g_base + blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
+    const int fz = fz_dev ? *fz_dev : fz_host;
+    const bool same = (src.kcodes == dst.kcodes);
+    const int p0 = gi * XSV_G;
+    const int cnt = min(XSV_G, T_new - p0);
+
+    if (gi < fz) {   // frozen: the group keeps its members, positions, codes and parameters
+        if (same) return;
+        const uint32_t* s = reinterpret_cast<const uint32_t*>(src.kcodes + ((size_t)h * src.cap + p0) * ROWB);
+        uint32_t* d = reinterpret_cast<uint32_t*>(dst.kcodes + ((size_t)h * dst.cap + p0) * ROWB);
+        for (int i = tid; i < XSV_G * WPR; i += 256) d[i] = s[i];
+        if (tid < 64) dst.kscale[((size_t)h * dst.capg + gi) * 64 + tid] = src.kscale[((size_t)h * src.capg + gi) * 64 + tid];
+        else if (tid < 128) dst.kzero[((size_t)h * dst.capg + gi) * 64 + tid - 64] = src.kzero[((size_t)h * src.capg + gi) * 64 + tid - 64];
+        return;
+    }
+
+    __shared__ float tile[XSV_G][XSV_D + 1];
+    __shared__ float smn[4][64], smx[4][64];
+    __shared__ float ss[64];
+    __shared__ int sz[64];
+
+    for (int i = tid; i < cnt * WPR; i += 256) {
+        const int m = i / WPR, j = i % WPR, p = p0 + m;
+        if (p < n_old_new) {
+            const int sp = (srcmap != nullptr && p >= T_first) ? srcmap[p - T_first] : p;
+            const uint32_t w = *reinterpret_cast<const uint32_t*>(src.kcodes + ((size_t)h * src.cap + sp) * ROWB + 4 * j);
+            const size_t mo = ((size_t)h * src.capg + (sp >> 6)) * 64 + j * CPW;
+#pragma unroll
+            for (int e = 0; e < CPW; ++e) {
+                int code = (int)((w >> (e * BITS)) & (uint32_t)NMAX);
+                tile[m][j * CPW + e] = xsv_dequant(code, src.kzero[mo + e], src.kscale[mo + e]);
+            }
+        } else {
+            const T* row = Kf + ((size_t)h * F + (p - n_old_new)) * XSV_D + j * CPW;
+#pragma unroll
+            for (int e = 0; e < CPW; ++e) tile[m][j * CPW + e] = xsv_to_float<T>(row[e]);
+        }
+    }
+    __syncthreads();
+    {
+        const int c = tid & 63, part = tid >> 6;
+        float mn = INFINITY, mx = -INFINITY;
+        for (int m = part; m < cnt; m += 4) {
+            float v = tile[m][c];
+            mn = fminf(mn, v);
+            mx = fmaxf(mx, v);
+        }
+        smn[part][c] = mn;
+        smx[part][c] = mx;
+    }
+    __syncthreads();
+    if (tid < 64) {
+        float mn = fminf(fminf(smn[0][tid], smn[1][tid]), fminf(smn[2][tid], smn[3][tid]));
+        float mx = fmaxf(fmaxf(smx[0][tid], smx[1][tid]), fmaxf(smx[2][tid], smx[3][tid]));
+        float s;
+        int z;
+        xsv_quant_params(mn, mx, NMAX, s, z, status);
+        ss[tid] = s;
+        sz[tid] = z;
+        dst.kscale[((size_t)h * dst.capg + gi) * 64 + tid] = s;
+        dst.kzero[((size_t)h * dst.capg + gi) * 64 + tid] = z;
+    }
+    __syncthreads();
+    for (int i = tid; i < cnt * WPR; i += 256) {
+        const int m = i / WPR, j = i % WPR;
+        uint32_t w = 0;
+#pragma unroll
+        for (int e = 0; e < CPW; ++e) {
+            const int c = j * CPW + e;
+            w |= (uint32_t)xsv_quant_code(tile[m][c], ss[c], sz[c], NMAX) << (e * BITS);
+        }
+        *reinterpret_cast<uint32_t*>(dst.kcodes + ((size_t)h * dst.cap + p0 + m) * ROWB + 4 * j) = w;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Values of kept tokens move verbatim: codes row, scale, zero-point, origin.
+// One thread per (head, new position, 16-byte piece).
+// ---------------------------------------------------------------------------
+template <int ROWB>
+__global__ void __launch_bounds__(256) gather_v_kernel(LayerView src, LayerView dst, int H, int n_old_new,
+                                                       int T_first, const int* __restrict__ srcmap) {
+    constexpr int PPR = ROWB / 16;
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    const long long total = (long long)H * n_old_new * PPR;
+    if (idx >= total) return;
+    const int piece = (int)(idx % PPR);
+    const long long hp = idx / PPR;
+    const int p = (int)(hp % n_old_new), h = (int)(hp / n_old_new);
+    const int sp = (srcmap != nullptr && p >= T_first) ? srcmap[p - T_first] : p;
+    const uint4* s = reinterpret_cast<const uint4*>(src.vcodes + ((size_t)h * src.cap + sp) * ROWB) + piece;
+    uint4* d = reinterpret_cast<uint4*>(dst.vcodes + ((size_t)h * dst.cap + p) * ROWB) + piece;
+    *d = *s;
+    if (piece == 0) {
+        if (dst.bits < 16) {
+            dst.vscale[(size_t)h * dst.cap + p] = src.vscale[(size_t)h * src.cap + sp];
+            dst.vzero[(size_t)h * dst.cap + p] = src.vzero[(size_t)h * src.cap + sp];
+        }
+        if (h == 0) dst.origin[p] = src.origin[sp];
+    }
+}
+
+// Same for raw 16-bit key rows (bits == 16).
+__global__ void __launch_bounds__(256) gather_kraw_kernel(LayerView src, LayerView dst, int H, int n_old_new,
+                                                          int T_first, const int* __restrict__ srcmap) {
+    constexpr int PPR = 8;
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    const long long total = (long long)H * n_old_new * PPR;
+    if (idx >= total) return;
+    const int piece = (int)(idx % PPR);
+    const long long hp = idx / PPR;
+    const int p = (int)(hp % n_old_new), h = (int)(hp / n_old_new);
+    const int sp = (srcmap != nullptr && p >= T_first) ? srcmap[p - T_first] : p;
+    const uint4* s = reinterpret_cast<const uint4*>(src.kcodes + ((size_t)h * src.cap + sp) * 128) + piece;
+    uint4* d = reinterpret_cast<uint4*>(dst.kcodes + ((size_t)h * dst.cap + p) * 128) + piece;
+    *d = *s;
+}
+
+// Append the fresh frame's raw rows of K and V (bits == 16) and their origins.
+__global__ void __launch_bounds__(256) append_raw_kernel(LayerView dst, const uint4* __restrict__ Kf,
+                                                         const uint4* __restrict__ Vf, int H, int F,
+                                                         int n_old_new, long long origin0) {
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    const long long total = (long long)H * F * 8;
+    if (idx >= total) return;
+    const int piece = (int)(idx % 8);
+    const long long hf = idx / 8;
+    const int f = (int)(hf % F), h = (int)(hf / F);
+    const size_t d = ((size_t)h * dst.cap + n_old_new + f) * 8 + piece;
+    reinterpret_cast<uint4*>(dst.kcodes)[d] = Kf[idx];
+    reinterpret_cast<uint4*>(dst.vcodes)[d] = Vf[idx];
+    if (h == 0 && piece == 0) dst.origin[n_old_new + f] = origin0 + f;
+}
+
+// ---------------------------------------------------------------------------
+// Eq. 9-11 for the fresh frame's values: one warp per (head, token) row of 64
+// channels, two channels per lane, shuffle reductions for min / max.
+// ---------------------------------------------------------------------------
+template <typename T, int BITS>
+__global__ void __launch_bounds__(256) quant_v_kernel(LayerView dst, const T* __restrict__ Vf, int H, int F,
+                                                      int n_old_new, long long origin0, int* __restrict__ status) {
+    constexpr int ROWB = XSV_D * BITS / 8;
+    constexpr int NMAX = (1 << BITS) - 1;
+    constexpr int LPW = 16 / BITS;            // lanes that share one 32-bit word
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (row >= (long long)H * F) return;
+    const int f = (int)(row % F), h = (int)(row / F);
+    const T* src = Vf + ((size_t)h * F + f) * XSV_D + 2 * lane;
+    const float x0 = xsv_to_float<T>(src[0]), x1 = xsv_to_float<T>(src[1]);
+    float mn = fminf(x0, x1), mx = fmaxf(x0, x1);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+    }
+    float s;
+    int z;
+    xsv_quant_params(mn, mx, NMAX, s, z, status);
+    const uint32_t c0 = (uint32_t)xsv_quant_code(x0, s, z, NMAX), c1 = (uint32_t)xsv_quant_code(x1, s, z, NMAX);
+    uint32_t w = (c0 | (c1 << BITS)) << (2 * BITS * (lane % LPW));
+#pragma unroll
+    for (int o = 1; o < LPW; o <<= 1) w |= __shfl_xor_sync(0xFFFFFFFFu, w, o);
+    const int p = n_old_new + f;
+    if (lane % LPW == 0)
+        *reinterpret_cast<uint32_t*>(dst.vcodes + ((size_t)h * dst.cap + p) * ROWB + 4 * (lane / LPW)) = w;
+    if (lane == 0) {
+        dst.vscale[(size_t)h * dst.cap + p] = s;
+        dst.vzero[(size_t)h * dst.cap + p] = z;
+        if (h == 0) dst.origin[p] = origin0 + f;
+    }
+}
+
+}  // namespace
+
+// ------------------------------ launchers ----------------------------------
+cudaError_t xsv_launch_qtilde(const void* Q, int dtype, int H, int F, int n_special, int g, float* qpart,
+                              cudaStream_t st) {
+    dim3 grid(XSV_QCHUNKS, H);
+    if (dtype == 0) qtilde_partial_kernel<__half><<<grid, 256, 0, st>>>((const __half*)Q, F, n_special, g, qpart);
+    else qtilde_partial_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)Q, F, n_special, g, qpart);
+    xsv_count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t xsv_launch_score(const LayerView& lv, int H, int T_first, int T_c, const float* qpart, float qnorm,
+                             float* scores, cudaStream_t st) {
+    const int n = T_c - T_first;
+    if (n <= 0) return cudaSuccess;
+    const int grid = (n + SCORE_TPB - 1) / SCORE_TPB;
+    const size_t smem = (64 + 2 * (size_t)H * SCORE_MAXG * 64) * sizeof(float);
+    cudaError_t e = cudaSuccess;
+#define XSV_SCORE(B)                                                                                       \
+    {                                                                                                      \
+        static bool attr_set = false;                                                                      \
+        if (!attr_set && smem > 48 * 1024) {                                                               \
+            e = cudaFuncSetAttribute(score_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+            if (e != cudaSuccess) return e;                                                                \
+            attr_set = true;                                                                               \
+        }                                                                                                  \
+        score_kernel<B><<<grid, SCORE_TPB, smem, st>>>(lv, H, T_first, T_c, qpart, qnorm, scores);         \
+    }
+    switch (lv.bits) {
+        case 2: XSV_SCORE(2) break;
+        case 4: XSV_SCORE(4) break;
+        case 8: XSV_SCORE(8) break;
+        default: return cudaErrorInvalidValue;
+    }
+#undef XSV_SCORE
+    xsv_count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t xsv_launch_score_raw(const LayerView& lv, int dtype, int H, int T_first, int T_c, const float* qpart,
+                                 float qnorm, float* scores, cudaStream_t st) {
+    const int n = T_c - T_first;
+    if (n <= 0) return cudaSuccess;
+    const int grid = (n + SCORE_TPB - 1) / SCORE_TPB;
+    if (dtype == 0) score_raw_kernel<__half><<<grid, SCORE_TPB, 0, st>>>(lv, H, T_first, T_c, qpart, qnorm, scores);
+    else score_raw_kernel<__nv_bfloat16><<<grid, SCORE_TPB, 0, st>>>(lv, H, T_first, T_c, qpart, qnorm, scores);
+    xsv_count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t xsv_launch_select(const float* scores, int n, int k, int T_first, int T_c, int* srcmap, int* dscal,
+                              cudaStream_t st) {
+    select_kernel<<<1, 1024, 0, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);
+    xsv_count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t xsv_launch_requant_k(const LayerView& src, const LayerView& dst, const void* Kf, int dtype, int H,
+                                 int F, int n_old_new, int T_new, int T_first, const int* srcmap,
+                                 const int* fz_dev, int fz_host, int* status, cudaStream_t st) {
+    const int ngroups = (T_new + XSV_G - 1) / XSV_G;
+    const int g0 = (fz_dev == nullptr && src.kcodes == dst.kcodes) ? fz_host : 0;   // in place: skip the frozen prefix
+    if (ngroups - g0 <= 0) return cudaSuccess;
+    dim3 grid(ngroups - g0, H);
+#define XSV_RQ(TT, B)                                                                                         \
+    requant_k_kernel<TT, B><<<grid, 256, 0, st>>>(src, dst, (const TT*)Kf, F, n_old_new, T_new, T_first, srcmap, \
+                                                  fz_dev, fz_host, g0, status)
+    if (dtype == 0) {
+        switch (src.bits) {
+            case 2: XSV_RQ(__half, 2); break;
+            case 4: XSV_RQ(__half, 4); break;
+            case 8: XSV_RQ(__half, 8); break;
+            default: return cudaErrorInvalidValue;
+        }
+    } else {
+        switch (src.bits) {
+            case 2: XSV_RQ(__nv_bfloat16, 2); break;
+            case 4: XSV_RQ(__nv_bfloat16, 4); break;
+            case 8: XSV_RQ(__nv_bfloat16, 8); break;
+            default: return cudaErrorInvalidValue;
+        }
+    }
+#undef XSV_RQ
+    xsv_count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t xsv_launch_gather_v(const LayerView& src, const LayerView& dst, int H, int n_old_new, int T_first,
+                                const int* srcmap, cudaStream_t st) {
+    if (n_old_new <= 0) return cudaSuccess;
+    const long long total = (long long)H * n_old_new * (src.rowb / 16);
+    const int grid = (int)((total + 255) / 256);
+    switch (src.rowb) {
+        case 16: gather_v_kernel<16><<<grid, 256, 0, st>>>(src, dst, H, n_old_new, T_first, srcmap); break;
+        case 32: gather_v_kernel<32><<<grid, 256, 0, st>>>(src, dst, H, n_old_new, T_first, srcmap); break;
+        case 64: gather_v_kernel<64><<<grid, 256, 0, st>>>(src, dst, H, n_old_new, T_first, srcmap); break;
+        case 128: gather_v_kernel<128><<<grid, 256, 0, st>>>(src, dst, H, n_old_new, T_first, srcmap); break;
+        default: return cudaErrorInvalidValue;
+    }
+    xsv_count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t xsv_launch_quant_v(const LayerView& dst, const void* Vf, int dtype, int H, int F, int n_old_new,
+                               long long origin0, int* status, cudaStream_t st) {
+    const int grid = (int)(((long long)H * F + 7) / 8);
+#define XSV_QV(TT, B) quant_v_kernel<TT, B><<<grid, 256, 0, st>>>(dst, (const TT*)Vf, H, F, n_old_new, origin0, status)
+    if (dtype == 0) {
+        switch (dst.bits) {
+            case 2: XSV_QV(__half, 2); break;
+            case 4: XSV_QV(__half, 4); break;
+            case 8: XSV_QV(__half, 8); break;
+            default: return cudaErrorInvalidValue;
+        }
+    } else {
+        switch (dst.bits) {
+            case 2: XSV_QV(__nv_bfloat16, 2); break;
+            case 4: XSV_QV(__nv_bfloat16, 4); break;
+            case 8: XSV_QV(__nv_bfloat16, 8); break;
+            default: return cudaErrorInvalidValue;
+        }
+    }
+#undef XSV_QV
+    xsv_count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t xsv_launch_raw_update(const LayerView& src, const LayerView& dst, const void* Kf, const void* Vf,
+                                  int H, int F, int n_old_new, int T_first, const int* srcmap, long long origin0,
+                                  cudaStream_t st) {
+    if (src.kcodes != dst.kcodes && n_old_new > 0) {
+        const long long total = (long long)H * n_old_new * 8;
+        const int grid = (int)((total + 255) / 256);
+        gather_kraw_kernel<<<grid, 256, 0, st>>>(src, dst, H, n_old_new, T_first, srcmap);
+        gather_v_kernel<128><<<grid, 256, 0, st>>>(src, dst, H, n_old_new, T_first, srcmap);
+        xsv_count_launch(2);
+    }
+    const long long total = (long long)H * F * 8;
+    append_raw_kernel<<<(int)((total + 255) / 256), 256, 0, st>>>(dst, (const uint4*)Kf, (const uint4*)Vf, H, F,
+                                                                  n_old_new, origin0);
+    xsv_count_launch();
+    return cudaGetLastError();
+}

@@ -1,0 +1,494 @@
+// Host layer of the xsv library: the cache object, its HBM layout and buffer
+// rotation, the closed-form length schedule and the per-step launch sequence.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/xsv.h"
+#include "xsv_kernels.h"
+
+static std::atomic<long long> g_launches{0};
+void xsv_count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct BufSet {
+    void* slab = nullptr;
+    LayerView view{};
+};
+
+struct PendingEvent {
+    int phase;
+    cudaEvent_t a, b;
+};
+
+}  // namespace
+
+struct xsv_cache {
+    int device = 0;
+    int layers = 0, H = 0, d = 0, bits = 0;
+    long long L_max = 0;
+    int n_special = 5, g = 16, G = 64;
+    int F = 0;               // tokens per frame (0 until known)
+    int dtype = -1;          // xsv_dtype of the first step
+    long long max_cache_tokens = 0;
+    long long cap = 0;       // capacity in tokens of each buffer set
+    bool allocated = false;
+    bool stepped = false;
+    int attn_impl = XSV_ATTN_AUTO;
+
+    std::vector<BufSet> bufs;          // layers + 1 (one spare for out-of-place compaction)
+    std::vector<int> buf_of_layer;
+    int spare = 0;
+    std::vector<long long> len, frames;
+
+    // scratch shared by all layers (steps are ordered on one stream)
+    float* qpart = nullptr;
+    float* scores = nullptr;
+    int* srcmap = nullptr;
+    int* dscal = nullptr;    // [0] frozen key groups of the current pruning step
+    int* status = nullptr;   // sticky device status word
+    void* scratch_slab = nullptr;
+    long long last_scores_n = 0;
+
+    // staging for xsv_step_host
+    void* stage = nullptr;
+    size_t stage_bytes = 0;
+
+    size_t bytes = 0;
+
+    bool profiling = false;
+    std::vector<PendingEvent> pending;
+    std::vector<cudaEvent_t> free_events;
+    double prof_ms[XSV_PHASE_COUNT] = {0, 0, 0, 0};
+    long long prof_launches[XSV_PHASE_COUNT] = {0, 0, 0, 0};
+};
+
+namespace {
+
+size_t bufset_bytes(const xsv_cache* c, long long cap, size_t off[7]) {
+    const int rowb = c->bits == 16 ? c->d * 2 : c->d * c->bits / 8;
+    const long long capg = (cap + XSV_G - 1) / XSV_G;
+    size_t o = 0;
+    off[0] = o; o = align_up(o + (size_t)c->H * cap * rowb, 256);                 // kcodes
+    off[1] = o; o = align_up(o + (size_t)c->H * cap * rowb, 256);                 // vcodes
+    off[2] = o; if (c->bits < 16) o = align_up(o + (size_t)c->H * capg * 64 * 4, 256);   // kscale
+    off[3] = o; if (c->bits < 16) o = align_up(o + (size_t)c->H * capg * 64 * 4, 256);   // kzero
+    off[4] = o; if (c->bits < 16) o = align_up(o + (size_t)c->H * cap * 4, 256);  // vscale
+    off[5] = o; if (c->bits < 16) o = align_up(o + (size_t)c->H * cap * 4, 256);  // vzero
+    off[6] = o; o = align_up(o + (size_t)cap * 8, 256);                           // origin
+    return o;
+}
+
+xsv_status allocate(xsv_cache* c) {
+    if (c->allocated) return XSV_OK;
+    const long long F = c->F;
+    long long cap;
+    if (c->L_max > 0) cap = c->L_max > 2 * F ? c->L_max : 2 * F;
+    else cap = c->max_cache_tokens > 0 ? c->max_cache_tokens : 16 * F;
+    if (cap < F) cap = F;
+    cap = (long long)align_up((size_t)cap, 128);   // whole attention tiles
+    c->cap = cap;
+    size_t off[7];
+    const size_t per = bufset_bytes(c, cap, off);
+    const int nb = c->layers + (c->L_max > 0 ? 1 : 0);
+    c->bufs.resize(nb);
+    size_t total = 0;
+    for (int i = 0; i < nb; ++i) {
+        void* p = nullptr;
+        if (cudaMalloc(&p, per) != cudaSuccess) { cudaGetLastError(); return XSV_ERR_OOM; }
+        if (cudaMemset(p, 0, per) != cudaSuccess) return XSV_ERR_CUDA;
+        BufSet& b = c->bufs[i];
+        b.slab = p;
+        uint8_t* base = (uint8_t*)p;
+        b.view.kcodes = base + off[0];
+        b.view.vcodes = base + off[1];
+        b.view.kscale = (float*)(base + off[2]);
+        b.view.kzero = (int*)(base + off[3]);
+        b.view.vscale = (float*)(base + off[4]);
+        b.view.vzero = (int*)(base + off[5]);
+        b.view.origin = (long long*)(base + off[6]);
+        b.view.cap = cap;
+        b.view.capg = (int)((cap + XSV_G - 1) / XSV_G);
+        b.view.rowb = c->bits == 16 ? c->d * 2 : c->d * c->bits / 8;
+        b.view.bits = c->bits;
+        total += per;
+    }
+    c->buf_of_layer.resize(c->layers);
+    for (int l = 0; l < c->layers; ++l) c->buf_of_layer[l] = l;
+    c->spare = c->layers;   // valid only when nb == layers + 1
+    // scratch: qpart | scores | srcmap | dscal | status
+    size_t so = 0;
+    const size_t o_q = so; so = align_up(so + (size_t)c->H * XSV_QCHUNKS * 64 * 4, 256);
+    const size_t o_s = so; so = align_up(so + (size_t)cap * 4, 256);
+    const size_t o_m = so; so = align_up(so + (size_t)cap * 4, 256);
+    const size_t o_d = so; so = align_up(so + 64, 256);
+    const size_t o_t = so; so = align_up(so + 64, 256);
+    if (cudaMalloc(&c->scratch_slab, so) != cudaSuccess) { cudaGetLastError(); return XSV_ERR_OOM; }
+    if (cudaMemset(c->scratch_slab, 0, so) != cudaSuccess) return XSV_ERR_CUDA;
+    uint8_t* sb = (uint8_t*)c->scratch_slab;
+    c->qpart = (float*)(sb + o_q);
+    c->scores = (float*)(sb + o_s);
+    c->srcmap = (int*)(sb + o_m);
+    c->dscal = (int*)(sb + o_d);
+    c->status = (int*)(sb + o_t);
+    c->bytes = total + so;
+    c->allocated = true;
+    return XSV_OK;
+}
+
+cudaEvent_t get_event(xsv_cache* c) {
+    if (!c->free_events.empty()) {
+        cudaEvent_t e = c->free_events.back();
+        c->free_events.pop_back();
+        return e;
+    }
+    cudaEvent_t e = nullptr;
+    cudaEventCreate(&e);
+    return e;
+}
+
+struct PhaseTimer {
+    xsv_cache* c;
+    cudaStream_t st;
+    int phase;
+    cudaEvent_t a = nullptr, b = nullptr;
+    long long launches0;
+    PhaseTimer(xsv_cache* c_, cudaStream_t st_, int phase_) : c(c_), st(st_), phase(phase_) {
+        launches0 = g_launches.load(std::memory_order_relaxed);
+        if (c->profiling) {
+            a = get_event(c);
+            b = get_event(c);
+            cudaEventRecord(a, st);
+        }
+    }
+    ~PhaseTimer() {
+        if (c->profiling) {
+            cudaEventRecord(b, st);
+            c->pending.push_back({phase, a, b});
+            c->prof_launches[phase] += g_launches.load(std::memory_order_relaxed) - launches0;
+        }
+    }
+};
+
+}  // namespace
+
+extern "C" {
+
+const char* xsv_strerror(xsv_status s) {
+    switch (s) {
+        case XSV_OK: return "ok";
+        case XSV_ERR_ARG: return "invalid argument";
+        case XSV_ERR_SHAPE: return "shape, dtype or alignment mismatch";
+        case XSV_ERR_ORDER: return "call out of order";
+        case XSV_ERR_OOM: return "out of memory";
+        case XSV_ERR_CUDA: return "CUDA runtime error";
+        case XSV_ERR_TIMEOUT: return "bounded device-side wait ran out";
+        case XSV_ERR_RANGE: return "zero-point outside the int32 range";
+        case XSV_ERR_CAPACITY: return "unbounded cache exceeded max_cache_tokens";
+    }
+    return "unknown status";
+}
+
+long long xsv_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+xsv_status xsv_cache_create(xsv_cache** out, int layers, int heads, int head_dim, long long budget_tokens, int bits) {
+    if (!out) return XSV_ERR_ARG;
+    *out = nullptr;
+    if (layers <= 0 || layers > 4096 || heads <= 0 || heads > 1024) return XSV_ERR_ARG;
+    if (head_dim != XSV_D) return XSV_ERR_ARG;
+    if (!(bits == 2 || bits == 4 || bits == 8 || bits == 16)) return XSV_ERR_ARG;
+    if (budget_tokens > (1LL << 30)) return XSV_ERR_ARG;
+    xsv_cache* c = new (std::nothrow) xsv_cache();
+    if (!c) return XSV_ERR_OOM;
+    if (cudaGetDevice(&c->device) != cudaSuccess) { delete c; cudaGetLastError(); return XSV_ERR_CUDA; }
+    c->layers = layers; c->H = heads; c->d = head_dim; c->bits = bits;
+    c->L_max = budget_tokens > 0 ? budget_tokens : 0;
+    c->len.assign(layers, 0);
+    c->frames.assign(layers, 0);
+    *out = c;
+    return XSV_OK;
+}
+
+xsv_status xsv_cache_set_options(xsv_cache* c, int n_special, int pool_group, int quant_group, int max_frame_tokens,
+                                 long long max_cache_tokens) {
+    if (!c) return XSV_ERR_ARG;
+    if (c->stepped || c->allocated) return XSV_ERR_ORDER;
+    if (pool_group == 0 || (quant_group >= 0 && quant_group != XSV_G)) return XSV_ERR_ARG;
+    if (max_frame_tokens > (1 << 24) || max_cache_tokens > (1LL << 30)) return XSV_ERR_ARG;
+    if (n_special >= 0) c->n_special = n_special;
+    if (pool_group > 0) c->g = pool_group;
+    if (max_cache_tokens >= 0) c->max_cache_tokens = max_cache_tokens;
+    if (max_frame_tokens > 0) {
+        if (c->n_special > max_frame_tokens) return XSV_ERR_ARG;
+        c->F = max_frame_tokens;
+        cudaSetDevice(c->device);
+        return allocate(c);
+    }
+    return XSV_OK;
+}
+
+xsv_status xsv_cache_set_attn_impl(xsv_cache* c, xsv_attn_impl impl) {
+    if (!c || impl < XSV_ATTN_AUTO || impl > XSV_ATTN_TC5) return XSV_ERR_ARG;
+    c->attn_impl = impl;
+    return XSV_OK;
+}
+
+xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const void* V, int n_tokens,
+                    xsv_dtype dtype, void* out, void* stream) {
+    if (!c || !Q || !K || !V || !out) return XSV_ERR_ARG;
+    if (layer < 0 || layer >= c->layers || n_tokens <= 0) return XSV_ERR_ARG;
+    if (dtype != XSV_F16 && dtype != XSV_BF16) return XSV_ERR_ARG;
+    if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)out) & 15) return XSV_ERR_SHAPE;
+    if (out == Q || out == K || out == V) return XSV_ERR_ARG;
+    if (c->F != 0 && n_tokens != c->F) return XSV_ERR_SHAPE;
+    if (c->dtype >= 0 && (int)dtype != c->dtype) return XSV_ERR_SHAPE;
+    if (c->n_special > n_tokens) return XSV_ERR_ARG;
+    long long min_frames = c->frames[0];
+    for (int l = 1; l < c->layers; ++l) min_frames = c->frames[l] < min_frames ? c->frames[l] : min_frames;
+    if (c->frames[layer] > min_frames) return XSV_ERR_ORDER;   // this layer already took the current frame
+
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!c->allocated) {
+        c->F = n_tokens;
+        cudaSetDevice(c->device);
+        xsv_status s = allocate(c);
+        if (s != XSV_OK) { c->F = 0; return s; }
+    }
+    const int F = c->F, H = c->H;
+    const long long T_c = c->len[layer];
+    const long long T = T_c + F;
+    const long long t = c->frames[layer] + 1;
+    const bool prune = t >= 2 && c->L_max > 0 && T > c->L_max;
+    if (!prune && T > c->cap) return XSV_ERR_CAPACITY;
+    c->dtype = (int)dtype;
+    c->stepped = true;
+
+    const int cur = c->buf_of_layer[layer];
+    const LayerView& lv = c->bufs[cur].view;
+    cudaError_t e;
+
+    // ---- Eq. 2 / Eq. 12: attention over [cache ; frame]
+    {
+        PhaseTimer pt(c, st, XSV_PHASE_ATTN);
+        e = cudaErrorNotSupported;
+        if (c->attn_impl != XSV_ATTN_MMA)
+            e = xsv_launch_attn_tc5(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, c->status, st);
+        if (e == cudaErrorNotSupported) {
+            if (c->attn_impl == XSV_ATTN_TC5) return XSV_ERR_ARG;
+            e = xsv_launch_attn_mma(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, st);
+        }
+        if (e != cudaSuccess) return XSV_ERR_CUDA;
+    }
+
+    const long long origin0 = (t - 1) * (long long)F;
+    if (prune) {
+        const int T_first = F;   // constant frame size: the first frame holds F tokens
+        const int n_mid = (int)(T_c - T_first);
+        const long long kk = c->L_max - T_first - F;
+        const int k = (int)(kk > 0 ? kk : 0);
+        const int n_old_new = T_first + k;
+        const int T_new = n_old_new + F;
+        const LayerView& dv = c->bufs[c->spare].view;
+        {   // ---- Eq. 3-7
+            PhaseTimer pt(c, st, XSV_PHASE_SCORE);
+            e = xsv_launch_qtilde(Q, (int)dtype, H, F, c->n_special, c->g, c->qpart, st);
+            if (e != cudaSuccess) return XSV_ERR_CUDA;
+            const int n_pooled = c->n_special + (F - c->n_special + c->g - 1) / c->g;
+            const float qnorm = 1.0f / ((float)H * (float)n_pooled);
+            if (c->bits == 16) e = xsv_launch_score_raw(lv, (int)dtype, H, T_first, (int)T_c, c->qpart, qnorm, c->scores, st);
+            else e = xsv_launch_score(lv, H, T_first, (int)T_c, c->qpart, qnorm, c->scores, st);
+            if (e != cudaSuccess) return XSV_ERR_CUDA;
+        }
+        {   // ---- Eq. 8
+            PhaseTimer pt(c, st, XSV_PHASE_SELECT);
+            e = xsv_launch_select(c->scores, n_mid, k, T_first, (int)T_c, c->srcmap, c->dscal, st);
+            if (e != cudaSuccess) return XSV_ERR_CUDA;
+        }
+        {   // ---- Eq. 9-11 on the new order [first ; kept ; current], written to the spare buffer
+            PhaseTimer pt(c, st, XSV_PHASE_QUANT);
+            if (c->bits == 16) {
+                e = xsv_launch_raw_update(lv, dv, K, V, H, F, n_old_new, T_first, c->srcmap, origin0, st);
+            } else {
+                e = xsv_launch_gather_v(lv, dv, H, n_old_new, T_first, c->srcmap, st);
+                if (e == cudaSuccess) e = xsv_launch_quant_v(dv, V, (int)dtype, H, F, n_old_new, origin0, c->status, st);
+                if (e == cudaSuccess)
+                    e = xsv_launch_requant_k(lv, dv, K, (int)dtype, H, F, n_old_new, T_new, T_first, c->srcmap, c->dscal, 0,
+                                             c->status, st);
+            }
+            if (e != cudaSuccess) return XSV_ERR_CUDA;
+        }
+        c->buf_of_layer[layer] = c->spare;
+        c->spare = cur;
+        c->len[layer] = T_new;
+        c->last_scores_n = n_mid;
+    } else {
+        // append in place: cached tokens keep their slots; the partial tail key
+        // group (if any) is rebuilt together with the fresh tokens
+        PhaseTimer pt(c, st, XSV_PHASE_QUANT);
+        if (c->bits == 16) {
+            e = xsv_launch_raw_update(lv, lv, K, V, H, F, (int)T_c, F, nullptr, origin0, st);
+        } else {
+            e = xsv_launch_quant_v(lv, V, (int)dtype, H, F, (int)T_c, origin0, c->status, st);
+            if (e == cudaSuccess)
+                e = xsv_launch_requant_k(lv, lv, K, (int)dtype, H, F, (int)T_c, (int)T, F, nullptr, nullptr,
+                                         (int)(T_c / XSV_G), c->status, st);
+        }
+        if (e != cudaSuccess) return XSV_ERR_CUDA;
+        c->len[layer] = T;
+        c->last_scores_n = 0;
+    }
+    c->frames[layer] = t;
+    return XSV_OK;
+}
+
+xsv_status xsv_step_host(xsv_cache* c, int layer, const void* Qh, const void* Kh, const void* Vh, int n_tokens,
+                         xsv_dtype dtype, void* out_h, void* stream) {
+    if (!c || !Qh || !Kh || !Vh || !out_h || n_tokens <= 0) return XSV_ERR_ARG;
+    if (c->F != 0 && n_tokens != c->F) return XSV_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t nb = (size_t)c->H * n_tokens * c->d * 2;
+    if (c->stage_bytes < 4 * nb) {
+        cudaSetDevice(c->device);
+        if (c->stage) { cudaStreamSynchronize(st); cudaFree(c->stage); c->bytes -= c->stage_bytes; c->stage = nullptr; c->stage_bytes = 0; }
+        if (cudaMalloc(&c->stage, 4 * nb) != cudaSuccess) { cudaGetLastError(); return XSV_ERR_OOM; }
+        c->stage_bytes = 4 * nb;
+        c->bytes += c->stage_bytes;
+    }
+    uint8_t* s = (uint8_t*)c->stage;
+    if (cudaMemcpyAsync(s, Qh, nb, cudaMemcpyHostToDevice, st) != cudaSuccess) return XSV_ERR_CUDA;
+    if (cudaMemcpyAsync(s + nb, Kh, nb, cudaMemcpyHostToDevice, st) != cudaSuccess) return XSV_ERR_CUDA;
+    if (cudaMemcpyAsync(s + 2 * nb, Vh, nb, cudaMemcpyHostToDevice, st) != cudaSuccess) return XSV_ERR_CUDA;
+    xsv_status r = xsv_step(c, layer, s, s + nb, s + 2 * nb, n_tokens, dtype, s + 3 * nb, stream);
+    if (r != XSV_OK) return r;
+    if (cudaMemcpyAsync(out_h, s + 3 * nb, nb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return XSV_ERR_CUDA;
+    return XSV_OK;
+}
+
+size_t xsv_cache_bytes(const xsv_cache* c) { return c ? c->bytes : 0; }
+
+size_t xsv_cache_layer_kv_bytes(const xsv_cache* c, int layer) {
+    if (!c || layer < 0 || layer >= c->layers) return 0;
+    const size_t T = (size_t)c->len[layer], H = c->H, d = c->d;
+    if (c->bits == 16) return 2 * H * T * d * 2;
+    const size_t groups = (T + XSV_G - 1) / XSV_G;
+    return 2 * H * T * d * c->bits / 8 + H * groups * d * 8 + H * T * 8;
+}
+
+void xsv_cache_destroy(xsv_cache* c) {
+    if (!c) return;
+    cudaSetDevice(c->device);
+    cudaDeviceSynchronize();
+    for (auto& b : c->bufs) if (b.slab) cudaFree(b.slab);
+    if (c->scratch_slab) cudaFree(c->scratch_slab);
+    if (c->stage) cudaFree(c->stage);
+    for (auto& p : c->pending) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
+    for (auto e : c->free_events) cudaEventDestroy(e);
+    delete c;
+}
+
+long long xsv_cache_len(const xsv_cache* c, int layer) {
+    if (!c || layer < 0 || layer >= c->layers) return -1;
+    return c->len[layer];
+}
+
+long long xsv_cache_frames(const xsv_cache* c, int layer) {
+    if (!c || layer < 0 || layer >= c->layers) return -1;
+    return c->frames[layer];
+}
+
+xsv_status xsv_cache_export_layer(xsv_cache* c, int layer, unsigned char* k_codes, float* k_scale, int* k_zero,
+                                  unsigned char* v_codes, float* v_scale, int* v_zero, long long* origin,
+                                  unsigned short* k_raw, unsigned short* v_raw, void* stream) {
+    if (!c || layer < 0 || layer >= c->layers) return XSV_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return XSV_ERR_CUDA;
+    const long long T = c->len[layer];
+    if (T == 0 || !c->allocated) return XSV_OK;
+    const LayerView& lv = c->bufs[c->buf_of_layer[layer]].view;
+    const int H = c->H, d = c->d, rowb = lv.rowb, bits = c->bits;
+    const long long groups = (T + XSV_G - 1) / XSV_G;
+    std::vector<uint8_t> tmp((size_t)T * rowb);
+    for (int pass = 0; pass < 2; ++pass) {
+        const uint8_t* dev = pass == 0 ? lv.kcodes : lv.vcodes;
+        unsigned char* codes = pass == 0 ? k_codes : v_codes;
+        unsigned short* raw = pass == 0 ? k_raw : v_raw;
+        if ((bits < 16 && !codes) || (bits == 16 && !raw)) continue;
+        for (int h = 0; h < H; ++h) {
+            if (cudaMemcpy(tmp.data(), dev + (size_t)h * lv.cap * rowb, (size_t)T * rowb, cudaMemcpyDeviceToHost) != cudaSuccess)
+                return XSV_ERR_CUDA;
+            if (bits == 16) {
+                memcpy(raw + (size_t)h * T * d, tmp.data(), (size_t)T * rowb);
+            } else {
+                const unsigned mask = (1u << bits) - 1u;
+                for (long long p = 0; p < T; ++p)
+                    for (int ch = 0; ch < d; ++ch) {
+                        const int bit = ch * bits;
+                        codes[((size_t)h * T + p) * d + ch] = (tmp[(size_t)p * rowb + bit / 8] >> (bit % 8)) & mask;
+                    }
+            }
+        }
+    }
+    if (bits < 16) {
+        for (int h = 0; h < H; ++h) {
+            if (k_scale && cudaMemcpy(k_scale + (size_t)h * groups * 64, lv.kscale + (size_t)h * lv.capg * 64, (size_t)groups * 64 * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return XSV_ERR_CUDA;
+            if (k_zero && cudaMemcpy(k_zero + (size_t)h * groups * 64, lv.kzero + (size_t)h * lv.capg * 64, (size_t)groups * 64 * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return XSV_ERR_CUDA;
+            if (v_scale && cudaMemcpy(v_scale + (size_t)h * T, lv.vscale + (size_t)h * lv.cap, (size_t)T * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return XSV_ERR_CUDA;
+            if (v_zero && cudaMemcpy(v_zero + (size_t)h * T, lv.vzero + (size_t)h * lv.cap, (size_t)T * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return XSV_ERR_CUDA;
+        }
+    }
+    if (origin && cudaMemcpy(origin, lv.origin, (size_t)T * 8, cudaMemcpyDeviceToHost) != cudaSuccess) return XSV_ERR_CUDA;
+    return XSV_OK;
+}
+
+xsv_status xsv_last_scores(xsv_cache* c, float* scores_host, long long cap, long long* n, void* stream) {
+    if (!c || !n) return XSV_ERR_ARG;
+    *n = c->last_scores_n;
+    if (c->last_scores_n == 0) return XSV_OK;
+    if (!scores_host || cap < c->last_scores_n) return XSV_ERR_ARG;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return XSV_ERR_CUDA;
+    if (cudaMemcpy(scores_host, c->scores, (size_t)c->last_scores_n * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return XSV_ERR_CUDA;
+    return XSV_OK;
+}
+
+xsv_status xsv_cache_status(xsv_cache* c, void* stream) {
+    if (!c) return XSV_ERR_ARG;
+    if (!c->allocated) return XSV_OK;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return XSV_ERR_CUDA;
+    int w = 0;
+    if (cudaMemcpy(&w, c->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return XSV_ERR_CUDA;
+    if (w & XSV_DEV_TIMEOUT) return XSV_ERR_TIMEOUT;
+    if (w & XSV_DEV_RANGE) return XSV_ERR_RANGE;
+    return XSV_OK;
+}
+
+xsv_status xsv_cache_set_profiling(xsv_cache* c, int on) {
+    if (!c) return XSV_ERR_ARG;
+    c->profiling = on != 0;
+    return XSV_OK;
+}
+
+xsv_status xsv_cache_profile_read(xsv_cache* c, double ms[XSV_PHASE_COUNT], long long launches[XSV_PHASE_COUNT], int reset) {
+    if (!c) return XSV_ERR_ARG;
+    for (auto& p : c->pending) {
+        if (cudaEventSynchronize(p.b) != cudaSuccess) return XSV_ERR_CUDA;
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, p.a, p.b) != cudaSuccess) return XSV_ERR_CUDA;
+        c->prof_ms[p.phase] += t;
+        c->free_events.push_back(p.a);
+        c->free_events.push_back(p.b);
+    }
+    c->pending.clear();
+    for (int i = 0; i < XSV_PHASE_COUNT; ++i) {
+        if (ms) ms[i] = c->prof_ms[i];
+        if (launches) launches[i] = c->prof_launches[i];
+        if (reset) { c->prof_ms[i] = 0; c->prof_launches[i] = 0; }
+    }
+    return XSV_OK;
+}
+
+}  // extern "C"

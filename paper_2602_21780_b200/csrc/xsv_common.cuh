@@ -1,0 +1,81 @@
+// Shared declarations of the xsv CUDA library: cache layout in HBM, the
+// per-layer view handed to kernels, small device helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#define XSV_D 64   // channels per head (head_dim)
+#define XSV_G 64   // quantisation group size (tokens for K, channels for V)
+
+// Bits of the sticky device status word.
+#define XSV_DEV_TIMEOUT 1
+#define XSV_DEV_RANGE 2
+
+// One layer's cache as the kernels see it.  All arrays live in one slab.
+//   kcodes/vcodes [H][cap][rowb] : packed codes of one (head, token) row, code c
+//                                  at bit offset c*bits of the row (little endian);
+//                                  rowb = 64*bits/8 bytes.  bits == 16: the raw
+//                                  16-bit elements.
+//   kscale/kzero  [H][capg][64]  : Eq. 10 parameters per channel per 64-token group.
+//   vscale/vzero  [H][cap]       : Eq. 10 parameters per token (64 channels).
+//   origin        [cap]          : frame_index * F + token_index of each slot.
+struct LayerView {
+    uint8_t* kcodes;
+    float* kscale;
+    int* kzero;
+    uint8_t* vcodes;
+    float* vscale;
+    int* vzero;
+    long long* origin;
+    long long cap;
+    int capg;
+    int rowb;
+    int bits;
+};
+
+template <typename T> __device__ __forceinline__ float xsv_to_float(T v);
+template <> __device__ __forceinline__ float xsv_to_float<__half>(__half v) { return __half2float(v); }
+template <> __device__ __forceinline__ float xsv_to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T xsv_from_float(float v);
+template <> __device__ __forceinline__ __half xsv_from_float<__half>(float v) { return __float2half_rn(v); }
+template <> __device__ __forceinline__ __nv_bfloat16 xsv_from_float<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// Pack two floats into one 32-bit register of two 16-bit values (lo = a).
+template <typename T> __device__ __forceinline__ uint32_t xsv_pack2(float a, float b);
+template <> __device__ __forceinline__ uint32_t xsv_pack2<__half>(float a, float b) {
+    __half2 h = __floats2half2_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+template <> __device__ __forceinline__ uint32_t xsv_pack2<__nv_bfloat16>(float a, float b) {
+    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+
+// Eq. 12: x~ = (code - z) * s, one float32 multiply.
+__device__ __forceinline__ float xsv_dequant(int code, int z, float s) {
+    return __fmul_rn(__int2float_rn(code - z), s);
+}
+
+// Eq. 10 in float32, one rounding per operation; degenerate groups
+// (s below the smallest normal) take s = |mn| (or 1 when mn == 0).
+__device__ __forceinline__ void xsv_quant_params(float mn, float mx, int n, float& s, int& z, int* status) {
+    s = __fdiv_rn(__fsub_rn(mx, mn), __int2float_rn(n));
+    if (!(s >= 1.17549435e-38f)) s = (mn != 0.f) ? fabsf(mn) : 1.f;
+    float zf = rintf(__fdiv_rn(-mn, s));
+    if (!(fabsf(zf) < 2147483648.f)) atomicOr(status, XSV_DEV_RANGE);
+    z = __float2int_rn(zf);   // saturates at the int32 limits
+}
+
+// Eq. 9: clamp(round(x / s) + z, 0, n), round = nearest-even.
+__device__ __forceinline__ int xsv_quant_code(float x, float s, int z, int n) {
+    int q = __float2int_rn(__fdiv_rn(x, s));   // saturating
+    long long v = (long long)q + (long long)z;
+    return (int)(v < 0 ? 0 : (v > n ? n : v));
+}
+
+// Launch counter (host side), bumped by every kernel launch of the library.
+void xsv_count_launch(int n = 1);

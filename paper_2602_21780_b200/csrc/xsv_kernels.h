@@ -1,0 +1,58 @@
+// Host-side launchers of the xsv kernels (one per phase of the step).
+#pragma once
+#include "xsv_common.cuh"
+
+// dtype: 0 = fp16, 1 = bf16 (xsv_dtype).
+
+// Eq. 3-4 folded by linearity: per-(head, chunk) partial sums of the pooling-weighted
+// queries; qpart [H * XSV_QCHUNKS][64].
+#define XSV_QCHUNKS 8
+cudaError_t xsv_launch_qtilde(const void* Q, int dtype, int H, int F, int n_special, int g,
+                              float* qpart, cudaStream_t st);
+
+// Eq. 5-7: scores[j] for the middle segment positions [T_first, T_c).
+cudaError_t xsv_launch_score(const LayerView& lv, int H, int T_first, int T_c, const float* qpart,
+                             float qnorm /* 1 / (H * N_pooled) */, float* scores, cudaStream_t st);
+
+// bits == 16: same scores from the raw 16-bit keys.
+cudaError_t xsv_launch_score_raw(const LayerView& lv, int dtype, int H, int T_first, int T_c,
+                                 const float* qpart, float qnorm, float* scores, cudaStream_t st);
+
+// Eq. 8: top-k of scores[0..n) (score descending, position ascending).  Writes
+// srcmap[0..k) = T_first + selected positions (ascending) and
+// dscal[0] = number of frozen key groups = min(first evicted position, T_c) / 64.
+cudaError_t xsv_launch_select(const float* scores, int n, int k, int T_first, int T_c, int* srcmap,
+                              int* dscal, cudaStream_t st);
+
+// Eq. 9-11 for keys: rebuild the key groups of the new cache order.
+//   new position p < n_old_new comes from cache position (p < T_first ? p : srcmap[p - T_first])
+//   (srcmap == nullptr: identity); p >= n_old_new is fresh token p - n_old_new.
+//   Groups below the frozen count (fz_dev ? *fz_dev : fz_host) are copied verbatim
+//   (skipped when src and dst are the same buffer).
+cudaError_t xsv_launch_requant_k(const LayerView& src, const LayerView& dst, const void* Kf, int dtype,
+                                 int H, int F, int n_old_new, int T_new, int T_first, const int* srcmap,
+                                 const int* fz_dev, int fz_host, int* status, cudaStream_t st);
+
+// Values: gather kept rows (codes, scale, zero-point, origin) into dst for new
+// positions [0, n_old_new); only needed when dst != src.
+cudaError_t xsv_launch_gather_v(const LayerView& src, const LayerView& dst, int H, int n_old_new,
+                                int T_first, const int* srcmap, cudaStream_t st);
+
+// Values: Eq. 9-11 per token for the fresh frame, written at new positions
+// [n_old_new, n_old_new + F); also writes their origin ids.
+cudaError_t xsv_launch_quant_v(const LayerView& dst, const void* Vf, int dtype, int H, int F,
+                               int n_old_new, long long origin0, int* status, cudaStream_t st);
+
+// bits == 16: gather / append raw 16-bit rows of K and V (no quantisation).
+cudaError_t xsv_launch_raw_update(const LayerView& src, const LayerView& dst, const void* Kf,
+                                  const void* Vf, int H, int F, int n_old_new, int T_first,
+                                  const int* srcmap, long long origin0, cudaStream_t st);
+
+// Eq. 2 + Eq. 12: out = softmax(Q [K~;K]^T / 8) [V~;V]; warp-level mma.sync kernel.
+cudaError_t xsv_launch_attn_mma(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V,
+                                void* out, int dtype, int H, int F, cudaStream_t st);
+
+// Same contract; tcgen05 + TMEM kernel.  Returns cudaErrorNotSupported for
+// shapes it does not cover.
+cudaError_t xsv_launch_attn_tc5(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V,
+                                void* out, int dtype, int H, int F, int* status, cudaStream_t st);

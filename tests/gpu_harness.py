@@ -1,0 +1,115 @@
+"""Step-locked comparison of the CUDA path (through the C ABI) with the CPU oracle.
+
+Before each checked step the GPU layer state is exported and loaded into the
+oracle; both run the step on the same inputs; then the outputs are compared:
+attention within 1e-2 * max|out_oracle|, scores within 1e-3 * max|S_oracle|,
+the kept set exactly (the oracle's Eq. 8 evaluated on the GPU's own scores),
+codes / scales / zero-points bit for bit."""
+import numpy as np
+import torch
+
+from oracle import xsv_oracle as orc
+from paper_2602_21780_b200 import binding, synth
+
+ATTN_TOL = 1e-2
+SCORE_TOL = 1e-3
+
+
+def torch_dtype(name):
+    return torch.float16 if name == "fp16" else torch.bfloat16
+
+
+def to_dev(x, dtype):
+    return torch.from_numpy(np.ascontiguousarray(x)).to("cuda:0", torch_dtype(dtype)).contiguous()
+
+
+def load_oracle_state(ref, st, frames_done, F):
+    if ref.bits == 16:
+        dt = "fp16" if ref._dtype == "fp16" else "bf16"
+        ref.load_state(frames_done, F, synth.from_bits16(st["Kraw"], dt), np.zeros((ref.H, 0, ref.d)),
+                       np.zeros((ref.H, 0, ref.d)), synth.from_bits16(st["Vraw"], dt),
+                       np.zeros((ref.H, 0, 1)), np.zeros((ref.H, 0, 1)), st["origin"])
+    else:
+        ref.load_state(frames_done, F, st["Kc"], st["Ks"], st["Kz"], st["Vc"], st["Vs"][..., None],
+                       st["Vz"][..., None], st["origin"])
+
+
+def check_state_invariants(st, bits, F, frames_done, L_max):
+    T = st["T"]
+    assert T == orc.expected_cache_len(frames_done, F, L_max)
+    o = st["origin"]
+    assert np.all(np.diff(o) > 0)
+    assert np.array_equal(o[:F], np.arange(F))
+    assert np.array_equal(o[-F:], (frames_done - 1) * F + np.arange(F))
+    if bits < 16:
+        n = (1 << bits) - 1
+        assert st["Kc"].max() <= n and st["Vc"].max() <= n
+        assert np.all(st["Ks"] > 0) and np.all(st["Vs"] > 0)
+
+
+def compare_states(st, ref, bits, tag):
+    assert st["T"] == ref.T, f"{tag}: length {st['T']} vs {ref.T}"
+    assert np.array_equal(st["origin"], ref.origin), f"{tag}: kept set differs"
+    if bits == 16:
+        dt = ref._dtype
+        assert np.array_equal(synth.from_bits16(st["Kraw"], dt), ref.Kc), f"{tag}: raw K differs"
+        assert np.array_equal(synth.from_bits16(st["Vraw"], dt), ref.Vc), f"{tag}: raw V differs"
+        return
+    for name, a, b in (("V codes", st["Vc"], ref.Vc), ("V zero", st["Vz"], ref.Vz[..., 0]),
+                       ("K codes", st["Kc"], ref.Kc), ("K zero", st["Kz"], ref.Kz)):
+        assert np.array_equal(a, b), f"{tag}: {name} differ at {np.argwhere(a != b)[:4].tolist()}"
+    assert np.array_equal(st["Vs"].view(np.uint32), ref.Vs[..., 0].view(np.uint32)), f"{tag}: V scales differ"
+    assert np.array_equal(st["Ks"].view(np.uint32), np.ascontiguousarray(ref.Ks).view(np.uint32)), f"{tag}: K scales differ"
+
+
+def run_stream(stream, frames, L_max, bits, check_steps=None, impl=binding.ATTN_AUTO, n_special=5, g=16,
+               frame_fn=None, max_cache_tokens=-1, layers=1, layer=0):
+    """Run `frames` steps on the GPU; verify the steps in check_steps (0-based; None = all).
+    Returns a dict of the worst errors seen."""
+    H, d, F, dtype = stream.H, stream.d, stream.F, stream.dtype
+    cache = binding.Cache(layers, H, d, L_max, bits)
+    cache.set_attn_impl(impl)
+    if (n_special, g) != (5, 16) or max_cache_tokens >= 0:
+        cache.set_options(n_special=n_special, pool_group=g, max_cache_tokens=max_cache_tokens)
+    ref = orc.LayerCache(H, d, L_max, bits, n_special=n_special, g=g)
+    ref._dtype = dtype
+    worst = dict(attn=0.0, score=0.0, pruned_steps=0, checked=0)
+    for t in range(frames):
+        q, k, v = frame_fn(t) if frame_fn else stream.frame(t)
+        Q, K, V = to_dev(q, dtype), to_dev(k, dtype), to_dev(v, dtype)
+        out = torch.empty_like(Q)
+        checked = check_steps is None or t in check_steps
+        if checked:
+            st0 = cache.export_layer(layer)
+            if t > 0:
+                check_state_invariants(st0, bits, F, t, L_max)
+            load_oracle_state(ref, st0, t, F)
+        for l in range(layers):            # other layers take the same inputs; only `layer` is verified
+            cache.step(l, Q, K, V, out)
+        torch.cuda.synchronize()
+        assert cache.len(layer) == orc.expected_cache_len(t + 1, F, L_max)
+        if not checked:
+            continue
+        S_gpu = cache.last_scores()
+        o_ref = ref.step(q, k, v, select_on=S_gpu.astype(np.float64) if S_gpu.size else None)
+        o_gpu = out.float().cpu().numpy().astype(np.float64)
+        assert np.all(np.isfinite(o_gpu)), f"step {t}: non-finite attention output"
+        e = float(np.max(np.abs(o_gpu - o_ref)) / np.max(np.abs(o_ref)))
+        worst["attn"] = max(worst["attn"], e)
+        assert e <= ATTN_TOL, f"step {t}: attention error {e:.3e} of max|out|"
+        if ref.last_scores is not None:
+            assert S_gpu.shape == ref.last_scores.shape, f"step {t}: score count"
+            es = float(np.max(np.abs(S_gpu - ref.last_scores)) / np.max(np.abs(ref.last_scores)))
+            worst["score"] = max(worst["score"], es)
+            worst["pruned_steps"] += 1
+            assert es <= SCORE_TOL, f"step {t}: score error {es:.3e} of max|S|"
+        else:
+            assert S_gpu.size == 0, f"step {t}: GPU pruned but the oracle did not"
+        compare_states(cache.export_layer(layer), ref, bits, f"step {t}")
+        worst["checked"] += 1
+    assert cache.status() == 0
+    worst["bytes"] = cache.bytes()
+    worst["kv_bytes"] = cache.layer_kv_bytes(layer)
+    assert worst["kv_bytes"] == ref.kv_bytes_packed()
+    cache.destroy()
+    return worst

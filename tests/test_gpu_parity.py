@@ -1,0 +1,125 @@
+"""CUDA path vs oracle, through the C ABI (run on the B200 machine: -m gpu)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2602_21780_b200 import binding, synth
+from tests.gpu_harness import run_stream
+
+pytestmark = pytest.mark.gpu
+
+IMPLS = [binding.ATTN_MMA, binding.ATTN_AUTO]
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_config0_every_step(impl):
+    c = synth.CONFIGS[0]
+    st = synth.config_stream(0)
+    w = run_stream(st, c["frames"], c["L_max"], c["bits"], impl=impl)
+    assert w["checked"] == 8 and w["pruned_steps"] == 4
+
+
+@pytest.mark.parametrize("bits", [2, 4, 8])
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_small_ragged_shapes(bits, dtype):
+    # F not a multiple of any tile, budget not a multiple of the group, ragged pooling tail
+    st = synth.Stream(H=3, d=64, F=75, dtype=dtype, layer=2)
+    w = run_stream(st, 7, 331, bits)
+    assert w["pruned_steps"] == 3
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_budget_below_two_frames_and_exact_fit(impl):
+    st = synth.Stream(H=2, d=64, F=130, dtype="bf16", layer=3)
+    run_stream(st, 5, 200, 4, impl=impl)            # L_max < 2F: k = 0, cache = first + current
+    st = synth.Stream(H=2, d=64, F=64, dtype="fp16", layer=4)
+    w = run_stream(st, 7, 256, 4, impl=impl)        # T == L_max at step 4: no prune; step 5 prunes
+    assert w["pruned_steps"] == 3
+
+
+def test_ties_are_broken_by_position():
+    # identical keys everywhere -> all scores equal -> the lowest positions of the middle are kept
+    base = synth.Stream(H=2, d=64, F=40, dtype="fp16", layer=5)
+
+    def frame(t):
+        q, k, v = base.frame(t)
+        k = np.broadcast_to(base.frame(0)[1][:, :1, :], k.shape).copy()
+        return q, k, v
+
+    w = run_stream(base, 6, 100, 4, frame_fn=frame)
+    assert w["pruned_steps"] == 4
+
+
+@pytest.mark.parametrize("L_max", [0, 150])
+def test_quantisation_off(L_max):
+    st = synth.Stream(H=2, d=64, F=50, dtype="bf16", layer=6)
+    run_stream(st, 6, L_max, 16, max_cache_tokens=400 if L_max == 0 else -1)
+
+
+def test_pooling_options_and_multi_layer():
+    st = synth.Stream(H=4, d=64, F=37, dtype="fp16", layer=7)
+    run_stream(st, 6, 100, 4, n_special=1, g=4, layers=3, layer=2)
+
+
+def test_drifting_stream_two_bits():
+    st = synth.Stream(H=16, d=64, F=261, dtype="bf16", layer=1, drift_rho=0.95)
+    w = run_stream(st, 8, 783, 2)
+    assert w["pruned_steps"] == 5
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_config1_sampled_steps(impl):
+    # paper shape: 1374 tokens/frame, budget 21984; verify the first step, the end of the ramp,
+    # the first pruning steps and a later steady-state step
+    c = synth.CONFIGS[1]
+    st = synth.config_stream(1)
+    w = run_stream(st, 20, c["L_max"], c["bits"], check_steps={0, 1, 15, 16, 17, 19}, impl=impl)
+    assert w["pruned_steps"] == 3
+
+
+def test_api_errors_and_bytes_constant():
+    c = binding.Cache(2, 16, 64, 600, 4)
+    Q = torch.randn(16, 261, 64, device="cuda", dtype=torch.float16)
+    out = torch.empty_like(Q)
+    lib = binding.load()
+    assert lib.xsv_step(c._h, 5, Q.data_ptr(), Q.data_ptr(), Q.data_ptr(), 261, 0, out.data_ptr(), None) == 1
+    assert lib.xsv_step(c._h, 0, Q.data_ptr(), Q.data_ptr(), Q.data_ptr(), 261, 0, Q.data_ptr(), None) == 1
+    assert lib.xsv_step(c._h, 0, Q.data_ptr() + 2, Q.data_ptr(), Q.data_ptr(), 261, 0, out.data_ptr(), None) == 2
+    c.step(0, Q, Q, Q, out)
+    with pytest.raises(binding.XsvError) as e:
+        c.step(0, Q, Q, Q, out)                       # layer 0 twice before layer 1
+    assert e.value.code == 3
+    with pytest.raises(binding.XsvError) as e:
+        c.set_options(n_special=3)                    # options after the first step
+    assert e.value.code == 3
+    Q2 = torch.randn(16, 100, 64, device="cuda", dtype=torch.float16)
+    assert lib.xsv_step(c._h, 1, Q2.data_ptr(), Q2.data_ptr(), Q2.data_ptr(), 100, 0, out.data_ptr(), None) == 2
+    assert lib.xsv_step(c._h, 1, Q.data_ptr(), Q.data_ptr(), Q.data_ptr(), 261, 1, out.data_ptr(), None) == 2
+    c.step(1, Q, Q, Q, out)
+    b0 = c.bytes()
+    for _ in range(6):
+        for l in range(2):
+            c.step(l, Q, Q, Q, out)
+    torch.cuda.synchronize()
+    assert c.bytes() == b0 and c.len(0) == 600 and c.status() == 0
+    c.destroy()
+
+
+def test_host_step_matches_device_step():
+    st = synth.Stream(H=4, d=64, F=90, dtype="bf16", layer=8)
+    a = binding.Cache(1, 4, 64, 300, 4)
+    b = binding.Cache(1, 4, 64, 300, 4)
+    for t in range(6):
+        q, k, v = (torch.from_numpy(x).to(torch.bfloat16) for x in st.frame(t))
+        Qh, Kh, Vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
+        oh = torch.empty_like(Qh).pin_memory()
+        a.step_host(0, Qh, Kh, Vh, oh)
+        Q, K, V = q.cuda(), k.cuda(), v.cuda()
+        od = torch.empty_like(Q)
+        b.step(0, Q, K, V, od)
+        torch.cuda.synchronize()
+        assert torch.equal(oh, od.cpu())
+    sa, sb = a.export_layer(0), b.export_layer(0)
+    for key in sa:
+        assert np.array_equal(sa[key], sb[key])
+    a.destroy(); b.destroy()
