@@ -120,6 +120,20 @@ xsv_status xsv_step_host(xsv_cache* c, int layer, const void* Q_host, const void
                          const void* V_host, int n_tokens, xsv_dtype dtype, void* out_host,
                          void* stream);
 
+/*
+ * Eq. 3-7 on their own: importance scores of `n_keys` keys for one frame's
+ * queries, without a cache object.
+ *   Q      : device, [heads][n_tokens][64], 16-bit (`dtype`).
+ *   keys   : device, [heads][n_keys][64], 16-bit, same dtype (un-quantised keys).
+ *   scores : device, float[n_keys]; scores[j] = mean_i (Q_bar K_bar^T)[i][j] with
+ *            Q_bar the head-averaged pooled queries (n_special rows kept, patch
+ *            rows averaged in groups of pool_group) and K_bar the head-averaged keys.
+ * Allocates and frees 32 KB of scratch per call, stream-ordered on `stream`.
+ */
+xsv_status xsv_importance_scores(const void* Q, const void* keys, int heads, int n_tokens,
+                                 long long n_keys, xsv_dtype dtype, int n_special, int pool_group,
+                                 float* scores, void* stream);
+
 /* Device bytes held now: codes, scales, zero-points, origin ids of all layer
  * buffers plus the spare buffer and scratch (section 4.6's memory figure). */
 size_t xsv_cache_bytes(const xsv_cache* c);

@@ -25,6 +25,7 @@ SYMBOLS = {
     "xsv_cache_set_attn_impl": (_i, [_vp, _i]),
     "xsv_step": (_i, [_vp, _i, _vp, _vp, _vp, _i, _i, _vp, _vp]),
     "xsv_step_host": (_i, [_vp, _i, _vp, _vp, _vp, _i, _i, _vp, _vp]),
+    "xsv_importance_scores": (_i, [_vp, _vp, _i, _i, _ll, _i, _i, _i, _vp, _vp]),
     "xsv_cache_bytes": (C.c_size_t, [_vp]),
     "xsv_cache_layer_kv_bytes": (C.c_size_t, [_vp, _i]),
     "xsv_cache_destroy": (None, [_vp]),
@@ -186,6 +187,16 @@ class Cache:
             self.destroy()
         except Exception:
             pass
+
+
+def importance_scores(Q, keys, n_special=5, pool_group=16, stream=None):
+    """xsv_importance_scores: Q [H, F, 64], keys [H, n_keys, 64] CUDA tensors -> float32 CUDA tensor [n_keys]."""
+    import torch
+    scores = torch.empty(keys.shape[1], device=keys.device, dtype=torch.float32)
+    _check(load().xsv_importance_scores(Q.data_ptr(), keys.data_ptr(), Q.shape[0], Q.shape[1], keys.shape[1],
+                                        _dtype_code(Q), n_special, pool_group, scores.data_ptr(),
+                                        _stream_ptr(stream)), "xsv_importance_scores")
+    return scores
 
 
 def kernel_launches():

@@ -369,6 +369,31 @@ xsv_status xsv_step_host(xsv_cache* c, int layer, const void* Qh, const void* Kh
     return XSV_OK;
 }
 
+xsv_status xsv_importance_scores(const void* Q, const void* keys, int heads, int n_tokens, long long n_keys,
+                                 xsv_dtype dtype, int n_special, int pool_group, float* scores, void* stream) {
+    if (!Q || !keys || !scores || heads <= 0 || n_tokens <= 0 || n_keys <= 0 || n_keys > (1LL << 30)) return XSV_ERR_ARG;
+    if (dtype != XSV_F16 && dtype != XSV_BF16) return XSV_ERR_ARG;
+    if (n_special < 0 || n_special > n_tokens || pool_group <= 0) return XSV_ERR_ARG;
+    if (((uintptr_t)Q | (uintptr_t)keys) & 15) return XSV_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    float* qpart = nullptr;
+    if (cudaMallocAsync((void**)&qpart, (size_t)heads * XSV_QCHUNKS * 64 * sizeof(float), st) != cudaSuccess) {
+        cudaGetLastError();
+        return XSV_ERR_OOM;
+    }
+    LayerView lv{};
+    lv.kcodes = (uint8_t*)const_cast<void*>(keys);
+    lv.cap = n_keys;
+    lv.rowb = XSV_D * 2;
+    lv.bits = 16;
+    const int n_pooled = n_special + (n_tokens - n_special + pool_group - 1) / pool_group;
+    const float qnorm = 1.0f / ((float)heads * (float)n_pooled);
+    cudaError_t e = xsv_launch_qtilde(Q, (int)dtype, heads, n_tokens, n_special, pool_group, qpart, st);
+    if (e == cudaSuccess) e = xsv_launch_score_raw(lv, (int)dtype, heads, 0, (int)n_keys, qpart, qnorm, scores, st);
+    cudaFreeAsync(qpart, st);
+    return e == cudaSuccess ? XSV_OK : XSV_ERR_CUDA;
+}
+
 size_t xsv_cache_bytes(const xsv_cache* c) { return c ? c->bytes : 0; }
 
 size_t xsv_cache_layer_kv_bytes(const xsv_cache* c, int layer) {

@@ -77,6 +77,22 @@ def test_config1_sampled_steps(impl):
     assert w["pruned_steps"] == 3
 
 
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_importance_scores_entry_point(dtype):
+    from oracle import xsv_oracle as orc
+    from tests.gpu_harness import to_dev
+    st = synth.Stream(H=16, d=64, F=1374, dtype=dtype, layer=9)
+    q, k, _ = st.frame(0)
+    keys = np.concatenate([k, st.frame(1)[1], st.frame(2)[1]], axis=1)[:, :3001]
+    S = binding.importance_scores(to_dev(q, dtype), to_dev(keys, dtype)).cpu().numpy()
+    ref = orc.importance_scores(q, keys, 5, 16)
+    assert np.max(np.abs(S - ref)) <= 1e-3 * np.max(np.abs(ref))
+    # pooling parameters reach the kernel
+    S2 = binding.importance_scores(to_dev(q, dtype), to_dev(keys, dtype), n_special=1, pool_group=7).cpu().numpy()
+    ref2 = orc.importance_scores(q, keys, 1, 7)
+    assert np.max(np.abs(S2 - ref2)) <= 1e-3 * np.max(np.abs(ref2))
+
+
 def test_api_errors_and_bytes_constant():
     c = binding.Cache(2, 16, 64, 600, 4)
     Q = torch.randn(16, 261, 64, device="cuda", dtype=torch.float16)
