@@ -52,7 +52,8 @@ typedef enum {
     XSV_ERR_CUDA = 5,    /* a CUDA runtime call failed                                */
     XSV_ERR_TIMEOUT = 6, /* a bounded device-side wait ran out (status word)          */
     XSV_ERR_RANGE = 7,   /* a zero-point left the int32 range (status word)           */
-    XSV_ERR_CAPACITY = 8 /* unbounded cache grew past max_cache_tokens                */
+    XSV_ERR_CAPACITY = 8,/* unbounded cache grew past max_cache_tokens                */
+    XSV_ERR_LIMIT = 9    /* size beyond the fixed maximum of a no-allocation entry point */
 } xsv_status;
 
 typedef enum { XSV_F16 = 0, XSV_BF16 = 1 } xsv_dtype;
@@ -133,6 +134,34 @@ xsv_status xsv_step_host(xsv_cache* c, int layer, const void* Q_host, const void
 xsv_status xsv_importance_scores(const void* Q, const void* keys, int heads, int n_tokens,
                                  long long n_keys, xsv_dtype dtype, int n_special, int pool_group,
                                  float* scores, void* stream);
+
+/*
+ * xsv_importance_scores for callers that must not allocate.  (The paper has no
+ * counterpart: this is a property of the library, not of the method.)
+ *
+ * Some code cannot call cudaMalloc, or anything that may: a frame loop with a
+ * latency bound (an allocation can synchronise the whole device), a process
+ * whose device memory has all been handed to its own pool, work issued while
+ * another thread is capturing a CUDA graph in global capture mode.  This entry point computes
+ * the same scores as xsv_importance_scores with the same kernels, but its
+ * scratch (the per-head partial sums of the pooled queries) is a fixed array
+ * inside the library's device image: 128 KB, present on every GPU that loads
+ * the library until the process exits.  It calls no cudaMalloc, cudaFree or
+ * other allocating routine; inputs and outputs stay the caller's.
+ *
+ *   Arguments: as xsv_importance_scores.
+ *   Limit    : heads <= 64; more returns XSV_ERR_LIMIT and launches nothing.
+ *   Set-up   : the first call on each device looks up the array's device
+ *              address (cudaGetSymbolAddress, with that device current).  Make
+ *              that first call outside any stream capture.
+ *   Sharing  : every call on a device uses the same array.  Contents left by an
+ *              earlier call are never read (each call rewrites all it uses), but
+ *              two calls that overlap on the GPU -- different streams, no
+ *              ordering between them -- race on it.  Order them.
+ */
+xsv_status xsv_importance_scores_static(const void* Q, const void* keys, int heads, int n_tokens,
+                                        long long n_keys, xsv_dtype dtype, int n_special,
+                                        int pool_group, float* scores, void* stream);
 
 /* Device bytes held now: codes, scales, zero-points, origin ids of all layer
  * buffers plus the spare buffer and scratch (section 4.6's memory figure). */

@@ -26,6 +26,7 @@ SYMBOLS = {
     "xsv_step": (_i, [_vp, _i, _vp, _vp, _vp, _i, _i, _vp, _vp]),
     "xsv_step_host": (_i, [_vp, _i, _vp, _vp, _vp, _i, _i, _vp, _vp]),
     "xsv_importance_scores": (_i, [_vp, _vp, _i, _i, _ll, _i, _i, _i, _vp, _vp]),
+    "xsv_importance_scores_static": (_i, [_vp, _vp, _i, _i, _ll, _i, _i, _i, _vp, _vp]),
     "xsv_cache_bytes": (C.c_size_t, [_vp]),
     "xsv_cache_layer_kv_bytes": (C.c_size_t, [_vp, _i]),
     "xsv_cache_destroy": (None, [_vp]),
@@ -197,6 +198,14 @@ def importance_scores(Q, keys, n_special=5, pool_group=16, stream=None):
                                         _dtype_code(Q), n_special, pool_group, scores.data_ptr(),
                                         _stream_ptr(stream)), "xsv_importance_scores")
     return scores
+
+
+def importance_scores_static(Q, keys, scores, n_special=5, pool_group=16, stream=None):
+    """xsv_importance_scores_static: as importance_scores, but the caller passes the output tensor
+    (float32 CUDA, [n_keys]) and the library allocates nothing.  Returns the status code."""
+    return int(load().xsv_importance_scores_static(Q.data_ptr(), keys.data_ptr(), Q.shape[0], Q.shape[1],
+                                                   keys.shape[1], _dtype_code(Q), n_special, pool_group,
+                                                   scores.data_ptr(), _stream_ptr(stream)))
 
 
 def kernel_launches():

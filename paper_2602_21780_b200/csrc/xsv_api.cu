@@ -190,6 +190,7 @@ const char* xsv_strerror(xsv_status s) {
         case XSV_ERR_TIMEOUT: return "bounded device-side wait ran out";
         case XSV_ERR_RANGE: return "zero-point outside the int32 range";
         case XSV_ERR_CAPACITY: return "unbounded cache exceeded max_cache_tokens";
+        case XSV_ERR_LIMIT: return "size exceeds the fixed maximum of this no-allocation entry point";
     }
     return "unknown status";
 }
