@@ -191,6 +191,8 @@ def main():
     ap.add_argument("--attn", default="auto", choices=["auto", "mma", "tc5"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--layers", type=int, default=LAYERS,
+                    help="layers in the stack (default 24 = the benchmark; fewer only for profiling a small case)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -198,6 +200,10 @@ def main():
     if args.impl == "reference":
         run_reference(args, rank)
         return
+    global LAYERS, WORKLOAD
+    if args.layers != LAYERS:
+        WORKLOAD = WORKLOAD.replace("24 layers", f"{args.layers} layers (profiling case, not the benchmark)")
+        LAYERS = args.layers
     if args.warmup < 3:
         args.warmup = 3
 
@@ -276,14 +282,16 @@ def main():
 
     # ---- roofline of the dominant kernel (attention), live CUDA-event durations
     peaks = measured_peaks()
-    attn_ms, attn_n = prof["attn"]
+    attn_ms, attn_launches = prof["attn"]
+    attn_n = args.steps * LAYERS                      # attention launches its main kernel once per layer-step
     T_all = L_MAX + F
     flops = 4.0 * F * T_all * D * H
     achieved = flops / (attn_ms / attn_n * 1e-3) / 1e12 if attn_n else None
     roofline = {"bound": "tensor", "kernel": "fused dequant+attention", "achieved": achieved,
                 "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"] if achieved else None,
                 "traffic": attn_traffic_bytes(), "peak_source": peaks["source"],
-                "flops_per_launch": flops, "avg_launch_ms": attn_ms / attn_n if attn_n else None}
+                "flops_per_launch": flops, "avg_launch_ms": attn_ms / attn_n if attn_n else None,
+                "kernels_per_launch": attn_launches / attn_n if attn_n else None}
     # the bandwidth-bound phases: algorithmic bytes per layer-step / live duration
     k_keep = L_MAX - 2 * F
     n_mid = L_MAX - F

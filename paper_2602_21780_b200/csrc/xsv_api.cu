@@ -48,6 +48,7 @@ struct xsv_cache {
 
     // scratch shared by all layers (steps are ordered on one stream)
     float* qpart = nullptr;
+    float* attn_ws = nullptr;   // parts of query tiles shared by several CTAs (tcgen05 attention)
     float* scores = nullptr;
     int* srcmap = nullptr;
     int* dscal = nullptr;    // [0] frozen key groups of the current pruning step
@@ -121,13 +122,14 @@ xsv_status allocate(xsv_cache* c) {
     c->buf_of_layer.resize(c->layers);
     for (int l = 0; l < c->layers; ++l) c->buf_of_layer[l] = l;
     c->spare = c->layers;   // valid only when nb == layers + 1
-    // scratch: qpart | scores | srcmap | dscal | status
+    // scratch: qpart | scores | srcmap | dscal | status | attention parts
     size_t so = 0;
     const size_t o_q = so; so = align_up(so + (size_t)c->H * XSV_QCHUNKS * 64 * 4, 256);
     const size_t o_s = so; so = align_up(so + (size_t)cap * 4, 256);
     const size_t o_m = so; so = align_up(so + (size_t)cap * 4, 256);
     const size_t o_d = so; so = align_up(so + 64, 256);
     const size_t o_t = so; so = align_up(so + 64, 256);
+    const size_t o_w = so; so = align_up(so + xsv_attn_tc5_workspace_bytes(), 256);
     if (cudaMalloc(&c->scratch_slab, so) != cudaSuccess) { cudaGetLastError(); return XSV_ERR_OOM; }
     if (cudaMemset(c->scratch_slab, 0, so) != cudaSuccess) return XSV_ERR_CUDA;
     uint8_t* sb = (uint8_t*)c->scratch_slab;
@@ -136,6 +138,7 @@ xsv_status allocate(xsv_cache* c) {
     c->srcmap = (int*)(sb + o_m);
     c->dscal = (int*)(sb + o_d);
     c->status = (int*)(sb + o_t);
+    c->attn_ws = (float*)(sb + o_w);
     c->bytes = total + so;
     c->allocated = true;
     return XSV_OK;
@@ -278,7 +281,7 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
         PhaseTimer pt(c, st, XSV_PHASE_ATTN);
         e = cudaErrorNotSupported;
         if (c->attn_impl != XSV_ATTN_MMA)
-            e = xsv_launch_attn_tc5(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, c->status, st);
+            e = xsv_launch_attn_tc5(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, c->attn_ws, c->status, st);
         if (e == cudaErrorNotSupported) {
             if (c->attn_impl == XSV_ATTN_TC5) return XSV_ERR_ARG;
             e = xsv_launch_attn_mma(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, st);

@@ -52,7 +52,12 @@ cudaError_t xsv_launch_raw_update(const LayerView& src, const LayerView& dst, co
 cudaError_t xsv_launch_attn_mma(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V,
                                 void* out, int dtype, int H, int F, cudaStream_t st);
 
-// Same contract; tcgen05 + TMEM kernel.  Returns cudaErrorNotSupported for
-// shapes it does not cover.
+// Same contract; tcgen05 + TMEM kernel (followed by a small kernel that merges
+// the parts of query tiles shared by several CTAs).  `workspace` holds those
+// parts: xsv_attn_tc5_workspace_bytes() bytes of device memory; nullptr returns
+// cudaErrorNotSupported.  A bounded wait that runs out sets XSV_DEV_TIMEOUT in
+// *status.
+size_t xsv_attn_tc5_workspace_bytes();
 cudaError_t xsv_launch_attn_tc5(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V,
-                                void* out, int dtype, int H, int F, int* status, cudaStream_t st);
+                                void* out, int dtype, int H, int F, float* workspace, int* status,
+                                cudaStream_t st);
