@@ -183,6 +183,7 @@ def run_reference(args, rank):
 
 
 def main():
+    global LAYERS, WORKLOAD
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=40)
@@ -200,7 +201,6 @@ def main():
     if args.impl == "reference":
         run_reference(args, rank)
         return
-    global LAYERS, WORKLOAD
     if args.layers != LAYERS:
         WORKLOAD = WORKLOAD.replace("24 layers", f"{args.layers} layers (profiling case, not the benchmark)")
         LAYERS = args.layers
