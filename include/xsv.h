@@ -216,6 +216,11 @@ long long xsv_kernel_launches(void);
 
 const char* xsv_strerror(xsv_status s);
 
+/* Text of the CUDA runtime error behind the calling thread's most recent
+ * XSV_ERR_CUDA from xsv_step / xsv_step_host / xsv_importance_scores
+ * ("no error" if there was none).  The pointer is to static storage. */
+const char* xsv_last_cuda_error(void);
+
 #ifdef __cplusplus
 }
 #endif

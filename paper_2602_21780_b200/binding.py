@@ -39,6 +39,7 @@ SYMBOLS = {
     "xsv_cache_profile_read": (_i, [_vp, C.POINTER(C.c_double), C.POINTER(_ll), _i]),
     "xsv_kernel_launches": (_ll, []),
     "xsv_strerror": (C.c_char_p, [_i]),
+    "xsv_last_cuda_error": (C.c_char_p, []),
 }
 
 _lib = None
@@ -62,7 +63,8 @@ def load():
 class XsvError(RuntimeError):
     def __init__(self, code, where):
         self.code = code
-        super().__init__(f"{where}: {load().xsv_strerror(code).decode()} (status {code})")
+        detail = f": {load().xsv_last_cuda_error().decode()}" if code == 5 else ""
+        super().__init__(f"{where}: {load().xsv_strerror(code).decode()}{detail} (status {code})")
 
 
 def _check(code, where):

@@ -121,6 +121,18 @@ __device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok;
 }
+// non-blocking test of a phase
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
 // Bounded wait.  On expiry (or once another thread gave up) it raises the abort
 // flag, records XSV_DEV_TIMEOUT and returns, so the kernel always terminates.
 __device__ __noinline__ void mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
@@ -199,6 +211,20 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16
         ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
           "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
         : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&v)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
 }
 __device__ __forceinline__ float ex2(float x) {
     float y;
@@ -333,199 +359,50 @@ __device__ __forceinline__ void dq_params(float s, int z, uint16_t& ah, uint16_t
     }
 }
 
-// ------------------------------------------------------------------ the kernel
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// 32 logits of one row -> 32 probabilities 2^(s * sc - m) packed as fp16 pairs;
+// accumulates their sum and the running maximum of the raw logits.
+__device__ __forceinline__ void softmax32(const uint32_t (&v)[32], float sc, float nm, float& mx, float& ls, uint32_t (&pk)[16]) {
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        const float s0 = __uint_as_float(v[i]), s1 = __uint_as_float(v[i + 1]);
+        mx = fmax3(mx, s0, s1);
+        const float p0 = ex2(fmaf(s0, sc, nm)), p1 = ex2(fmaf(s1, sc, nm));
+        ls += p0 + p1;
+        pk[i >> 1] = pack_h2(p0, p1);
+    }
+}
+
+// What every role needs to know about its CTA.
+struct Cta {
+    uint8_t* smem;            // 1024-byte aligned base of the dynamic shared memory
+    uint32_t smem_base;       // the same as a shared-window address
+    uint32_t bar_base;        // first mbarrier
+    uint32_t tmem_base;       // first allocated tensor-memory column
+    volatile int* abort_flag;
+    int b, u_first, u_last;   // CTA index, first and last unit of its span
+};
+
+// Producer warps: one token row of the kv tile per thread.  Kept out of line so
+// that its register allocation does not weigh on the softmax path.
 template <typename T, int BITS>
-__global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const Params p) {
-    constexpr int W = BITS == 16 ? 2 : 32 / BITS;     // channels per packed word
-    constexpr int ROWB = XSV_D * BITS / 8;            // bytes of one cached (head, token) row
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const uint32_t smem_base = smem_u32(smem);
-    const uint32_t bar_base = smem_base + OFF_BAR;
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_BAR + B_COUNT * 8);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_BAR + B_COUNT * 8 + 4);
-    auto BAR = [&](int i) { return bar_base + 8u * (uint32_t)i; };
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int b = blockIdx.x;
-    const long long tick0 = cta_tick(p, b), tick1 = cta_tick(p, b + 1);
-    if (tick0 >= tick1) return;                       // uniform: nothing to do, nothing allocated
-    const int u_first = unit_of_tick(p, tick0), u_last = unit_of_tick(p, tick1 - 1);
-
-    if (tid == 0) {
-        for (int i = 0; i < NSTAGE; ++i) {
-            mbar_init(BAR(B_KFULL + i), 128);
-            mbar_init(BAR(B_VFULL + i), 128);
-            mbar_init(BAR(B_EMPTY + i), 1);
-        }
-        for (int x = 0; x < 2; ++x) {
-            mbar_init(BAR(B_SFULL + x), 1);
-            mbar_init(BAR(B_SFREE + x), 128);
-            mbar_init(BAR(B_PREADY + x), 128);
-            mbar_init(BAR(B_PVDONE + x), 1);
-            mbar_init(BAR(B_QFULL + x), 128);
-        }
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 12) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(512u) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-
-    const T* Qg = reinterpret_cast<const T*>(p.Q);
+__device__ __noinline__ void producer_loop(const Params& p, const Cta c) {
+    constexpr int W = BITS == 16 ? 2 : 32 / BITS;
+    [[maybe_unused]] constexpr int ROWB = XSV_D * BITS / 8;
+    uint8_t* const smem = c.smem;
+    volatile int* const abort_flag = c.abort_flag;
+    const int b = c.b, u_first = c.u_first, u_last = c.u_last;
+    auto BAR = [&](int i) { return c.bar_base + 8u * (uint32_t)i; };
+    const int tid = threadIdx.x, lane = tid & 31;
     const T* Kg = reinterpret_cast<const T*>(p.K);
     const T* Vg = reinterpret_cast<const T*>(p.V);
-    T* Og = reinterpret_cast<T*>(p.out);
-    const int F = p.F, nkv = p.nkv, n_ct = p.n_ct;
-
-    if (warp < 8) {
-        // =============================================================== softmax + epilogue
-        const int X = warp >> 2;                       // query tile of this warpgroup
-        const int row = tid & 127;
-        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem_base + lane_base + (uint32_t)(X * 128);
-        const uint32_t tP = tmem_base + lane_base + 256u + (uint32_t)(X * 64);
-        const uint32_t tO = tmem_base + lane_base + 384u + (uint32_t)(X * 64);
-        uint8_t* sQ = smem + OFF_Q + X * TILE_BYTES;
-        const float SC = 0.125f * 1.4426950408889634f;   // 1/sqrt(64) * log2(e)
-        uint32_t cX = 0, uX = 0;
-        for (int u = u_first; u <= u_last; ++u) {
-            const Span sp = cta_span(p, b, u);
-            if (sp.kv0 >= sp.kv1) continue;
-            const int h = u / p.npair, mp = u - h * p.npair;
-            const int q0 = mp * 2 * BM + X * BM;
-            if (q0 >= F) continue;                     // second tile of the last pair may be empty
-            const int grow = q0 + row;
-            // ---- this unit's queries -> shared memory (all MMAs reading the previous unit's tile are complete:
-            //      the last S of that unit has been received)
-            row16_to_tile<T, W>(grow < F ? Qg + ((size_t)h * F + grow) * XSV_D : nullptr, sQ, row);
-            fence_async_smem();
-            mbar_arrive(BAR(B_QFULL + X));
-            ++uX;
-
-            float m_used = -INFINITY, l = 0.f;
-            for (int kv = sp.kv0; kv < sp.kv1; ++kv) {
-                const int cnt = kv < n_ct ? min(BN, p.T_c - kv * BN) : min(BN, F - (kv - n_ct) * BN);
-                const bool tail = cnt < BN;
-                mbar_wait(BAR(B_SFULL + X), cX & 1u, abort_flag, p.status);
-                tc_fence_after();
-                // ---- pass 1: row maximum
-                float mx = -INFINITY;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(tS + 32u * c, v);
-                    tc_wait_ld();
-                    if (tail) {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) if (32 * c + i < cnt) mx = fmaxf(mx, __uint_as_float(v[i]));
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
-                    }
-                }
-                const float m_new = mx * SC;
-                if (kv == sp.kv0) {
-                    m_used = m_new;                    // first tile of the span: the accumulator is overwritten, not rescaled
-                } else {
-                    // PV of the previous tile must be complete before P is overwritten or O rescaled
-                    mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, p.status);
-                    tc_fence_after();
-                    const bool need = m_new > m_used + RESCALE_THRESHOLD;
-                    if (__any_sync(0xFFFFFFFFu, need)) {
-                        const float alpha = need ? ex2(m_used - m_new) : 1.f;
-                        if (need) m_used = m_new;
-                        l *= alpha;
-#pragma unroll
-                        for (int c = 0; c < 2; ++c) {
-                            uint32_t o[32];
-                            tmem_ld32(tO + 32u * c, o);
-                            tc_wait_ld();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                            tmem_st32(tO + 32u * c, o);
-                        }
-                        tc_wait_st();
-                    }
-                }
-                // ---- pass 2: probabilities -> tensor memory (fp16), row sum
-                const float nm = -m_used;
-                float ls = 0.f;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t v[32];
-                    tmem_ld32(tS + 32u * c, v);
-                    tc_wait_ld();
-                    if (c == 3) {                      // S is in registers: the next QK^T may overwrite it
-                        tc_fence_before();
-                        mbar_arrive(BAR(B_SFREE + X));
-                    }
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        float p0 = ex2(fmaf(__uint_as_float(v[i]), SC, nm));
-                        float p1 = ex2(fmaf(__uint_as_float(v[i + 1]), SC, nm));
-                        if (tail) {
-                            if (32 * c + i >= cnt) p0 = 0.f;
-                            if (32 * c + i + 1 >= cnt) p1 = 0.f;
-                        }
-                        ls += p0 + p1;
-                        pk[i >> 1] = pack_h2(p0, p1);
-                    }
-                    tmem_st16(tP + 16u * c, pk);
-                }
-                l += ls;
-                tc_wait_st();
-                tc_fence_before();
-                mbar_arrive(BAR(B_PREADY + X));
-                ++cX;
-            }
-            // ---- epilogue of the span
-            mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, p.status);
-            tc_fence_after();
-            const bool full = sp.kv0 == 0 && sp.kv1 == nkv;
-            const float inv = 1.f / l;
-            float* part = p.part + ((size_t)b * 2 + (sp.kv0 > 0 ? 0 : 1)) * PART_STRIDE;
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t o[32];
-                tmem_ld32(tO + 32u * c, o);
-                tc_wait_ld();
-                if (full) {
-                    if (grow < F) {
-                        uint32_t w[16];
-#pragma unroll
-                        for (int q = 0; q < 16; ++q) {   // channels 32c + 2q, 32c + 2q + 1
-                            const float a = __uint_as_float(o[inv_perm<W>(32 * c + 2 * q) - 32 * c]) * inv;
-                            const float bb = __uint_as_float(o[inv_perm<W>(32 * c + 2 * q + 1) - 32 * c]) * inv;
-                            w[q] = xsv_pack2<T>(a, bb);
-                        }
-                        uint4* dst = reinterpret_cast<uint4*>(Og + ((size_t)h * F + grow) * XSV_D + 32 * c);
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) dst[q] = make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
-                    }
-                } else {
-                    float4* dst = reinterpret_cast<float4*>(part + (size_t)(X * BM + row) * 64 + 32 * c);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q)
-                        dst[q] = make_float4(__uint_as_float(o[inv_perm<W>(32 * c + 4 * q) - 32 * c]),
-                                             __uint_as_float(o[inv_perm<W>(32 * c + 4 * q + 1) - 32 * c]),
-                                             __uint_as_float(o[inv_perm<W>(32 * c + 4 * q + 2) - 32 * c]),
-                                             __uint_as_float(o[inv_perm<W>(32 * c + 4 * q + 3) - 32 * c]));
-                }
-            }
-            if (!full) {
-                float2* ml = reinterpret_cast<float2*>(part + 256 * 64);
-                ml[X * BM + row] = make_float2(m_used, l);
-            }
-            tc_fence_before();   // the accumulator has been read: orders these loads before this thread's next arrive
-        }
-    } else if (warp < 12) {
+    const int F = p.F, n_ct = p.n_ct;
+    {
         // =============================================================== producers
         const int t = tid - 256;                       // token row inside the kv tile
         uint16_t* sMeta = reinterpret_cast<uint16_t*>(smem + OFF_META);   // [buf][offset | scale | bias][group][64]
@@ -598,7 +475,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const Params p) {
                             }
                         }
                         fence_async_smem();
-                        mbar_arrive(BAR(B_KFULL + s));
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(BAR(B_KFULL + s));
                         // values: per-token parameters
                         {
                             uint16_t ah, sh, bh;
@@ -617,7 +495,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const Params p) {
                             }
                         }
                         fence_async_smem();
-                        mbar_arrive(BAR(B_VFULL + s));
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(BAR(B_VFULL + s));
                         done = true;
                     }
                 }
@@ -639,70 +518,330 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const Params p) {
                     }
                     row16_to_tile<T, W>(kr, sK, t);
                     fence_async_smem();
-                    mbar_arrive(BAR(B_KFULL + s));
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(BAR(B_KFULL + s));
                     row16_to_tile<T, W>(vr, sV, t);
                     fence_async_smem();
-                    mbar_arrive(BAR(B_VFULL + s));
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(BAR(B_VFULL + s));
                 }
             }
         }
-    } else if (lane == 0) {
-        // =============================================================== MMA issuer (one thread)
-        const uint32_t tS0 = tmem_base, tP0 = tmem_base + 256u, tO0 = tmem_base + 384u;
-        uint32_t it = 0, cT[2] = {0, 0}, uT[2] = {0, 0};
+    }
+}
+
+// Softmax warpgroups (warps 0-3: query tile A, warps 4-7: tile B) and the epilogue.
+template <typename T, int BITS>
+__device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
+    constexpr int W = BITS == 16 ? 2 : 32 / BITS;
+    uint8_t* const smem = cta.smem;
+    const uint32_t tmem_base = cta.tmem_base;
+    volatile int* const abort_flag = cta.abort_flag;
+    const int b = cta.b, u_first = cta.u_first, u_last = cta.u_last;
+    auto BAR = [&](int i) { return cta.bar_base + 8u * (uint32_t)i; };
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const T* Qg = reinterpret_cast<const T*>(p.Q);
+    T* Og = reinterpret_cast<T*>(p.out);
+    const int F = p.F, nkv = p.nkv, n_ct = p.n_ct;
+    {
+        // =============================================================== softmax + epilogue
+        const int X = warp >> 2;                       // query tile of this warpgroup
+        const int row = tid & 127;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem_base + lane_base + (uint32_t)(X * 128);
+        const uint32_t tP = tmem_base + lane_base + 256u + (uint32_t)(X * 64);
+        const uint32_t tO = tmem_base + lane_base + 384u + (uint32_t)(X * 64);
+        uint8_t* sQ = smem + OFF_Q + X * TILE_BYTES;
+        const float SC = 0.125f * 1.4426950408889634f;   // 1/sqrt(64) * log2(e)
+        uint32_t cX = 0, uX = 0;
         for (int u = u_first; u <= u_last; ++u) {
             const Span sp = cta_span(p, b, u);
             if (sp.kv0 >= sp.kv1) continue;
             const int h = u / p.npair, mp = u - h * p.npair;
+            const int q0 = mp * 2 * BM + X * BM;
+            if (q0 >= F) continue;                     // second tile of the last pair may be empty
+            const int grow = q0 + row;
+            // ---- this unit's queries -> shared memory (all MMAs reading the previous unit's tile are complete:
+            //      the last S of that unit has been received)
+            row16_to_tile<T, W>(grow < F ? Qg + ((size_t)h * F + grow) * XSV_D : nullptr, sQ, row);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(BAR(B_QFULL + X));
+            ++uX;
+
+            float m_used = -INFINITY, l = 0.f;
+            for (int kv = sp.kv0; kv < sp.kv1; ++kv) {
+                const int cnt = kv < n_ct ? min(BN, p.T_c - kv * BN) : min(BN, F - (kv - n_ct) * BN);
+                const bool tail = cnt < BN;
+                const bool first = kv == sp.kv0;
+                mbar_wait(BAR(B_SFULL + X), cX & 1u, abort_flag, p.status);
+                tc_fence_after();
+                float nm = -m_used, ls = 0.f, mx = -INFINITY;
+                if (!tail) {
+                    // ---- fast path: one pass with the row maximum in use (stale by at most the threshold).
+                    //      Probabilities go to tensor memory as fp16 while this tile's true maximum is gathered;
+                    //      the next 32 columns are in flight while the current ones are processed.
+                    uint32_t va[32], vb[32];
+                    tmem_ld32(tS, va);
+                    tc_wait_ld();
+#pragma unroll 1
+                    for (int i = 0; i < 2; ++i) {
+                        uint32_t pk[16];
+                        tmem_ld32(tS + 64u * i + 32u, vb);
+                        softmax32(va, SC, nm, mx, ls, pk);
+                        if (i == 0 && !first) {
+                            // PV of the previous tile must be complete before P is overwritten (or O rescaled)
+                            mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, p.status);
+                            tc_fence_after();
+                        }
+                        tmem_st16(tP + 32u * i, pk);
+                        tc_wait_ld();
+                        if (i == 0) tmem_ld32(tS + 64u, va);
+                        softmax32(vb, SC, nm, mx, ls, pk);
+                        tmem_st16(tP + 32u * i + 16u, pk);
+                        if (i == 0) tc_wait_ld();
+                    }
+                } else {
+                    // ---- ragged tile: masked maximum first (compact loop)
+#pragma unroll 1
+                    for (int c = 0; c < 8; ++c) {
+                        uint32_t v[16];
+                        tmem_ld16(tS + 16u * c, v);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            if (16 * c + i < cnt) mx = fmaxf(mx, __uint_as_float(v[i]));
+                    }
+                    if (!first) {
+                        mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, p.status);
+                        tc_fence_after();
+                    }
+                }
+                const float m_new = mx * SC;
+                const bool need = m_new > m_used + RESCALE_THRESHOLD;   // always on the span's first tile
+                const bool any_need = __any_sync(0xFFFFFFFFu, need);
+                if (any_need) {
+                    // ---- rare: the maximum moved by more than the threshold; rescale the accumulator and the row sum
+                    const float alpha = need ? ex2(m_used - m_new) : 1.f;
+                    if (need) m_used = m_new;
+                    l *= alpha;
+                    if (!first) {
+#pragma unroll 1
+                        for (int c = 0; c < 4; ++c) {
+                            uint32_t o[16];
+                            tmem_ld16(tO + 16u * c, o);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                            tmem_st16(tO + 16u * c, o);
+                        }
+                    }
+                }
+                if (any_need || tail) {
+                    // ---- (re)compute this tile's probabilities with the maximum now in use, masking a ragged tail
+                    nm = -m_used;
+                    ls = 0.f;
+#pragma unroll 1
+                    for (int c = 0; c < 8; ++c) {
+                        uint32_t v[16], pk[8];
+                        tmem_ld16(tS + 16u * c, v);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 16; i += 2) {
+                            float s0 = __uint_as_float(v[i]), s1 = __uint_as_float(v[i + 1]);
+                            if (16 * c + i >= cnt) s0 = -INFINITY;
+                            if (16 * c + i + 1 >= cnt) s1 = -INFINITY;
+                            const float p0 = ex2(fmaf(s0, SC, nm)), p1 = ex2(fmaf(s1, SC, nm));
+                            ls += p0 + p1;
+                            pk[i >> 1] = pack_h2(p0, p1);
+                        }
+                        tmem_st8(tP + 8u * c, pk);
+                    }
+                }
+                // S has been read for good: the next QK^T may overwrite it
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(BAR(B_SFREE + X));
+                l += ls;
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(BAR(B_PREADY + X));
+                ++cX;
+            }
+            // ---- epilogue of the span
+            mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, p.status);
+            tc_fence_after();
+            const bool full = sp.kv0 == 0 && sp.kv1 == nkv;
+            const float inv = 1.f / l;
+            float* part = p.part + ((size_t)b * 2 + (sp.kv0 > 0 ? 0 : 1)) * PART_STRIDE;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {          // 16 positions = 16 channels (the permutation stays inside)
+                uint32_t o[16];
+                tmem_ld16(tO + 16u * c, o);
+                tc_wait_ld();
+                if (full) {
+                    if (grow < F) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {    // channels 16c + 2q, 16c + 2q + 1
+                            const float a = __uint_as_float(o[inv_perm<W>(16 * c + 2 * q) - 16 * c]) * inv;
+                            const float bb = __uint_as_float(o[inv_perm<W>(16 * c + 2 * q + 1) - 16 * c]) * inv;
+                            w[q] = xsv_pack2<T>(a, bb);
+                        }
+                        uint4* dst = reinterpret_cast<uint4*>(Og + ((size_t)h * F + grow) * XSV_D + 16 * c);
+                        dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+                        dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+                    }
+                } else {
+                    float4* dst = reinterpret_cast<float4*>(part + (size_t)(X * BM + row) * 64 + 16 * c);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        dst[q] = make_float4(__uint_as_float(o[inv_perm<W>(16 * c + 4 * q) - 16 * c]),
+                                             __uint_as_float(o[inv_perm<W>(16 * c + 4 * q + 1) - 16 * c]),
+                                             __uint_as_float(o[inv_perm<W>(16 * c + 4 * q + 2) - 16 * c]),
+                                             __uint_as_float(o[inv_perm<W>(16 * c + 4 * q + 3) - 16 * c]));
+                }
+            }
+            if (!full) {
+                float2* ml = reinterpret_cast<float2*>(part + 256 * 64);
+                ml[X * BM + row] = make_float2(m_used, l);
+            }
+            tc_fence_before();   // the accumulator has been read: orders these loads before this thread's next arrive
+        }
+    }
+}
+
+// MMA issuer: one thread.
+__device__ __noinline__ void mma_loop(const Params& p, const Cta c) {
+    const uint32_t smem_base = c.smem_base, tmem_base = c.tmem_base;
+    volatile int* const abort_flag = c.abort_flag;
+    const int b = c.b, u_first = c.u_first, u_last = c.u_last;
+    auto BAR = [&](int i) { return c.bar_base + 8u * (uint32_t)i; };
+    const int F = p.F;
+    {
+        // =============================================================== MMA issuer (one thread)
+        // Each query tile has its own strictly ordered sequence QK(0), QK(1), PV(0), QK(2), PV(1), ... in which
+        // every operation is gated by one barrier phase; the two sequences are merged by readiness, so that a
+        // tile never waits for the other tile's softmax.
+        const uint32_t tS0 = tmem_base, tP0 = tmem_base + 256u, tO0 = tmem_base + 384u;
+        uint32_t it0 = 0, cT[2] = {0, 0}, uT[2] = {0, 0};
+        for (int u = u_first; u <= u_last; ++u) {
+            const Span sp = cta_span(p, b, u);
+            if (sp.kv0 >= sp.kv1) continue;
+            const int h = u / p.npair, mp = u - h * p.npair;
+            (void)h;
             const int ntile = (mp * 2 * BM + BM < F) ? 2 : 1;
             const int n = sp.kv1 - sp.kv0;
             for (int x = 0; x < ntile; ++x) mbar_wait(BAR(B_QFULL + x), uT[x] & 1u, abort_flag, p.status);
-            auto issue_qk = [&](int x, uint32_t stage) {
-                const uint64_t qd = smem_desc(smem_base + OFF_Q + x * TILE_BYTES);
-                const uint64_t kd = smem_desc(smem_base + OFF_KV + stage * 2 * TILE_BYTES);
+            tc_fence_after();
+            int qk_next[2] = {0, 0}, pv_next[2] = {0, 0};
+            if (ntile == 1) { qk_next[1] = n; pv_next[1] = n; }
+            unsigned long long t_idle = 0;
+            uint32_t idle = 0;
+            while (pv_next[0] < n || pv_next[1] < n) {
+                bool progress = false;
 #pragma unroll
-                for (int k = 0; k < 4; ++k)        // 16 channels = 32 bytes inside the swizzled row
-                    mma_ss(tS0 + (uint32_t)(x * 128), qd + 2u * k, kd + 2u * k, IDESC_QK, k > 0);
-                tc_commit(BAR(B_SFULL + x));
-            };
-            // S of the span's first tile
-            {
-                const uint32_t s = it % NSTAGE;
-                mbar_wait(BAR(B_KFULL + s), (it / NSTAGE) & 1u, abort_flag, p.status);
-                for (int x = 0; x < ntile; ++x) {
-                    if (cT[x] > 0) mbar_wait(BAR(B_SFREE + x), (cT[x] - 1u) & 1u, abort_flag, p.status);
-                    tc_fence_after();
-                    issue_qk(x, s);
-                }
-            }
-            for (int j = 0; j < n; ++j, ++it) {
-                const uint32_t s = it % NSTAGE;
-                if (j + 1 < n) {                       // S of the next tile, as soon as this one has been read
-                    const uint32_t s1 = (it + 1) % NSTAGE;
-                    mbar_wait(BAR(B_KFULL + s1), ((it + 1) / NSTAGE) & 1u, abort_flag, p.status);
-                    for (int x = 0; x < ntile; ++x) {
-                        mbar_wait(BAR(B_SFREE + x), cT[x] & 1u, abort_flag, p.status);
-                        tc_fence_after();
-                        issue_qk(x, s1);
+                for (int x = 0; x < 2; ++x) {
+                    if (qk_next[x] < n) {
+                        const uint32_t itq = it0 + (uint32_t)qk_next[x], sq = itq % NSTAGE;
+                        const uint32_t c = cT[x] + (uint32_t)qk_next[x];     // number of this tile's S among all of the CTA's
+                        if (mbar_test(BAR(B_KFULL + sq), (itq / NSTAGE) & 1u) &&
+                            (c == 0 || mbar_test(BAR(B_SFREE + x), (c - 1u) & 1u))) {
+                            tc_fence_after();
+                            const uint64_t qd = smem_desc(smem_base + OFF_Q + x * TILE_BYTES);
+                            const uint64_t kd = smem_desc(smem_base + OFF_KV + sq * 2 * TILE_BYTES);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)        // 16 channels = 32 bytes inside the swizzled row
+                                mma_ss(tS0 + (uint32_t)(x * 128), qd + 2u * k, kd + 2u * k, IDESC_QK, k > 0);
+                            tc_commit(BAR(B_SFULL + x));
+                            ++qk_next[x];
+                            progress = true;
+                        }
+                    }
+                    if (pv_next[x] < qk_next[x]) {
+                        const int j = pv_next[x];
+                        const uint32_t itp = it0 + (uint32_t)j, sv = itp % NSTAGE;
+                        if (mbar_test(BAR(B_VFULL + sv), (itp / NSTAGE) & 1u) &&
+                            mbar_test(BAR(B_PREADY + x), (cT[x] + (uint32_t)j) & 1u)) {
+                            tc_fence_after();
+                            const uint64_t vd = smem_desc(smem_base + OFF_KV + sv * 2 * TILE_BYTES + TILE_BYTES);
+#pragma unroll
+                            for (int k = 0; k < 8; ++k)        // 16 tokens: 8 columns of P, 2048 bytes of V
+                                mma_ts(tO0 + (uint32_t)(x * 64), tP0 + (uint32_t)(x * 64) + 8u * k, vd + 128u * k, IDESC_PV,
+                                       (j > 0 || k > 0) ? 1u : 0u);
+                            tc_commit(BAR(B_PVDONE + x));
+                            ++pv_next[x];
+                            if (pv_next[x ^ 1] > j) tc_commit(BAR(B_EMPTY + sv));   // both tiles are through with this stage
+                            progress = true;
+                        }
                     }
                 }
-                mbar_wait(BAR(B_VFULL + s), (it / NSTAGE) & 1u, abort_flag, p.status);
-                const uint64_t vd = smem_desc(smem_base + OFF_KV + s * 2 * TILE_BYTES + TILE_BYTES);
-                for (int x = 0; x < ntile; ++x) {
-                    mbar_wait(BAR(B_PREADY + x), cT[x] & 1u, abort_flag, p.status);
-                    tc_fence_after();
-#pragma unroll
-                    for (int k = 0; k < 8; ++k)        // 16 tokens: 8 columns of P, 2048 bytes of V
-                        mma_ts(tO0 + (uint32_t)(x * 64), tP0 + (uint32_t)(x * 64) + 8u * k, vd + 128u * k, IDESC_PV,
-                               (j > 0 || k > 0) ? 1u : 0u);
-                    tc_commit(BAR(B_PVDONE + x));
-                    ++cT[x];
+                if (progress) {
+                    idle = 0;
+                } else {
+                    if (*abort_flag) break;
+                    if (++idle == 64u) t_idle = globaltimer();
+                    if (idle > 64u && (idle & 255u) == 0u && globaltimer() - t_idle > WAIT_LIMIT_NS) {
+                        *abort_flag = 1;
+                        atomicOr(p.status, XSV_DEV_TIMEOUT);
+                        break;
+                    }
                 }
-                tc_commit(BAR(B_EMPTY + s));
             }
-            for (int x = 0; x < ntile; ++x) ++uT[x];
+            it0 += (uint32_t)n;
+            for (int x = 0; x < ntile; ++x) { cT[x] += (uint32_t)n; ++uT[x]; }
         }
     }
+}
+
+// ------------------------------------------------------------------ the kernel
+template <typename T, int BITS>
+__global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_constant__ Params p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t bar_base = smem_base + OFF_BAR;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_BAR + B_COUNT * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_BAR + B_COUNT * 8 + 4);
+    auto BAR = [&](int i) { return bar_base + 8u * (uint32_t)i; };
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int b = blockIdx.x;
+    const long long tick0 = cta_tick(p, b), tick1 = cta_tick(p, b + 1);
+    if (tick0 >= tick1) return;                       // uniform: nothing to do, nothing allocated
+    const int u_first = unit_of_tick(p, tick0), u_last = unit_of_tick(p, tick1 - 1);
+
+    if (tid == 0) {
+        for (int i = 0; i < NSTAGE; ++i) {
+            mbar_init(BAR(B_KFULL + i), 4);     // one arrival per producer warp
+            mbar_init(BAR(B_VFULL + i), 4);
+            mbar_init(BAR(B_EMPTY + i), 1);
+        }
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(BAR(B_SFULL + x), 1);
+            mbar_init(BAR(B_SFREE + x), 4);     // one arrival per softmax warp
+            mbar_init(BAR(B_PREADY + x), 4);
+            mbar_init(BAR(B_PVDONE + x), 1);
+            mbar_init(BAR(B_QFULL + x), 4);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 12) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const Cta cta{smem, smem_base, bar_base, tmem_base, abort_flag, b, u_first, u_last};
+
+    if (warp < 8) softmax_loop<T, BITS>(p, cta);
+    else if (warp < 12) producer_loop<T, BITS>(p, cta);
+    else if (lane == 0) mma_loop(p, cta);
     tc_fence_before();
     __syncthreads();
     if (warp == 12) {

@@ -12,7 +12,16 @@
 static std::atomic<long long> g_launches{0};
 void xsv_count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+static thread_local cudaError_t g_last_cuda = cudaSuccess;
+
 namespace {
+
+// records the CUDA error behind an XSV_ERR_CUDA return (see xsv_last_cuda_error)
+inline xsv_status cuda_fail(cudaError_t e) {
+    g_last_cuda = e;
+    cudaGetLastError();   // clear the runtime's sticky copy of a launch-configuration error
+    return XSV_ERR_CUDA;
+}
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
@@ -198,6 +207,8 @@ const char* xsv_strerror(xsv_status s) {
     return "unknown status";
 }
 
+const char* xsv_last_cuda_error(void) { return cudaGetErrorString(g_last_cuda); }
+
 long long xsv_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
 
 xsv_status xsv_cache_create(xsv_cache** out, int layers, int heads, int head_dim, long long budget_tokens, int bits) {
@@ -286,7 +297,7 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
             if (c->attn_impl == XSV_ATTN_TC5) return XSV_ERR_ARG;
             e = xsv_launch_attn_mma(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, st);
         }
-        if (e != cudaSuccess) return XSV_ERR_CUDA;
+        if (e != cudaSuccess) return cuda_fail(e);
     }
 
     const long long origin0 = (t - 1) * (long long)F;
@@ -301,17 +312,17 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
         {   // ---- Eq. 3-7
             PhaseTimer pt(c, st, XSV_PHASE_SCORE);
             e = xsv_launch_qtilde(Q, (int)dtype, H, F, c->n_special, c->g, c->qpart, st);
-            if (e != cudaSuccess) return XSV_ERR_CUDA;
+            if (e != cudaSuccess) return cuda_fail(e);
             const int n_pooled = c->n_special + (F - c->n_special + c->g - 1) / c->g;
             const float qnorm = 1.0f / ((float)H * (float)n_pooled);
             if (c->bits == 16) e = xsv_launch_score_raw(lv, (int)dtype, H, T_first, (int)T_c, c->qpart, qnorm, c->scores, st);
             else e = xsv_launch_score(lv, H, T_first, (int)T_c, c->qpart, qnorm, c->scores, st);
-            if (e != cudaSuccess) return XSV_ERR_CUDA;
+            if (e != cudaSuccess) return cuda_fail(e);
         }
         {   // ---- Eq. 8
             PhaseTimer pt(c, st, XSV_PHASE_SELECT);
             e = xsv_launch_select(c->scores, n_mid, k, T_first, (int)T_c, c->srcmap, c->dscal, st);
-            if (e != cudaSuccess) return XSV_ERR_CUDA;
+            if (e != cudaSuccess) return cuda_fail(e);
         }
         {   // ---- Eq. 9-11 on the new order [first ; kept ; current], written to the spare buffer
             PhaseTimer pt(c, st, XSV_PHASE_QUANT);
@@ -324,7 +335,7 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
                     e = xsv_launch_requant_k(lv, dv, K, (int)dtype, H, F, n_old_new, T_new, T_first, c->srcmap, c->dscal, 0,
                                              c->status, st);
             }
-            if (e != cudaSuccess) return XSV_ERR_CUDA;
+            if (e != cudaSuccess) return cuda_fail(e);
         }
         c->buf_of_layer[layer] = c->spare;
         c->spare = cur;
@@ -342,7 +353,7 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
                 e = xsv_launch_requant_k(lv, lv, K, (int)dtype, H, F, (int)T_c, (int)T, F, nullptr, nullptr,
                                          (int)(T_c / XSV_G), c->status, st);
         }
-        if (e != cudaSuccess) return XSV_ERR_CUDA;
+        if (e != cudaSuccess) return cuda_fail(e);
         c->len[layer] = T;
         c->last_scores_n = 0;
     }
@@ -395,7 +406,7 @@ xsv_status xsv_importance_scores(const void* Q, const void* keys, int heads, int
     cudaError_t e = xsv_launch_qtilde(Q, (int)dtype, heads, n_tokens, n_special, pool_group, qpart, st);
     if (e == cudaSuccess) e = xsv_launch_score_raw(lv, (int)dtype, heads, 0, (int)n_keys, qpart, qnorm, scores, st);
     cudaFreeAsync(qpart, st);
-    return e == cudaSuccess ? XSV_OK : XSV_ERR_CUDA;
+    return e == cudaSuccess ? XSV_OK : cuda_fail(e);
 }
 
 size_t xsv_cache_bytes(const xsv_cache* c) { return c ? c->bytes : 0; }
