@@ -10,14 +10,14 @@
 // it writes its unnormalised accumulator with the row maxima and sums, and
 // attn_combine_kernel merges the parts in a fixed order (deterministic).
 //
-// Inside a CTA (13 warps):
+// Inside a CTA (16 warps):
 //   warps 0-3, 4-7 : softmax of query tile A / B, one query row per thread
 //                    (tensor-memory lane == row), online softmax in float32 with
 //                    lazy rescaling of the accumulator;
-//   warps 8-11     : producers: unpack the packed codes of a kv tile, dequantise
+//   warps 8-14     : producers: unpack the packed codes of a kv tile, dequantise
 //                    in registers (Eq. 12) and write fp16 tiles to shared memory
 //                    in the 128-byte-swizzled layout the MMA descriptors expect;
-//   warp 12        : one thread issues S = Q K^T (operands in shared memory) and
+//   warp 15        : one thread issues S = Q K^T (operands in shared memory) and
 //                    O += P V (P read from tensor memory, V from shared memory).
 // Stages are handed over with mbarriers; every wait is bounded and on expiry
 // sets XSV_DEV_TIMEOUT in the status word, after which all waits fall through
@@ -34,7 +34,8 @@ namespace {
 constexpr int BM = 128;            // query rows per tile
 constexpr int BN = 128;            // keys per kv tile
 constexpr int NSTAGE = 3;          // kv stages in shared memory
-constexpr int NTHREADS = 13 * 32;
+constexpr int NPROD = 7;              // producer warps
+constexpr int NTHREADS = (8 + NPROD + 1) * 32;   // 8 softmax warps, the producers, the MMA issuer
 constexpr uint32_t TILE_BYTES = 128u * 128u;   // 128 rows x 64 fp16
 constexpr int COST_PAIR = 4, COST_SINGLE = 3;  // relative cost of a kv step with two / one active query tile
 constexpr float RESCALE_THRESHOLD = 8.f;       // log2 units; below it the stale row maximum is kept
@@ -43,14 +44,15 @@ constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 // shared-memory map (from a 1024-byte aligned base)
 constexpr uint32_t OFF_Q = 0;                                  // 2 tiles
 constexpr uint32_t OFF_KV = 2 * TILE_BYTES;                    // NSTAGE x (K tile, V tile)
-constexpr uint32_t OFF_META = OFF_KV + NSTAGE * 2 * TILE_BYTES;   // key parameters as halves: [2 buf][offset | scale | bias][2 groups][64]
-constexpr uint32_t OFF_BAR = OFF_META + 2 * 3 * 2 * 64 * 2;
+constexpr uint32_t OFF_META = OFF_KV + NSTAGE * 2 * TILE_BYTES;   // key parameters as halves: [producer warp][offset | scale | bias][64]
+constexpr uint32_t OFF_BAR = OFF_META + 3072;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + 256 + 1024;          // + alignment slack
 
 // barrier slots (8 bytes each) inside the barrier block
 enum { B_KFULL = 0, B_VFULL = NSTAGE, B_EMPTY = 2 * NSTAGE, B_SFULL = 3 * NSTAGE, B_SFREE = B_SFULL + 2,
        B_PREADY = B_SFREE + 2, B_PVDONE = B_PREADY + 2, B_QFULL = B_PVDONE + 2, B_COUNT = B_QFULL + 2 };
 static_assert(B_COUNT * 8 + 16 <= 256, "barrier block");
+static_assert(NPROD * 3 * 64 * 2 <= 3072, "staging area of the key parameters");
 
 struct Params {
     LayerView lv;
@@ -305,23 +307,27 @@ __device__ __forceinline__ void row16_to_tile(const T* grow, uint8_t* tile, int 
     }
 }
 
-// Constants of the in-register unpack.  A code is moved (one shift, one
-// and-or) into the mantissa of an fp16 whose hidden bit is worth OFF and whose
-// unit in the last place at the code's position is 1, which reads as OFF + code.
-template <int BITS> struct Unpack;
-template <> struct Unpack<2> { static constexpr int TB = 8; static constexpr uint32_t MAGIC = 0x44004400u; static constexpr int OFF = 4; };
-template <> struct Unpack<4> { static constexpr int TB = 6; static constexpr uint32_t MAGIC = 0x4C004C00u; static constexpr int OFF = 16; };
-template <> struct Unpack<8> { static constexpr int TB = 0; static constexpr uint32_t MAGIC = 0x64006400u; static constexpr int OFF = 1024; };
+// In-register unpack.  The codes of one packed 32-bit word come out as pairs
+// (i, i + W/2), W = 32 / BITS codes per word.  A pair is masked (after at most
+// one shift per word half) into the mantissas of two fp16 whose exponent makes the
+// unit in the last place at the code's position worth 1: with the code at mantissa
+// bit TB the fp16 reads OFF + code, OFF = 1024 >> TB, exactly.
+template <int BITS> __host__ __device__ constexpr int unpack_shift(int i) {   // right shift applied to the word
+    return BITS == 4 ? (i < 2 ? 0 : 8) : BITS == 2 ? (i < 5 ? 0 : 10) : (i == 0 ? 0 : 8);
+}
+template <int BITS> __host__ __device__ constexpr int unpack_tb(int i) {      // mantissa bit of the code afterwards
+    return BITS == 4 ? 4 * (i & 1) : BITS == 2 ? (i < 5 ? 2 * i : 2 * (i - 5)) : 0;
+}
+template <int BITS> __host__ __device__ constexpr int unpack_off(int i) { return 1024 >> unpack_tb<BITS>(i); }
 
-// half2 (OFF + code_i, OFF + code_{i + W/2}) of packed word w; i is a compile-time
+// half2 (OFF_i + code_i, OFF_i + code_{i + W/2}) of packed word w; i is a compile-time
 // constant after unrolling
 template <int BITS>
 __device__ __forceinline__ uint32_t code_pair(uint32_t w, int i) {
-    const int sh = Unpack<BITS>::TB - i * BITS;
-    constexpr uint32_t m1 = ((1u << BITS) - 1u) << Unpack<BITS>::TB;
-    constexpr uint32_t mask = m1 | (m1 << 16);
-    const uint32_t x = sh >= 0 ? (w << sh) : (w >> (-sh));
-    return (x & mask) | Unpack<BITS>::MAGIC;
+    const int tb = unpack_tb<BITS>(i);
+    const uint32_t m1 = ((1u << BITS) - 1u) << tb;
+    const uint32_t magic = (uint32_t)(25 - tb) << 10;
+    return ((w >> unpack_shift<BITS>(i)) & (m1 | (m1 << 16))) | (magic | (magic << 16));
 }
 // Eq. 12 on a pair of codes: ((OFF + code) - a) * s + b.  For a zero-point z with
 // OFF + z exactly representable in fp16 (|OFF + z| <= 2047) a = OFF + z, b = 0:
@@ -332,9 +338,6 @@ template <int BITS>
 __device__ __forceinline__ uint32_t dq_pair(uint32_t w, int i, uint32_t a2, uint32_t s2, uint32_t b2) {
     return hfma2_u(hsub2_u(code_pair<BITS>(w, i), a2), s2, b2);
 }
-// the fp16 parameters (a, s, b) of dq_pair for scale s and zero-point z
-template <int BITS>
-__device__ __forceinline__ void dq_params(float s, int z, uint16_t& ah, uint16_t& sh, uint16_t& bh);
 
 __device__ __forceinline__ uint16_t f2h_sat(float x) {
     uint16_t h;
@@ -346,9 +349,9 @@ __device__ __forceinline__ float h2f(uint16_t h) {
     asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"(h));
     return f;
 }
-template <int BITS>
-__device__ __forceinline__ void dq_params(float s, int z, uint16_t& ah, uint16_t& sh, uint16_t& bh) {
-    const long long zo = (long long)z + Unpack<BITS>::OFF;
+// the fp16 parameters (a, s, b) of dq_pair for scale s, zero-point z and offset off
+__device__ __forceinline__ void dq_params(float s, int z, int off, uint16_t& ah, uint16_t& sh, uint16_t& bh) {
+    const int zo = z > 0x70000000 ? z : z + off;   // no overflow; such a z takes the far branch anyway
     sh = f2h_sat(s);
     if (zo >= -2047 && zo <= 2047) {
         ah = f2h_sat((float)zo);      // exact
@@ -388,145 +391,195 @@ struct Cta {
     int b, u_first, u_last;   // CTA index, first and last unit of its span
 };
 
-// Producer warps: one token row of the kv tile per thread.  Kept out of line so
-// that its register allocation does not weigh on the softmax path.
+// Walks the (unit, kv tile) steps of a CTA's span in order.
+struct TileIter {
+    int u, kv, kv1, h;
+    bool valid;
+};
+__device__ __forceinline__ void tile_iter_settle(const Params& p, int b, int u_last, TileIter& t) {
+    while (t.u <= u_last) {            // skip units in which this CTA has no step
+        const Span sp = cta_span(p, b, t.u);
+        if (sp.kv0 < sp.kv1) {
+            t.kv = sp.kv0;
+            t.kv1 = sp.kv1;
+            t.h = t.u / p.npair;
+            t.valid = true;
+            return;
+        }
+        ++t.u;
+    }
+    t.valid = false;
+}
+__device__ __forceinline__ void tile_iter_next(const Params& p, int b, int u_last, TileIter& t) {
+    if (++t.kv < t.kv1) return;
+    ++t.u;
+    tile_iter_settle(p, b, u_last, t);
+}
+
+// What a producer lane fetches from HBM for its row of one slab of a quantised
+// kv tile: the packed row, and either the row's value parameters or (key slab)
+// the key parameters of two channels, which the warp shares through shared memory.
+template <int NW>
+struct SlabRegs {
+    uint32_t w[NW];
+    float s0, s1;
+    int z0, z1;
+    bool valid;
+};
+
+// Producer warps.  A kv tile is eight slabs: 32 rows of keys (slabs 0-3) or of
+// values (slabs 4-7); slabs are dealt to the NPROD producer warps round-robin, one
+// row per lane.  The global loads of a warp's next slab are issued before its
+// current slab is unpacked, so that their latency is covered.  Kept out of line
+// so that its register allocation does not weigh on the softmax path.
 template <typename T, int BITS>
 __device__ __noinline__ void producer_loop(const Params& p, const Cta c) {
     constexpr int W = BITS == 16 ? 2 : 32 / BITS;
-    [[maybe_unused]] constexpr int ROWB = XSV_D * BITS / 8;
+    constexpr int UB = BITS == 16 ? 4 : BITS;        // the unpack code must compile for raw caches too
+    constexpr int ROWB = XSV_D * BITS / 8;
+    constexpr int NW = BITS == 16 ? 1 : ROWB / 4;    // packed words per row
+    constexpr int SPW = (32 / UB) / 2;               // half2 slots per word
     uint8_t* const smem = c.smem;
     volatile int* const abort_flag = c.abort_flag;
-    const int b = c.b, u_first = c.u_first, u_last = c.u_last;
+    const int b = c.b, u_last = c.u_last;
     auto BAR = [&](int i) { return c.bar_base + 8u * (uint32_t)i; };
-    const int tid = threadIdx.x, lane = tid & 31;
+    const int lane = threadIdx.x & 31, pw = (threadIdx.x >> 5) - 8;   // producer warp 0 .. NPROD-1
     const T* Kg = reinterpret_cast<const T*>(p.K);
     const T* Vg = reinterpret_cast<const T*>(p.V);
-    const int F = p.F, n_ct = p.n_ct;
-    {
-        // =============================================================== producers
-        const int t = tid - 256;                       // token row inside the kv tile
-        uint16_t* sMeta = reinterpret_cast<uint16_t*>(smem + OFF_META);   // [buf][offset | scale | bias][group][64]
-        uint32_t it = 0, cc = 0;                       // kv tiles, quantised kv tiles produced so far
-        for (int u = u_first; u <= u_last; ++u) {
-            const Span sp = cta_span(p, b, u);
-            if (sp.kv0 >= sp.kv1) continue;
-            const int h = u / p.npair;
-            for (int kv = sp.kv0; kv < sp.kv1; ++kv, ++it) {
-                const uint32_t s = it % NSTAGE;
-                uint8_t* sK = smem + OFF_KV + s * 2 * TILE_BYTES;
-                uint8_t* sV = sK + TILE_BYTES;
-                if (it >= NSTAGE) mbar_wait(BAR(B_EMPTY + s), ((it / NSTAGE) - 1u) & 1u, abort_flag, p.status);
-                const bool cached = kv < n_ct;
-                bool done = false;
-                if constexpr (BITS < 16) {
-                    if (cached) {
-                        constexpr int NW = ROWB / 4;   // packed words per row
-                        constexpr int SPW = W / 2;     // half2 slots per word
-                        const int tok = kv * BN + t;
-                        const bool valid = tok < p.T_c;
-                        const size_t r = (size_t)h * p.lv.cap + (valid ? tok : 0);
-                        uint32_t kw[NW], vw[NW];
-                        {
-                            const uint4* kp = reinterpret_cast<const uint4*>(p.lv.kcodes + r * ROWB);
-                            const uint4* vp = reinterpret_cast<const uint4*>(p.lv.vcodes + r * ROWB);
+    const int F = p.F, n_ct = p.n_ct, T_c = p.T_c;
+    int* const status = p.status;
+    const LayerView lv = p.lv;
+    uint16_t* const mA = reinterpret_cast<uint16_t*>(smem + OFF_META) + pw * 192;   // this warp's [offset | scale | bias][64]
+    uint16_t* const mS = mA + 64;
+    uint16_t* const mB = mA + 128;
+
+    // slab g of the CTA: tile g / 8, slab g % 8; this warp owns g = pw, pw + NPROD, ...
+    auto fetch = [&](const TileIter& ti, int sl, SlabRegs<NW>& r) {
+        if (BITS == 16 || !ti.valid || ti.kv >= n_ct) return;
+        const int tok = ti.kv * BN + (sl & 3) * 32 + lane;
+        r.valid = tok < T_c;
+        const size_t row = (size_t)ti.h * lv.cap + (r.valid ? tok : 0);
+        const uint4* src = reinterpret_cast<const uint4*>((sl < 4 ? lv.kcodes : lv.vcodes) + row * ROWB);
 #pragma unroll
-                            for (int i = 0; i < NW / 4; ++i) {
-                                const uint4 a = kp[i], c = vp[i];
-                                kw[4 * i] = a.x; kw[4 * i + 1] = a.y; kw[4 * i + 2] = a.z; kw[4 * i + 3] = a.w;
-                                vw[4 * i] = c.x; vw[4 * i + 1] = c.y; vw[4 * i + 2] = c.z; vw[4 * i + 3] = c.w;
-                            }
-                        }
-                        const float vs = p.lv.vscale[r];
-                        const int vz = p.lv.vzero[r];
-                        // this tile's key parameters as fp16 (offset, scale, bias), in shared-memory position order
-                        uint16_t* mA = sMeta + (cc & 1u) * 384;
-                        uint16_t* mS = mA + 128;
-                        uint16_t* mB = mA + 256;
-                        {
-                            const int g = t >> 6, pos = t & 63, ch = perm<W>(pos);
-                            const int grp = kv * 2 + g;
-                            float ks = 0.f;
-                            int kz = 0;
-                            if (grp * XSV_G < p.T_c) {
-                                ks = p.lv.kscale[((size_t)h * p.lv.capg + grp) * 64 + ch];
-                                kz = p.lv.kzero[((size_t)h * p.lv.capg + grp) * 64 + ch];
-                            }
-                            dq_params<BITS>(ks, kz, mA[g * 64 + pos], mS[g * 64 + pos], mB[g * 64 + pos]);
-                        }
-                        asm volatile("bar.sync 1, 128;" ::: "memory");
-                        ++cc;
-                        // keys: per-channel parameters of this row's 64-token group
-                        {
-                            const uint4* a4p = reinterpret_cast<const uint4*>(mA + (t >> 6) * 64);
-                            const uint4* s4p = reinterpret_cast<const uint4*>(mS + (t >> 6) * 64);
-                            const uint4* b4p = reinterpret_cast<const uint4*>(mB + (t >> 6) * 64);
+        for (int i = 0; i < NW / 4; ++i) {
+            const uint4 a = src[i];
+            r.w[4 * i] = a.x; r.w[4 * i + 1] = a.y; r.w[4 * i + 2] = a.z; r.w[4 * i + 3] = a.w;
+        }
+        if (sl < 4) {                       // key parameters of the channels at positions lane and lane + 32
+            const int grp = ti.kv * 2 + ((sl & 3) >> 1);
+            r.s0 = r.s1 = 0.f;
+            r.z0 = r.z1 = 0;
+            if (grp * XSV_G < T_c) {
+                const size_t m = ((size_t)ti.h * lv.capg + grp) * 64;
+                r.s0 = lv.kscale[m + perm<W>(lane)];
+                r.z0 = lv.kzero[m + perm<W>(lane)];
+                r.s1 = lv.kscale[m + perm<W>(lane + 32)];
+                r.z1 = lv.kzero[m + perm<W>(lane + 32)];
+            }
+        } else {
+            r.s0 = lv.vscale[row];
+            r.z0 = lv.vzero[row];
+        }
+    };
+
+    TileIter cur{c.u_first, 0, 0, 0, false}, nxt;
+    tile_iter_settle(p, b, u_last, cur);
+    uint32_t it = 0;                                // kv tile of `cur`
+    uint32_t g = (uint32_t)pw;                      // this warp's current slab
+    auto seek = [&](TileIter& ti, uint32_t& ti_it, uint32_t tile) {   // advance an iterator to kv tile `tile`
+        while (ti.valid && ti_it < tile) {
+            tile_iter_next(p, b, u_last, ti);
+            ++ti_it;
+        }
+    };
+    seek(cur, it, g >> 3);
+    SlabRegs<NW> rc{}, rn{};
+    fetch(cur, (int)(g & 7u), rc);
+    while (cur.valid) {
+        const int sl = (int)(g & 7u);
+        // the next slab of this warp: start its loads now
+        const uint32_t gn = g + NPROD;
+        nxt = cur;
+        uint32_t itn = it;
+        seek(nxt, itn, gn >> 3);
+        fetch(nxt, (int)(gn & 7u), rn);
+
+        const uint32_t st = it % NSTAGE;
+        uint8_t* tile = smem + OFF_KV + st * 2 * TILE_BYTES + (sl < 4 ? 0u : TILE_BYTES);
+        const int row = (sl & 3) * 32 + lane;
+        if (it >= NSTAGE) mbar_wait(BAR(B_EMPTY + st), ((it / NSTAGE) - 1u) & 1u, abort_flag, status);
+        const bool cached = cur.kv < n_ct;
+        if (BITS < 16 && cached) {
+            if (sl < 4) {
+                // keys: stage the group's per-channel parameters (fp16, position order), then unpack the row
+                __syncwarp();                      // the previous slab's reads of the staging area are over
+                dq_params(rc.s0, rc.z0, unpack_off<UB>((lane >> 1) % SPW), mA[lane], mS[lane], mB[lane]);
+                dq_params(rc.s1, rc.z1, unpack_off<UB>(((lane + 32) >> 1) % SPW), mA[lane + 32], mS[lane + 32], mB[lane + 32]);
+                __syncwarp();
+                const uint4* a4p = reinterpret_cast<const uint4*>(mA);
+                const uint4* s4p = reinterpret_cast<const uint4*>(mS);
+                const uint4* b4p = reinterpret_cast<const uint4*>(mB);
 #pragma unroll
-                            for (int ck = 0; ck < 8; ++ck) {   // 16-byte chunk = half2 slots 4ck .. 4ck+3
-                                const uint4 a4 = a4p[ck], s4 = s4p[ck], b4 = b4p[ck];
-                                const uint32_t av[4] = {a4.x, a4.y, a4.z, a4.w}, sv[4] = {s4.x, s4.y, s4.z, s4.w},
-                                               bv[4] = {b4.x, b4.y, b4.z, b4.w};
-                                uint32_t o[4];
+                for (int ck = 0; ck < 8; ++ck) {   // 16-byte chunk = half2 slots 4ck .. 4ck+3
+                    const uint4 a4 = a4p[ck], s4 = s4p[ck], b4 = b4p[ck];
+                    const uint32_t av[4] = {a4.x, a4.y, a4.z, a4.w}, sv[4] = {s4.x, s4.y, s4.z, s4.w},
+                                   bv[4] = {b4.x, b4.y, b4.z, b4.w};
+                    uint32_t o[4];
 #pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    const int slot = 4 * ck + q;
-                                    o[q] = valid ? dq_pair<BITS>(kw[slot / SPW], slot % SPW, av[q], sv[q], bv[q]) : 0u;
-                                }
-                                *reinterpret_cast<uint4*>(sK + swz(t, ck)) = make_uint4(o[0], o[1], o[2], o[3]);
-                            }
-                        }
-                        fence_async_smem();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(BAR(B_KFULL + s));
-                        // values: per-token parameters
-                        {
-                            uint16_t ah, sh, bh;
-                            dq_params<BITS>(vs, vz, ah, sh, bh);
-                            const uint32_t a1 = (uint32_t)ah | ((uint32_t)ah << 16), s1 = (uint32_t)sh | ((uint32_t)sh << 16),
-                                           b1 = (uint32_t)bh | ((uint32_t)bh << 16);
+                    for (int q = 0; q < 4; ++q) {
+                        const int slot = 4 * ck + q;
+                        o[q] = dq_pair<UB>(rc.w[(slot / SPW) % NW], slot % SPW, av[q], sv[q], bv[q]);
+                    }
+                    *reinterpret_cast<uint4*>(tile + swz(row, ck)) = make_uint4(o[0], o[1], o[2], o[3]);
+                }
+            } else {
+                // values: the row's own parameters, one offset variant per code position inside a word
+                uint32_t a2[SPW], s2, b2[SPW];
+                {
+                    uint16_t ah, sh, bh;
 #pragma unroll
-                            for (int ck = 0; ck < 8; ++ck) {
-                                uint32_t o[4];
-#pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    const int slot = 4 * ck + q;
-                                    o[q] = valid ? dq_pair<BITS>(vw[slot / SPW], slot % SPW, a1, s1, b1) : 0u;
-                                }
-                                *reinterpret_cast<uint4*>(sV + swz(t, ck)) = make_uint4(o[0], o[1], o[2], o[3]);
-                            }
-                        }
-                        fence_async_smem();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(BAR(B_VFULL + s));
-                        done = true;
+                    for (int i = 0; i < SPW; ++i) {
+                        dq_params(rc.s0, rc.z0, unpack_off<UB>(i), ah, sh, bh);
+                        a2[i] = (uint32_t)ah | ((uint32_t)ah << 16);
+                        b2[i] = (uint32_t)bh | ((uint32_t)bh << 16);
+                        s2 = (uint32_t)sh | ((uint32_t)sh << 16);
                     }
                 }
-                if (!done) {
-                    // raw 16-bit rows: the fresh frame, or a cache kept unquantised (bits == 16)
-                    const T *kr = nullptr, *vr = nullptr;
-                    if (cached) {
-                        const int tok = kv * BN + t;
-                        if (tok < p.T_c) {
-                            kr = reinterpret_cast<const T*>(p.lv.kcodes) + ((size_t)h * p.lv.cap + tok) * XSV_D;
-                            vr = reinterpret_cast<const T*>(p.lv.vcodes) + ((size_t)h * p.lv.cap + tok) * XSV_D;
-                        }
-                    } else {
-                        const int tok = (kv - n_ct) * BN + t;
-                        if (tok < F) {
-                            kr = Kg + ((size_t)h * F + tok) * XSV_D;
-                            vr = Vg + ((size_t)h * F + tok) * XSV_D;
-                        }
+#pragma unroll
+                for (int ck = 0; ck < 8; ++ck) {
+                    uint32_t o[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int slot = 4 * ck + q;
+                        o[q] = dq_pair<UB>(rc.w[(slot / SPW) % NW], slot % SPW, a2[slot % SPW], s2, b2[slot % SPW]);
                     }
-                    row16_to_tile<T, W>(kr, sK, t);
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(BAR(B_KFULL + s));
-                    row16_to_tile<T, W>(vr, sV, t);
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(BAR(B_VFULL + s));
+                    *reinterpret_cast<uint4*>(tile + swz(row, ck)) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
             }
+            if (!rc.valid) {                       // rows past the end of the cache (last tile only) read as zero
+#pragma unroll
+                for (int ck = 0; ck < 8; ++ck) *reinterpret_cast<uint4*>(tile + swz(row, ck)) = make_uint4(0u, 0u, 0u, 0u);
+            }
+        } else {
+            // raw 16-bit rows: the fresh frame, or a cache kept unquantised (bits == 16)
+            const T* src = nullptr;
+            if (cached) {
+                const int tok = cur.kv * BN + row;
+                if (tok < T_c)
+                    src = reinterpret_cast<const T*>(sl < 4 ? lv.kcodes : lv.vcodes) + ((size_t)cur.h * lv.cap + tok) * XSV_D;
+            } else {
+                const int tok = (cur.kv - n_ct) * BN + row;
+                if (tok < F) src = (sl < 4 ? Kg : Vg) + ((size_t)cur.h * F + tok) * XSV_D;
+            }
+            row16_to_tile<T, W>(src, tile, row);
         }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR((sl < 4 ? B_KFULL : B_VFULL) + st));
+        rc = rn;
+        cur = nxt;
+        it = itn;
+        g = gn;
     }
 }
 
@@ -828,7 +881,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_cons
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 12) {
+    if (warp == 8 + NPROD) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -840,11 +893,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_cons
     const Cta cta{smem, smem_base, bar_base, tmem_base, abort_flag, b, u_first, u_last};
 
     if (warp < 8) softmax_loop<T, BITS>(p, cta);
-    else if (warp < 12) producer_loop<T, BITS>(p, cta);
+    else if (warp < 8 + NPROD) producer_loop<T, BITS>(p, cta);
     else if (lane == 0) mma_loop(p, cta);
     tc_fence_before();
     __syncthreads();
-    if (warp == 12) {
+    if (warp == 8 + NPROD) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     }
