@@ -370,11 +370,12 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
 
 // 32 logits of one row -> 32 probabilities 2^(s * sc - m) packed as fp16 pairs;
 // accumulates their sum and the running maximum of the raw logits.
+template <bool WITH_MAX>
 __device__ __forceinline__ void softmax32(const uint32_t (&v)[32], float sc, float nm, float& mx, float& ls, uint32_t (&pk)[16]) {
 #pragma unroll
     for (int i = 0; i < 32; i += 2) {
         const float s0 = __uint_as_float(v[i]), s1 = __uint_as_float(v[i + 1]);
-        mx = fmax3(mx, s0, s1);
+        if (WITH_MAX) mx = fmax3(mx, s0, s1);
         const float p0 = ex2(fmaf(s0, sc, nm)), p1 = ex2(fmaf(s1, sc, nm));
         ls += p0 + p1;
         pk[i >> 1] = pack_h2(p0, p1);
@@ -595,7 +596,8 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const T* Qg = reinterpret_cast<const T*>(p.Q);
     T* Og = reinterpret_cast<T*>(p.out);
-    const int F = p.F, nkv = p.nkv, n_ct = p.n_ct;
+    const int F = p.F, nkv = p.nkv, n_ct = p.n_ct, T_c = p.T_c;
+    int* const status = p.status;
     {
         // =============================================================== softmax + epilogue
         const int X = warp >> 2;                       // query tile of this warpgroup
@@ -624,35 +626,51 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
 
             float m_used = -INFINITY, l = 0.f;
             for (int kv = sp.kv0; kv < sp.kv1; ++kv) {
-                const int cnt = kv < n_ct ? min(BN, p.T_c - kv * BN) : min(BN, F - (kv - n_ct) * BN);
+                const int cnt = kv < n_ct ? min(BN, T_c - kv * BN) : min(BN, F - (kv - n_ct) * BN);
                 const bool tail = cnt < BN;
                 const bool first = kv == sp.kv0;
-                mbar_wait(BAR(B_SFULL + X), cX & 1u, abort_flag, p.status);
+                mbar_wait(BAR(B_SFULL + X), cX & 1u, abort_flag, status);
                 tc_fence_after();
                 float nm = -m_used, ls = 0.f, mx = -INFINITY;
+                bool s_released = false;
                 if (!tail) {
                     // ---- fast path: one pass with the row maximum in use (stale by at most the threshold).
                     //      Probabilities go to tensor memory as fp16 while this tile's true maximum is gathered;
                     //      the next 32 columns are in flight while the current ones are processed.
-                    uint32_t va[32], vb[32];
+                    uint32_t va[32], vb[32], pk[16];
                     tmem_ld32(tS, va);
                     tc_wait_ld();
-#pragma unroll 1
-                    for (int i = 0; i < 2; ++i) {
-                        uint32_t pk[16];
-                        tmem_ld32(tS + 64u * i + 32u, vb);
-                        softmax32(va, SC, nm, mx, ls, pk);
-                        if (i == 0 && !first) {
-                            // PV of the previous tile must be complete before P is overwritten (or O rescaled)
-                            mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, p.status);
-                            tc_fence_after();
-                        }
-                        tmem_st16(tP + 32u * i, pk);
-                        tc_wait_ld();
-                        if (i == 0) tmem_ld32(tS + 64u, va);
-                        softmax32(vb, SC, nm, mx, ls, pk);
-                        tmem_st16(tP + 32u * i + 16u, pk);
-                        if (i == 0) tc_wait_ld();
+                    tmem_ld32(tS + 32u, vb);
+                    softmax32<true>(va, SC, nm, mx, ls, pk);
+                    if (!first) {
+                        // PV of the previous tile must be complete before P is overwritten (or O rescaled)
+                        mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, status);
+                        tc_fence_after();
+                    }
+                    tmem_st16(tP, pk);
+                    tc_wait_ld();
+                    tmem_ld32(tS + 64u, va);
+                    softmax32<true>(vb, SC, nm, mx, ls, pk);
+                    tmem_st16(tP + 16u, pk);
+                    tc_wait_ld();
+                    tmem_ld32(tS + 96u, vb);
+                    tc_wait_ld();
+                    // All of S is in registers.  Its maximum decides now whether the stale row maximum may stay; if
+                    // so S is released here, half a tile early, so that the next QK^T overlaps the rest of this tile.
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        mx = fmax3(mx, __uint_as_float(va[i]), __uint_as_float(va[i + 1]));
+                        mx = fmax3(mx, __uint_as_float(vb[i]), __uint_as_float(vb[i + 1]));
+                    }
+                    if (!__any_sync(0xFFFFFFFFu, mx * SC > m_used + RESCALE_THRESHOLD)) {
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(BAR(B_SFREE + X));
+                        s_released = true;
+                        softmax32<false>(va, SC, nm, mx, ls, pk);
+                        tmem_st16(tP + 32u, pk);
+                        softmax32<false>(vb, SC, nm, mx, ls, pk);
+                        tmem_st16(tP + 48u, pk);
                     }
                 } else {
                     // ---- ragged tile: masked maximum first (compact loop)
@@ -666,7 +684,7 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
                             if (16 * c + i < cnt) mx = fmaxf(mx, __uint_as_float(v[i]));
                     }
                     if (!first) {
-                        mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, p.status);
+                        mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, status);
                         tc_fence_after();
                     }
                 }
@@ -711,10 +729,11 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
                         tmem_st8(tP + 8u * c, pk);
                     }
                 }
-                // S has been read for good: the next QK^T may overwrite it
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(BAR(B_SFREE + X));
+                if (!s_released) {   // S has been read for good: the next QK^T may overwrite it
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(BAR(B_SFREE + X));
+                }
                 l += ls;
                 tc_wait_st();
                 tc_fence_before();
@@ -723,7 +742,7 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
                 ++cX;
             }
             // ---- epilogue of the span
-            mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, p.status);
+            mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, status);
             tc_fence_after();
             const bool full = sp.kv0 == 0 && sp.kv1 == nkv;
             const float inv = 1.f / l;
@@ -765,86 +784,105 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
     }
 }
 
-// MMA issuer: one thread.
+// One lane of the warp, the same one every time (the lowest); lets the compiler
+// keep the operands of the instructions under it in uniform registers.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t p;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(p));
+    return p != 0;
+}
+
+// MMA issuer: one warp running converged; the tensor-core instructions and their
+// commits are issued by its elected lane (a single thread issuing from a diverged
+// warp measured about twice as slow per instruction).
 __device__ __noinline__ void mma_loop(const Params& p, const Cta c) {
     const uint32_t smem_base = c.smem_base, tmem_base = c.tmem_base;
     volatile int* const abort_flag = c.abort_flag;
     const int b = c.b, u_first = c.u_first, u_last = c.u_last;
     auto BAR = [&](int i) { return c.bar_base + 8u * (uint32_t)i; };
     const int F = p.F;
-    {
-        // =============================================================== MMA issuer (one thread)
-        // Each query tile has its own strictly ordered sequence QK(0), QK(1), PV(0), QK(2), PV(1), ... in which
-        // every operation is gated by one barrier phase; the two sequences are merged by readiness, so that a
-        // tile never waits for the other tile's softmax.
-        const uint32_t tS0 = tmem_base, tP0 = tmem_base + 256u, tO0 = tmem_base + 384u;
-        uint32_t it0 = 0, cT[2] = {0, 0}, uT[2] = {0, 0};
-        for (int u = u_first; u <= u_last; ++u) {
-            const Span sp = cta_span(p, b, u);
-            if (sp.kv0 >= sp.kv1) continue;
-            const int h = u / p.npair, mp = u - h * p.npair;
-            (void)h;
-            const int ntile = (mp * 2 * BM + BM < F) ? 2 : 1;
-            const int n = sp.kv1 - sp.kv0;
-            for (int x = 0; x < ntile; ++x) mbar_wait(BAR(B_QFULL + x), uT[x] & 1u, abort_flag, p.status);
-            tc_fence_after();
-            int qk_next[2] = {0, 0}, pv_next[2] = {0, 0};
-            if (ntile == 1) { qk_next[1] = n; pv_next[1] = n; }
-            unsigned long long t_idle = 0;
-            uint32_t idle = 0;
-            while (pv_next[0] < n || pv_next[1] < n) {
-                bool progress = false;
+    int* const status = p.status;
+    // Each query tile has its own strictly ordered sequence QK(0), QK(1), PV(0), QK(2), PV(1), ... in which
+    // every operation is gated by one barrier phase; the two sequences are merged by readiness, so that a
+    // tile never waits for the other tile's softmax.  Every lane takes the same decisions: a barrier test is
+    // broadcast from lane 0.
+    auto ready = [&](uint32_t bar, uint32_t parity) { return __shfl_sync(0xFFFFFFFFu, mbar_test(bar, parity), 0) != 0u; };
+    const uint32_t tS0 = tmem_base, tP0 = tmem_base + 256u, tO0 = tmem_base + 384u;
+    uint32_t it0 = 0, cT[2] = {0, 0}, uT[2] = {0, 0};
+    for (int u = u_first; u <= u_last; ++u) {
+        const Span sp = cta_span(p, b, u);
+        if (sp.kv0 >= sp.kv1) continue;
+        const int mp = u % p.npair;
+        const int ntile = (mp * 2 * BM + BM < F) ? 2 : 1;
+        const int n = sp.kv1 - sp.kv0;
+        for (int x = 0; x < ntile; ++x) mbar_wait(BAR(B_QFULL + x), uT[x] & 1u, abort_flag, status);
+        tc_fence_after();
+        int qk_next[2] = {0, 0}, pv_next[2] = {0, 0};
+        if (ntile == 1) { qk_next[1] = n; pv_next[1] = n; }
+        unsigned long long t_idle = 0;
+        uint32_t idle = 0;
+        while (pv_next[0] < n || pv_next[1] < n) {
+            bool progress = false;
 #pragma unroll
-                for (int x = 0; x < 2; ++x) {
-                    if (qk_next[x] < n) {
-                        const uint32_t itq = it0 + (uint32_t)qk_next[x], sq = itq % NSTAGE;
-                        const uint32_t c = cT[x] + (uint32_t)qk_next[x];     // number of this tile's S among all of the CTA's
-                        if (mbar_test(BAR(B_KFULL + sq), (itq / NSTAGE) & 1u) &&
-                            (c == 0 || mbar_test(BAR(B_SFREE + x), (c - 1u) & 1u))) {
-                            tc_fence_after();
-                            const uint64_t qd = smem_desc(smem_base + OFF_Q + x * TILE_BYTES);
-                            const uint64_t kd = smem_desc(smem_base + OFF_KV + sq * 2 * TILE_BYTES);
+            for (int x = 0; x < 2; ++x) {
+                if (qk_next[x] < n) {
+                    const uint32_t itq = it0 + (uint32_t)qk_next[x], sq = itq % NSTAGE;
+                    const uint32_t cq = cT[x] + (uint32_t)qk_next[x];   // number of this tile's S among all of the CTA's
+                    if (ready(BAR(B_KFULL + sq), (itq / NSTAGE) & 1u) && (cq == 0 || ready(BAR(B_SFREE + x), (cq - 1u) & 1u))) {
+                        tc_fence_after();
+                        const uint64_t qd = smem_desc(smem_base + OFF_Q + x * TILE_BYTES);
+                        const uint64_t kd = smem_desc(smem_base + OFF_KV + sq * 2 * TILE_BYTES);
+                        if (elect_one()) {
 #pragma unroll
                             for (int k = 0; k < 4; ++k)        // 16 channels = 32 bytes inside the swizzled row
                                 mma_ss(tS0 + (uint32_t)(x * 128), qd + 2u * k, kd + 2u * k, IDESC_QK, k > 0);
                             tc_commit(BAR(B_SFULL + x));
-                            ++qk_next[x];
-                            progress = true;
                         }
-                    }
-                    if (pv_next[x] < qk_next[x]) {
-                        const int j = pv_next[x];
-                        const uint32_t itp = it0 + (uint32_t)j, sv = itp % NSTAGE;
-                        if (mbar_test(BAR(B_VFULL + sv), (itp / NSTAGE) & 1u) &&
-                            mbar_test(BAR(B_PREADY + x), (cT[x] + (uint32_t)j) & 1u)) {
-                            tc_fence_after();
-                            const uint64_t vd = smem_desc(smem_base + OFF_KV + sv * 2 * TILE_BYTES + TILE_BYTES);
-#pragma unroll
-                            for (int k = 0; k < 8; ++k)        // 16 tokens: 8 columns of P, 2048 bytes of V
-                                mma_ts(tO0 + (uint32_t)(x * 64), tP0 + (uint32_t)(x * 64) + 8u * k, vd + 128u * k, IDESC_PV,
-                                       (j > 0 || k > 0) ? 1u : 0u);
-                            tc_commit(BAR(B_PVDONE + x));
-                            ++pv_next[x];
-                            if (pv_next[x ^ 1] > j) tc_commit(BAR(B_EMPTY + sv));   // both tiles are through with this stage
-                            progress = true;
-                        }
+                        __syncwarp();
+                        ++qk_next[x];
+                        progress = true;
                     }
                 }
-                if (progress) {
-                    idle = 0;
-                } else {
-                    if (*abort_flag) break;
-                    if (++idle == 64u) t_idle = globaltimer();
-                    if (idle > 64u && (idle & 255u) == 0u && globaltimer() - t_idle > WAIT_LIMIT_NS) {
-                        *abort_flag = 1;
-                        atomicOr(p.status, XSV_DEV_TIMEOUT);
-                        break;
+                if (pv_next[x] < qk_next[x]) {
+                    const int j = pv_next[x];
+                    const uint32_t itp = it0 + (uint32_t)j, sv = itp % NSTAGE;
+                    if (ready(BAR(B_VFULL + sv), (itp / NSTAGE) & 1u) && ready(BAR(B_PREADY + x), (cT[x] + (uint32_t)j) & 1u)) {
+                        tc_fence_after();
+                        const uint64_t vd = smem_desc(smem_base + OFF_KV + sv * 2 * TILE_BYTES + TILE_BYTES);
+                        const bool release = pv_next[x ^ 1] > j;   // both tiles are through with this stage
+                        if (elect_one()) {
+                            if (j > 0) {
+#pragma unroll
+                                for (int k = 0; k < 8; ++k)    // 16 tokens: 8 columns of P, 2048 bytes of V
+                                    mma_ts(tO0 + (uint32_t)(x * 64), tP0 + (uint32_t)(x * 64) + 8u * k, vd + 128u * k, IDESC_PV, 1u);
+                            } else {
+#pragma unroll
+                                for (int k = 0; k < 8; ++k)
+                                    mma_ts(tO0 + (uint32_t)(x * 64), tP0 + (uint32_t)(x * 64) + 8u * k, vd + 128u * k, IDESC_PV, k > 0);
+                            }
+                            tc_commit(BAR(B_PVDONE + x));
+                            if (release) tc_commit(BAR(B_EMPTY + sv));
+                        }
+                        __syncwarp();
+                        ++pv_next[x];
+                        progress = true;
                     }
                 }
             }
-            it0 += (uint32_t)n;
-            for (int x = 0; x < ntile; ++x) { cT[x] += (uint32_t)n; ++uT[x]; }
+            if (progress) {
+                idle = 0;
+            } else {
+                if (*abort_flag) break;
+                if (++idle == 64u) t_idle = globaltimer();
+                if (idle > 64u && (idle & 255u) == 0u && globaltimer() - t_idle > WAIT_LIMIT_NS) {
+                    *abort_flag = 1;
+                    atomicOr(status, XSV_DEV_TIMEOUT);
+                    break;
+                }
+            }
         }
+        it0 += (uint32_t)n;
+        for (int x = 0; x < ntile; ++x) { cT[x] += (uint32_t)n; ++uT[x]; }
     }
 }
 
@@ -894,7 +932,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_cons
 
     if (warp < 8) softmax_loop<T, BITS>(p, cta);
     else if (warp < 8 + NPROD) producer_loop<T, BITS>(p, cta);
-    else if (lane == 0) mma_loop(p, cta);
+    else mma_loop(p, cta);
     tc_fence_before();
     __syncthreads();
     if (warp == 8 + NPROD) {
