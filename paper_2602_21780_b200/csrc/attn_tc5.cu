@@ -33,7 +33,7 @@ namespace {
 
 constexpr int BM = 128;            // query rows per tile
 constexpr int BN = 128;            // keys per kv tile
-constexpr int NSTAGE = 3;          // kv stages in shared memory
+constexpr int NSTAGE = 5;          // kv stages in shared memory
 constexpr int NPROD = 7;              // producer warps
 constexpr int NTHREADS = (8 + NPROD + 1) * 32;   // 8 softmax warps, the producers, the MMA issuer
 constexpr uint32_t TILE_BYTES = 128u * 128u;   // 128 rows x 64 fp16
@@ -632,31 +632,25 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
                 mbar_wait(BAR(B_SFULL + X), cX & 1u, abort_flag, status);
                 tc_fence_after();
                 float nm = -m_used, ls = 0.f, mx = -INFINITY;
-                bool s_released = false;
+                bool done = false;
                 if (!tail) {
-                    // ---- fast path: one pass with the row maximum in use (stale by at most the threshold).
-                    //      Probabilities go to tensor memory as fp16 while this tile's true maximum is gathered;
-                    //      the next 32 columns are in flight while the current ones are processed.
-                    uint32_t va[32], vb[32], pk[16];
+                    // ---- whole tile, one pass with the row maximum in use (stale by at most the threshold).  The
+                    //      first two 32-column chunks are turned into probabilities (kept in registers) while the
+                    //      other two are fetched; then all of S has been read, its maximum is known, and if the
+                    //      maximum in use may stay, S is released: the next QK^T and its hand-over latency
+                    //      overlap the second half of the tile.  The wait for the previous PV (P is single-buffered)
+                    //      comes only then, half a tile after that PV was triggered.
+                    uint32_t va[32], vb[32], pa[16], pb[16];
                     tmem_ld32(tS, va);
                     tc_wait_ld();
                     tmem_ld32(tS + 32u, vb);
-                    softmax32<true>(va, SC, nm, mx, ls, pk);
-                    if (!first) {
-                        // PV of the previous tile must be complete before P is overwritten (or O rescaled)
-                        mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, status);
-                        tc_fence_after();
-                    }
-                    tmem_st16(tP, pk);
+                    softmax32<true>(va, SC, nm, mx, ls, pa);
                     tc_wait_ld();
                     tmem_ld32(tS + 64u, va);
-                    softmax32<true>(vb, SC, nm, mx, ls, pk);
-                    tmem_st16(tP + 16u, pk);
+                    softmax32<true>(vb, SC, nm, mx, ls, pb);
                     tc_wait_ld();
                     tmem_ld32(tS + 96u, vb);
                     tc_wait_ld();
-                    // All of S is in registers.  Its maximum decides now whether the stale row maximum may stay; if
-                    // so S is released here, half a tile early, so that the next QK^T overlaps the rest of this tile.
 #pragma unroll
                     for (int i = 0; i < 32; i += 2) {
                         mx = fmax3(mx, __uint_as_float(va[i]), __uint_as_float(va[i + 1]));
@@ -666,14 +660,18 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
                         tc_fence_before();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(BAR(B_SFREE + X));
-                        s_released = true;
-                        softmax32<false>(va, SC, nm, mx, ls, pk);
-                        tmem_st16(tP + 32u, pk);
-                        softmax32<false>(vb, SC, nm, mx, ls, pk);
-                        tmem_st16(tP + 48u, pk);
+                        mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, status);
+                        tc_fence_after();
+                        tmem_st16(tP, pa);
+                        tmem_st16(tP + 16u, pb);
+                        softmax32<false>(va, SC, nm, mx, ls, pa);
+                        tmem_st16(tP + 32u, pa);
+                        softmax32<false>(vb, SC, nm, mx, ls, pb);
+                        tmem_st16(tP + 48u, pb);
+                        done = true;
                     }
                 } else {
-                    // ---- ragged tile: masked maximum first (compact loop)
+                    // ---- ragged tile: masked maximum (compact loop)
 #pragma unroll 1
                     for (int c = 0; c < 8; ++c) {
                         uint32_t v[16];
@@ -683,33 +681,33 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
                         for (int i = 0; i < 16; ++i)
                             if (16 * c + i < cnt) mx = fmaxf(mx, __uint_as_float(v[i]));
                     }
-                    if (!first) {
+                }
+                if (!done) {
+                    // ---- rare (always on the span's first tile): the maximum moved by more than the threshold, or
+                    //      the tile is ragged
+                    if (!first) {   // PV of the previous tile must be complete before P is overwritten or O rescaled
                         mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, status);
                         tc_fence_after();
                     }
-                }
-                const float m_new = mx * SC;
-                const bool need = m_new > m_used + RESCALE_THRESHOLD;   // always on the span's first tile
-                const bool any_need = __any_sync(0xFFFFFFFFu, need);
-                if (any_need) {
-                    // ---- rare: the maximum moved by more than the threshold; rescale the accumulator and the row sum
-                    const float alpha = need ? ex2(m_used - m_new) : 1.f;
-                    if (need) m_used = m_new;
-                    l *= alpha;
-                    if (!first) {
+                    const float m_new = mx * SC;
+                    const bool need = m_new > m_used + RESCALE_THRESHOLD;
+                    if (__any_sync(0xFFFFFFFFu, need)) {   // rescale the accumulator and the row sum
+                        const float alpha = need ? ex2(m_used - m_new) : 1.f;
+                        if (need) m_used = m_new;
+                        l *= alpha;
+                        if (!first) {
 #pragma unroll 1
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t o[16];
-                            tmem_ld16(tO + 16u * c, o);
-                            tc_wait_ld();
+                            for (int c = 0; c < 4; ++c) {
+                                uint32_t o[16];
+                                tmem_ld16(tO + 16u * c, o);
+                                tc_wait_ld();
 #pragma unroll
-                            for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                            tmem_st16(tO + 16u * c, o);
+                                for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                                tmem_st16(tO + 16u * c, o);
+                            }
                         }
                     }
-                }
-                if (any_need || tail) {
-                    // ---- (re)compute this tile's probabilities with the maximum now in use, masking a ragged tail
+                    // this tile's probabilities with the maximum now in use, masking a ragged tail
                     nm = -m_used;
                     ls = 0.f;
 #pragma unroll 1
@@ -728,8 +726,7 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
                         }
                         tmem_st8(tP + 8u * c, pk);
                     }
-                }
-                if (!s_released) {   // S has been read for good: the next QK^T may overwrite it
+                    // S has been read for good: the next QK^T may overwrite it
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(BAR(B_SFREE + X));
@@ -806,7 +803,6 @@ __device__ __noinline__ void mma_loop(const Params& p, const Cta c) {
     // every operation is gated by one barrier phase; the two sequences are merged by readiness, so that a
     // tile never waits for the other tile's softmax.  Every lane takes the same decisions: a barrier test is
     // broadcast from lane 0.
-    auto ready = [&](uint32_t bar, uint32_t parity) { return __shfl_sync(0xFFFFFFFFu, mbar_test(bar, parity), 0) != 0u; };
     const uint32_t tS0 = tmem_base, tP0 = tmem_base + 256u, tO0 = tmem_base + 384u;
     uint32_t it0 = 0, cT[2] = {0, 0}, uT[2] = {0, 0};
     for (int u = u_first; u <= u_last; ++u) {
@@ -823,50 +819,56 @@ __device__ __noinline__ void mma_loop(const Params& p, const Cta c) {
         uint32_t idle = 0;
         while (pv_next[0] < n || pv_next[1] < n) {
             bool progress = false;
+            // Test the gates of the next QK and the next PV of both tiles at once: the eight barrier reads are
+            // independent, so their latencies overlap (one after the other they cost far more than the issue).
+            uint32_t itq[2], sq[2], cq[2], itp[2], sv[2], bits = 0;
 #pragma unroll
             for (int x = 0; x < 2; ++x) {
-                if (qk_next[x] < n) {
-                    const uint32_t itq = it0 + (uint32_t)qk_next[x], sq = itq % NSTAGE;
-                    const uint32_t cq = cT[x] + (uint32_t)qk_next[x];   // number of this tile's S among all of the CTA's
-                    if (ready(BAR(B_KFULL + sq), (itq / NSTAGE) & 1u) && (cq == 0 || ready(BAR(B_SFREE + x), (cq - 1u) & 1u))) {
-                        tc_fence_after();
-                        const uint64_t qd = smem_desc(smem_base + OFF_Q + x * TILE_BYTES);
-                        const uint64_t kd = smem_desc(smem_base + OFF_KV + sq * 2 * TILE_BYTES);
-                        if (elect_one()) {
+                const uint32_t jq = (uint32_t)min(qk_next[x], n - 1), jp = (uint32_t)min(pv_next[x], n - 1);
+                itq[x] = it0 + jq; sq[x] = itq[x] % NSTAGE; cq[x] = cT[x] + jq;   // cq: number of this tile's S among all of the CTA's
+                itp[x] = it0 + jp; sv[x] = itp[x] % NSTAGE;
+                bits |= mbar_test(BAR(B_KFULL + sq[x]), (itq[x] / NSTAGE) & 1u) << (4 * x);
+                bits |= (cq[x] == 0 ? 1u : mbar_test(BAR(B_SFREE + x), (cq[x] - 1u) & 1u)) << (4 * x + 1);
+                bits |= mbar_test(BAR(B_VFULL + sv[x]), (itp[x] / NSTAGE) & 1u) << (4 * x + 2);
+                bits |= mbar_test(BAR(B_PREADY + x), (cT[x] + jp) & 1u) << (4 * x + 3);
+            }
+            bits = __shfl_sync(0xFFFFFFFFu, bits, 0);      // every lane takes lane 0's view
 #pragma unroll
-                            for (int k = 0; k < 4; ++k)        // 16 channels = 32 bytes inside the swizzled row
-                                mma_ss(tS0 + (uint32_t)(x * 128), qd + 2u * k, kd + 2u * k, IDESC_QK, k > 0);
-                            tc_commit(BAR(B_SFULL + x));
-                        }
-                        __syncwarp();
-                        ++qk_next[x];
-                        progress = true;
+            for (int x = 0; x < 2; ++x) {
+                if (qk_next[x] < n && ((bits >> (4 * x)) & 3u) == 3u) {
+                    tc_fence_after();
+                    const uint64_t qd = smem_desc(smem_base + OFF_Q + x * TILE_BYTES);
+                    const uint64_t kd = smem_desc(smem_base + OFF_KV + sq[x] * 2 * TILE_BYTES);
+                    if (elect_one()) {
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)        // 16 channels = 32 bytes inside the swizzled row
+                            mma_ss(tS0 + (uint32_t)(x * 128), qd + 2u * k, kd + 2u * k, IDESC_QK, k > 0);
+                        tc_commit(BAR(B_SFULL + x));
                     }
-                }
-                if (pv_next[x] < qk_next[x]) {
+                    __syncwarp();
+                    ++qk_next[x];
+                    progress = true;
+                } else if (pv_next[x] < n && pv_next[x] < qk_next[x] && ((bits >> (4 * x + 2)) & 3u) == 3u) {
                     const int j = pv_next[x];
-                    const uint32_t itp = it0 + (uint32_t)j, sv = itp % NSTAGE;
-                    if (ready(BAR(B_VFULL + sv), (itp / NSTAGE) & 1u) && ready(BAR(B_PREADY + x), (cT[x] + (uint32_t)j) & 1u)) {
-                        tc_fence_after();
-                        const uint64_t vd = smem_desc(smem_base + OFF_KV + sv * 2 * TILE_BYTES + TILE_BYTES);
-                        const bool release = pv_next[x ^ 1] > j;   // both tiles are through with this stage
-                        if (elect_one()) {
-                            if (j > 0) {
+                    tc_fence_after();
+                    const uint64_t vd = smem_desc(smem_base + OFF_KV + sv[x] * 2 * TILE_BYTES + TILE_BYTES);
+                    const bool release = pv_next[x ^ 1] > j;   // both tiles are through with this stage
+                    if (elect_one()) {
+                        if (j > 0) {
 #pragma unroll
-                                for (int k = 0; k < 8; ++k)    // 16 tokens: 8 columns of P, 2048 bytes of V
-                                    mma_ts(tO0 + (uint32_t)(x * 64), tP0 + (uint32_t)(x * 64) + 8u * k, vd + 128u * k, IDESC_PV, 1u);
-                            } else {
+                            for (int k = 0; k < 8; ++k)    // 16 tokens: 8 columns of P, 2048 bytes of V
+                                mma_ts(tO0 + (uint32_t)(x * 64), tP0 + (uint32_t)(x * 64) + 8u * k, vd + 128u * k, IDESC_PV, 1u);
+                        } else {
 #pragma unroll
-                                for (int k = 0; k < 8; ++k)
-                                    mma_ts(tO0 + (uint32_t)(x * 64), tP0 + (uint32_t)(x * 64) + 8u * k, vd + 128u * k, IDESC_PV, k > 0);
-                            }
-                            tc_commit(BAR(B_PVDONE + x));
-                            if (release) tc_commit(BAR(B_EMPTY + sv));
+                            for (int k = 0; k < 8; ++k)
+                                mma_ts(tO0 + (uint32_t)(x * 64), tP0 + (uint32_t)(x * 64) + 8u * k, vd + 128u * k, IDESC_PV, k > 0);
                         }
-                        __syncwarp();
-                        ++pv_next[x];
-                        progress = true;
+                        tc_commit(BAR(B_PVDONE + x));
+                        if (release) tc_commit(BAR(B_EMPTY + sv[x]));
                     }
+                    __syncwarp();
+                    ++pv_next[x];
+                    progress = true;
                 }
             }
             if (progress) {
