@@ -944,51 +944,54 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_cons
 }
 
 // Merge the parts of the units that were shared by several CTAs, in CTA order.
+// Grid: (16, units); block: 256 threads = 16 rows x 16 groups of 4 channels, so
+// that a row's 256 bytes are read by 16 consecutive threads.
+constexpr int MAX_PARTS = 256;         // a unit can be shared by as many CTAs as there are; the launcher keeps G <= MAX_PARTS
 template <typename T>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const Params p) {
-    const int u = blockIdx.x, row = threadIdx.x;
-    long long base;
-    int cost;
-    unit_base_cost(p, u, base, cost);
-    // CTAs that may hold steps of this unit
-    int b0 = (int)(base * p.G / p.total), b1 = (int)((base + (long long)cost * (p.nkv - 1)) * p.G / p.total);
-    b0 = max(0, b0 - 1);
-    b1 = min(p.G - 1, b1 + 1);
-    const int h = u / p.npair, mp = u - h * p.npair;
-    const int grow = mp * 2 * BM + row;
-    float M = -INFINITY;
-    int nparts = 0;
-    for (int b = b0; b <= b1; ++b) {
-        const Span sp = cta_span(p, b, u);
-        if (sp.kv0 >= sp.kv1) continue;
-        if (sp.kv0 == 0 && sp.kv1 == p.nkv) return;   // whole unit in one CTA: already written
-        ++nparts;
-        const float* part = p.part + ((size_t)b * 2 + (sp.kv0 > 0 ? 0 : 1)) * PART_STRIDE;
-        M = fmaxf(M, reinterpret_cast<const float2*>(part + 256 * 64)[row].x);
+    __shared__ int s_slot[MAX_PARTS];
+    __shared__ int s_n;
+    const int u = blockIdx.y;
+    if (threadIdx.x == 0) {
+        long long base;
+        int cost;
+        unit_base_cost(p, u, base, cost);
+        // CTAs that may hold steps of this unit
+        int b0 = (int)(base * p.G / p.total), b1 = (int)((base + (long long)cost * (p.nkv - 1)) * p.G / p.total);
+        b0 = max(0, b0 - 1);
+        b1 = min(p.G - 1, b1 + 1);
+        int n = 0;
+        for (int b = b0; b <= b1; ++b) {
+            const Span sp = cta_span(p, b, u);
+            if (sp.kv0 >= sp.kv1) continue;
+            if (sp.kv0 == 0 && sp.kv1 == p.nkv) { n = 0; break; }   // whole unit in one CTA: already written
+            if (n < MAX_PARTS) s_slot[n++] = b * 2 + (sp.kv0 > 0 ? 0 : 1);
+        }
+        s_n = n;
     }
-    if (nparts == 0 || grow >= p.F) return;
-    float acc[64];
-#pragma unroll
-    for (int i = 0; i < 64; ++i) acc[i] = 0.f;
+    __syncthreads();
+    const int n = s_n;
+    if (n == 0) return;
+    const int h = u / p.npair, mp = u - h * p.npair;
+    const int row = blockIdx.x * 16 + (threadIdx.x >> 4), c4 = threadIdx.x & 15;
+    const int grow = mp * 2 * BM + row;
+    if (grow >= p.F) return;
+    float M = -INFINITY;
+    for (int i = 0; i < n; ++i)
+        M = fmaxf(M, reinterpret_cast<const float2*>(p.part + (size_t)s_slot[i] * PART_STRIDE + 256 * 64)[row].x);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float L = 0.f;
-    for (int b = b0; b <= b1; ++b) {
-        const Span sp = cta_span(p, b, u);
-        if (sp.kv0 >= sp.kv1) continue;
-        const float* part = p.part + ((size_t)b * 2 + (sp.kv0 > 0 ? 0 : 1)) * PART_STRIDE;
+    for (int i = 0; i < n; ++i) {
+        const float* part = p.part + (size_t)s_slot[i] * PART_STRIDE;
         const float2 ml = reinterpret_cast<const float2*>(part + 256 * 64)[row];
         const float w = exp2f(ml.x - M);
         L += ml.y * w;
-        const float4* src = reinterpret_cast<const float4*>(part + (size_t)row * 64);
-#pragma unroll
-        for (int q = 0; q < 16; ++q) {
-            const float4 v = src[q];
-            acc[4 * q] += v.x * w; acc[4 * q + 1] += v.y * w; acc[4 * q + 2] += v.z * w; acc[4 * q + 3] += v.w * w;
-        }
+        const float4 v = reinterpret_cast<const float4*>(part + (size_t)row * 64)[c4];
+        acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
     }
     const float inv = 1.f / L;
-    uint32_t* dst = reinterpret_cast<uint32_t*>(reinterpret_cast<T*>(p.out) + ((size_t)h * p.F + grow) * XSV_D);
-#pragma unroll
-    for (int q = 0; q < 32; ++q) dst[q] = xsv_pack2<T>(acc[2 * q] * inv, acc[2 * q + 1] * inv);
+    uint2* dst = reinterpret_cast<uint2*>(reinterpret_cast<T*>(p.out) + ((size_t)h * p.F + grow) * XSV_D) + c4;
+    *dst = make_uint2(xsv_pack2<T>(acc.x * inv, acc.y * inv), xsv_pack2<T>(acc.z * inv, acc.w * inv));
 }
 
 int sm_count() {
@@ -1010,7 +1013,7 @@ cudaError_t launch(const Params& p, cudaStream_t st) {
         attr_set = true;
     }
     attn_tc5_kernel<T, BITS><<<p.G, NTHREADS, SMEM_BYTES, st>>>(p);
-    attn_combine_kernel<T><<<p.H * p.npair, 256, 0, st>>>(p);
+    attn_combine_kernel<T><<<dim3(16, p.H * p.npair), 256, 0, st>>>(p);
     xsv_count_launch(2);
     return cudaGetLastError();
 }
@@ -1033,6 +1036,7 @@ cudaError_t xsv_launch_attn_tc5(const LayerView& lv, int T_c, const void* Q, con
     p.total = p.ticks_head * H;
     const long long steps = (long long)H * p.npair * p.nkv;
     p.G = (int)(steps < sm_count() ? steps : sm_count());
+    if (p.G > MAX_PARTS) p.G = MAX_PARTS;
 #define XSV_TC5(TT, B) return launch<TT, B>(p, st)
     if (dtype == 0) {
         switch (lv.bits) {
