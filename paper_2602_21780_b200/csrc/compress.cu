@@ -17,28 +17,34 @@ __global__ void __launch_bounds__(256) qtilde_partial_kernel(const T* __restrict
     const int h = blockIdx.y, chunk = blockIdx.x;
     const int per = (F + XSV_QCHUNKS - 1) / XSV_QCHUNKS;
     const int i0 = chunk * per, i1 = min(F, i0 + per);
-    const int c2 = threadIdx.x & 31, r = threadIdx.x >> 5;
+    const int c4 = threadIdx.x & 15, r = threadIdx.x >> 4;     // 4 channels (one 8-byte load), 16 rows in flight
     const int n_patch = F - n_special;
-    float a0 = 0.f, a1 = 0.f;
-    for (int i = i0 + r; i < i1; i += 8) {
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 4
+    for (int i = i0 + r; i < i1; i += 16) {
         float w = 1.f;
         if (i >= n_special) {
-            int gi = (i - n_special) / g;
-            int sz = min(g, n_patch - gi * g);
-            w = 1.f / (float)sz;
+            const int gi = (i - n_special) / g;
+            w = 1.f / (float)min(g, n_patch - gi * g);
         }
-        const T* row = Q + ((size_t)h * F + i) * XSV_D + 2 * c2;
-        a0 = fmaf(w, xsv_to_float<T>(row[0]), a0);
-        a1 = fmaf(w, xsv_to_float<T>(row[1]), a1);
+        const uint2 v = *reinterpret_cast<const uint2*>(Q + ((size_t)h * F + i) * XSV_D + 4 * c4);
+        T e[4];
+        *reinterpret_cast<uint2*>(e) = v;
+        a0 = fmaf(w, xsv_to_float<T>(e[0]), a0);
+        a1 = fmaf(w, xsv_to_float<T>(e[1]), a1);
+        a2 = fmaf(w, xsv_to_float<T>(e[2]), a2);
+        a3 = fmaf(w, xsv_to_float<T>(e[3]), a3);
     }
-    __shared__ float red[8][64];
-    red[r][2 * c2] = a0;
-    red[r][2 * c2 + 1] = a1;
+    __shared__ float red[16][64];
+    red[r][4 * c4] = a0;
+    red[r][4 * c4 + 1] = a1;
+    red[r][4 * c4 + 2] = a2;
+    red[r][4 * c4 + 3] = a3;
     __syncthreads();
     if (threadIdx.x < 64) {
         float s = 0.f;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) s += red[k][threadIdx.x];
+        for (int k = 0; k < 16; ++k) s += red[k][threadIdx.x];
         qpart[((size_t)h * XSV_QCHUNKS + chunk) * 64 + threadIdx.x] = s;
     }
 }
@@ -48,9 +54,20 @@ __global__ void __launch_bounds__(256) qtilde_partial_kernel(const T* __restrict
 // One thread per token; the (scale, zero-point) rows of the key groups a block
 // touches are staged in shared memory.
 // ---------------------------------------------------------------------------
-constexpr int SCORE_TPB = 256;
-constexpr int SCORE_MAXG = SCORE_TPB / XSV_G + 1;   // groups a block can span
+constexpr int SCORE_TPB = 256;             // 64 tokens x 4 slices of the heads
+constexpr int SCORE_TOK = 64;              // tokens per block
+constexpr int SCORE_MAXG = 2;              // key groups a block's 64 tokens can span
 
+// Sum of the fixed-order partial sums of the pooled queries, scaled: q~[c].
+__device__ __forceinline__ float qtilde_channel(const float* __restrict__ qpart, int n_part, int c, float qnorm) {
+    float s = 0.f;
+#pragma unroll 8
+    for (int k = 0; k < n_part; ++k) s += qpart[(size_t)k * 64 + c];
+    return s * qnorm;
+}
+
+// By linearity q~ . K~[h,j,:] = sum_c (q~_c s_c) code_c - sum_c q~_c s_c z_c: the weights q~_c s_c and the
+// bias are prepared once per (head, key group) of the block; a token then costs one multiply-add per code.
 template <int BITS>
 __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, int T_first, int T_c,
                                                           const float* __restrict__ qpart, float qnorm,
@@ -60,53 +77,72 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
     constexpr int CPW = 32 / BITS;             // codes per 32-bit word
     extern __shared__ float sm[];
     float* qt = sm;                             // [64]
-    float* sS = qt + 64;                        // [H][SCORE_MAXG][64]
-    float* sZ = sS + (size_t)H * SCORE_MAXG * 64;
+    float* sW = qt + 64;                        // [H][SCORE_MAXG][64] weights q~_c * s_c
+    float* sB = sW + (size_t)H * SCORE_MAXG * 64;   // [H][SCORE_MAXG] bias sum_c q~_c s_c z_c
 
-    const int j0 = blockIdx.x * SCORE_TPB;
+    const int j0 = blockIdx.x * SCORE_TOK;
     const int p0 = T_first + j0;
     const int g_lo = p0 >> 6;
-    const int p_last = min(T_c - 1, p0 + SCORE_TPB - 1);
+    const int p_last = min(T_c - 1, p0 + SCORE_TOK - 1);
     const int ng = (p_last >> 6) - g_lo + 1;
 
-    if (threadIdx.x < 64) {
-        float s = 0.f;
-        for (int k = 0; k < H * XSV_QCHUNKS; ++k) s += qpart[(size_t)k * 64 + threadIdx.x];
-        qt[threadIdx.x] = s * qnorm;
+    {   // q~: four threads per channel sum a quarter of the partial sums each, then a fixed-order sum of the four
+        const int c = threadIdx.x & 63, part = threadIdx.x >> 6, np = H * XSV_QCHUNKS, per = (np + 3) / 4;
+        float s4 = 0.f;
+        const int k1 = min(np, (part + 1) * per);
+#pragma unroll 8
+        for (int k = part * per; k < k1; ++k) s4 += qpart[(size_t)k * 64 + c];
+        sW[part * 64 + c] = s4;            // sW is free until the weights are staged
+        __syncthreads();
+        if (threadIdx.x < 64) qt[c] = (((sW[c] + sW[64 + c]) + sW[128 + c]) + sW[192 + c]) * qnorm;
     }
+    __syncthreads();
     for (int i = threadIdx.x; i < H * ng * 64; i += SCORE_TPB) {
-        int c = i & 63, gg = (i >> 6) % ng, h = (i >> 6) / ng;
-        size_t m = ((size_t)h * lv.capg + g_lo + gg) * 64 + c;
-        sS[(h * SCORE_MAXG + gg) * 64 + c] = lv.kscale[m];
-        sZ[(h * SCORE_MAXG + gg) * 64 + c] = (float)lv.kzero[m];
+        const int c = i & 63, gg = (i >> 6) % ng, h = (i >> 6) / ng;
+        const size_t m = ((size_t)h * lv.capg + g_lo + gg) * 64 + c;
+        sW[(h * SCORE_MAXG + gg) * 64 + c] = qt[c] * lv.kscale[m];
+    }
+    __syncthreads();
+    for (int i = threadIdx.x >> 5; i < H * ng; i += SCORE_TPB / 32) {   // one warp per (head, group): the bias
+        const int gg = i % ng, h = i / ng, lane = threadIdx.x & 31;
+        const size_t m = ((size_t)h * lv.capg + g_lo + gg) * 64;
+        float b = sW[(h * SCORE_MAXG + gg) * 64 + lane] * (float)lv.kzero[m + lane] +
+                  sW[(h * SCORE_MAXG + gg) * 64 + lane + 32] * (float)lv.kzero[m + lane + 32];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) b += __shfl_xor_sync(0xFFFFFFFFu, b, o);
+        if (lane == 0) sB[h * SCORE_MAXG + gg] = b;
     }
     __syncthreads();
 
-    const int p = p0 + threadIdx.x;
-    if (p >= T_c) return;
-    const int gg = (p >> 6) - g_lo;
+    const int tok = threadIdx.x >> 2, slice = threadIdx.x & 3;
+    const int p = p0 + tok;
     float acc = 0.f;
-    for (int h = 0; h < H; ++h) {
-        const uint4* row = reinterpret_cast<const uint4*>(lv.kcodes + ((size_t)h * lv.cap + p) * ROWB);
-        const float* s = sS + (h * SCORE_MAXG + gg) * 64;
-        const float* z = sZ + (h * SCORE_MAXG + gg) * 64;
+    if (p < T_c) {
+        const int gg = (p >> 6) - g_lo;
+        for (int h = slice; h < H; h += 4) {
+            const uint4* row = reinterpret_cast<const uint4*>(lv.kcodes + ((size_t)h * lv.cap + p) * ROWB);
+            const float* w = sW + (h * SCORE_MAXG + gg) * 64;
+            float a = 0.f;
 #pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            uint4 q = row[v];
-            uint32_t w[4] = {q.x, q.y, q.z, q.w};
+            for (int v = 0; v < NV; ++v) {
+                const uint4 q = row[v];
+                const uint32_t ww[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
+                for (int k = 0; k < 4; ++k) {
 #pragma unroll
-                for (int e = 0; e < CPW; ++e) {
-                    int c = (v * 4 + k) * CPW + e;
-                    float code = (float)((w[k] >> (e * BITS)) & ((1u << BITS) - 1u));
-                    float kt = __fmul_rn(__fsub_rn(code, z[c]), s[c]);
-                    acc = fmaf(qt[c], kt, acc);
+                    for (int e = 0; e < CPW; ++e) {
+                        const int c = (v * 4 + k) * CPW + e;
+                        a = fmaf(w[c], (float)((ww[k] >> (e * BITS)) & ((1u << BITS) - 1u)), a);
+                    }
                 }
             }
+            acc += a - sB[h * SCORE_MAXG + gg];
         }
     }
-    scores[j0 + threadIdx.x] = acc / (float)H;
+    // the four slices of a token sit in adjacent lanes: fixed-order sum
+    acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 1);
+    acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 2);
+    if (slice == 0 && p < T_c) scores[j0 + tok] = acc / (float)H;
 }
 
 // bits == 16: keys are raw 16-bit values.
@@ -115,11 +151,7 @@ __global__ void __launch_bounds__(SCORE_TPB) score_raw_kernel(LayerView lv, int 
                                                               const float* __restrict__ qpart, float qnorm,
                                                               float* __restrict__ scores) {
     __shared__ float qt[64];
-    if (threadIdx.x < 64) {
-        float s = 0.f;
-        for (int k = 0; k < H * XSV_QCHUNKS; ++k) s += qpart[(size_t)k * 64 + threadIdx.x];
-        qt[threadIdx.x] = s * qnorm;
-    }
+    if (threadIdx.x < 64) qt[threadIdx.x] = qtilde_channel(qpart, H * XSV_QCHUNKS, threadIdx.x, qnorm);
     __syncthreads();
     const int j = blockIdx.x * SCORE_TPB + threadIdx.x;
     const int p = T_first + j;
@@ -234,10 +266,132 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
 }
 
 // ---------------------------------------------------------------------------
-// Eq. 9-11 for keys.  One block per (new 64-token group, head): gather the
-// group's members as float32 (Eq. 12 for cached tokens, widening for fresh
-// ones), per-channel min/max over the tokens, parameters, codes, pack.
+// Eq. 8 again, for n <= 1024 * KPT: every thread keeps KPT consecutive keys in
+// registers, so the scores are read from memory once.  The four digit
+// histograms are built with warp-aggregated shared-memory atomics (scores
+// share their leading digits, which would otherwise serialise), the bins are
+// scanned by one warp, and the ordered compaction is a block-wide prefix sum
+// over per-thread counts.  Same total order as select_kernel.
 // ---------------------------------------------------------------------------
+__device__ __forceinline__ int block_exclusive_scan_1024(int v, int* warp_sums, int& total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t; }
+    __syncthreads();                       // warp_sums may still be read from a previous scan
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    int ws = warp_sums[lane], wincl = ws;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, wincl, o); if (lane >= o) wincl += t; }
+    total = __shfl_sync(0xFFFFFFFFu, wincl, 31);
+    const int wbase = __shfl_sync(0xFFFFFFFFu, wincl - ws, warp);
+    return wbase + incl - v;
+}
+
+template <int KPT>
+__global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restrict__ scores, int n, int k, int T_first,
+                                                          int T_c, int* __restrict__ srcmap, int* __restrict__ dscal) {
+    __shared__ int hist[256];
+    __shared__ int warp_sums[32];
+    __shared__ uint32_t s_prefix;
+    __shared__ int s_remaining;
+    __shared__ int s_first_evicted;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int j0 = tid * KPT;
+    uint32_t key[KPT];
+#pragma unroll
+    for (int i = 0; i < KPT; ++i) key[i] = (j0 + i < n) ? score_key(scores[j0 + i]) : 0u;
+
+    uint32_t thr = 0xFFFFFFFFu;
+    int need_eq = 0;
+    if (k > 0) {
+        uint32_t prefix = 0, mask = 0;
+        int remaining = k;
+        for (int pass = 3; pass >= 0; --pass) {
+            const int shift = pass * 8;
+            if (tid < 256) hist[tid] = 0;
+            __syncthreads();
+#pragma unroll
+            for (int i = 0; i < KPT; ++i) {
+                const bool act = (j0 + i < n) && (key[i] & mask) == prefix;
+                const uint32_t digit = act ? ((key[i] >> shift) & 255u) : 256u;
+                const uint32_t peers = __match_any_sync(0xFFFFFFFFu, digit);
+                if (act && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+            }
+            __syncthreads();
+            if (tid < 32) {
+                // bins from the top: find the digit at which the cumulated count reaches `remaining`
+                int c[8], sum = 0;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) { c[q] = hist[255 - (tid * 8 + q)]; sum += c[q]; }
+                int incl = sum;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t; }
+                int cum = incl - sum;          // count in the bins above this lane's
+                const bool here = cum < remaining && incl >= remaining;
+                if (here) {
+                    int digit = 0;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        if (cum + c[q] >= remaining) { digit = 255 - (tid * 8 + q); break; }
+                        cum += c[q];
+                    }
+                    s_remaining = remaining - cum;
+                    s_prefix = prefix | ((uint32_t)digit << shift);
+                }
+            }
+            __syncthreads();
+            prefix = s_prefix;
+            remaining = s_remaining;
+            mask |= 255u << shift;
+        }
+        thr = prefix;
+        need_eq = remaining;       // how many of the keys equal to thr are taken (lowest positions)
+    }
+    if (tid == 0) s_first_evicted = n;
+    int cgt = 0, ceq = 0;
+#pragma unroll
+    for (int i = 0; i < KPT; ++i) {
+        const bool valid = j0 + i < n;
+        cgt += (valid && key[i] > thr) ? 1 : 0;
+        ceq += (valid && k > 0 && key[i] == thr) ? 1 : 0;
+    }
+    int tot;
+    const int eq_before = block_exclusive_scan_1024(ceq, warp_sums, tot);
+    const int take_eq = max(0, min(ceq, need_eq - eq_before));
+    int off = block_exclusive_scan_1024(cgt + take_eq, warp_sums, tot);
+    int eq_rank = eq_before, first_ev = n;
+#pragma unroll
+    for (int i = 0; i < KPT; ++i) {
+        const int j = j0 + i;
+        if (j < n) {
+            const bool gt = key[i] > thr, eq = k > 0 && key[i] == thr;
+            const bool keep = gt || (eq && eq_rank < need_eq);
+            if (eq) ++eq_rank;
+            if (keep) srcmap[off++] = T_first + j;
+            else first_ev = min(first_ev, j);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) first_ev = min(first_ev, __shfl_xor_sync(0xFFFFFFFFu, first_ev, o));
+    if (lane == 0 && first_ev < n) atomicMin(&s_first_evicted, first_ev);
+    __syncthreads();
+    if (tid == 0) dscal[0] = min(T_first + s_first_evicted, T_c) >> 6;
+}
+
+// ---------------------------------------------------------------------------
+// Eq. 9-11 for keys.  One block per (new 64-token group, head), 256 threads =
+// 64 member tokens x 4 quarters of 16 channels.  A thread fetches the 16 codes
+// of its (token, quarter) with one vector load and dequantises them (Eq. 12)
+// with the parameters of the token's old group, which the block stages in
+// shared memory (kept tokens stay in order, so a new group draws on a short
+// run of old groups); fresh tokens are widened from the frame's 16-bit keys.
+// The values stay in registers; a shared-memory tile serves only the
+// per-channel min/max over the 64 tokens.  Then parameters, codes, pack.
+// ---------------------------------------------------------------------------
+constexpr int RQ_WIN = 4;   // old groups whose parameters are staged; tokens from further on read global memory
+
 template <typename T, int BITS>
 __global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView dst, const T* __restrict__ Kf,
                                                         int F, int n_old_new, int T_new, int T_first,
@@ -247,6 +401,7 @@ __global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView
     constexpr int ROWB = XSV_D * BITS / 8;
     constexpr int WPR = ROWB / 4;              // 32-bit words per row
     constexpr int CPW = 32 / BITS;             // codes per word
+    constexpr int WPQ = WPR / 4;               // words per 16-channel quarter
     constexpr int NMAX = (1 << BITS) - 1;
     const int gi = g_base + blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
     const int fz = fz_dev ? *fz_dev : fz_host;
@@ -266,32 +421,74 @@ __global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView
 
     __shared__ float tile[XSV_G][XSV_D + 1];
     __shared__ float smn[4][64], smx[4][64];
-    __shared__ float ss[64];
+    __shared__ float ss[64], si[64];
     __shared__ int sz[64];
+    __shared__ float w_s[RQ_WIN][64];
+    __shared__ int w_z[RQ_WIN][64];
+    __shared__ int s_sp[XSV_G];
 
-    for (int i = tid; i < cnt * WPR; i += 256) {
-        const int m = i / WPR, j = i % WPR, p = p0 + m;
-        if (p < n_old_new) {
-            const int sp = (srcmap != nullptr && p >= T_first) ? srcmap[p - T_first] : p;
-            const uint32_t w = *reinterpret_cast<const uint32_t*>(src.kcodes + ((size_t)h * src.cap + sp) * ROWB + 4 * j);
-            const size_t mo = ((size_t)h * src.capg + (sp >> 6)) * 64 + j * CPW;
+    // old position of every member that comes from the cache (-1: fresh token)
+    if (tid < XSV_G) {
+        const int p = p0 + tid;
+        int sp = -1;
+        if (tid < cnt && p < n_old_new) sp = (srcmap != nullptr && p >= T_first) ? srcmap[p - T_first] : p;
+        s_sp[tid] = sp;
+    }
+    __syncthreads();
+    const int g_lo = s_sp[0] >> 6;             // members are in ascending old position; -1 >> 6 == -1: no cached member
+    if (g_lo >= 0) {
+        for (int i = tid; i < RQ_WIN * 64; i += 256) {
+            const int g = g_lo + (i >> 6);
+            if (g < src.capg) {
+                w_s[i >> 6][i & 63] = src.kscale[((size_t)h * src.capg + g) * 64 + (i & 63)];
+                w_z[i >> 6][i & 63] = src.kzero[((size_t)h * src.capg + g) * 64 + (i & 63)];
+            }
+        }
+    }
+    __syncthreads();
+
+    const int m = tid >> 2, q = tid & 3;       // member token, quarter of 16 channels
+    float x[16];
+    if (m < cnt) {
+        const int sp = s_sp[m];
+        if (sp >= 0) {
+            uint32_t w[WPQ];
+            const uint8_t* rowp = src.kcodes + ((size_t)h * src.cap + sp) * ROWB + q * (ROWB / 4);
+            if (WPQ == 1) w[0] = *reinterpret_cast<const uint32_t*>(rowp);
+            else if (WPQ == 2) { const uint2 t = *reinterpret_cast<const uint2*>(rowp); w[0] = t.x; w[WPQ - 1] = t.y; }
+            else { const uint4 t = *reinterpret_cast<const uint4*>(rowp); w[0] = t.x; w[1 % WPQ] = t.y; w[2 % WPQ] = t.z; w[3 % WPQ] = t.w; }
+            const int g = (sp >> 6) - g_lo;
+            const float* ps;
+            const int* pz;
+            if (g < RQ_WIN) { ps = &w_s[g][16 * q]; pz = &w_z[g][16 * q]; }
+            else { ps = src.kscale + ((size_t)h * src.capg + (sp >> 6)) * 64 + 16 * q; pz = src.kzero + ((size_t)h * src.capg + (sp >> 6)) * 64 + 16 * q; }
 #pragma unroll
-            for (int e = 0; e < CPW; ++e) {
-                int code = (int)((w >> (e * BITS)) & (uint32_t)NMAX);
-                tile[m][j * CPW + e] = xsv_dequant(code, src.kzero[mo + e], src.kscale[mo + e]);
+            for (int e = 0; e < 16; ++e) {
+                const int code = (int)((w[e / CPW] >> ((e % CPW) * BITS)) & (uint32_t)NMAX);
+                x[e] = xsv_dequant(code, pz[e], ps[e]);
             }
         } else {
-            const T* row = Kf + ((size_t)h * F + (p - n_old_new)) * XSV_D + j * CPW;
+            const T* row = Kf + ((size_t)h * F + (p0 + m - n_old_new)) * XSV_D + 16 * q;
+            const uint4 a = reinterpret_cast<const uint4*>(row)[0], b = reinterpret_cast<const uint4*>(row)[1];
+            const uint32_t u[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
 #pragma unroll
-            for (int e = 0; e < CPW; ++e) tile[m][j * CPW + e] = xsv_to_float<T>(row[e]);
+            for (int e = 0; e < 8; ++e) {
+                T lo, hi;
+                *reinterpret_cast<uint16_t*>(&lo) = (uint16_t)(u[e] & 0xFFFFu);
+                *reinterpret_cast<uint16_t*>(&hi) = (uint16_t)(u[e] >> 16);
+                x[2 * e] = xsv_to_float<T>(lo);
+                x[2 * e + 1] = xsv_to_float<T>(hi);
+            }
         }
+#pragma unroll
+        for (int e = 0; e < 16; ++e) tile[m][16 * q + e] = x[e];
     }
     __syncthreads();
     {
         const int c = tid & 63, part = tid >> 6;
         float mn = INFINITY, mx = -INFINITY;
-        for (int m = part; m < cnt; m += 4) {
-            float v = tile[m][c];
+        for (int mm = part; mm < cnt; mm += 4) {
+            const float v = tile[mm][c];
             mn = fminf(mn, v);
             mx = fmaxf(mx, v);
         }
@@ -300,26 +497,29 @@ __global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView
     }
     __syncthreads();
     if (tid < 64) {
-        float mn = fminf(fminf(smn[0][tid], smn[1][tid]), fminf(smn[2][tid], smn[3][tid]));
-        float mx = fmaxf(fmaxf(smx[0][tid], smx[1][tid]), fmaxf(smx[2][tid], smx[3][tid]));
+        const float mn = fminf(fminf(smn[0][tid], smn[1][tid]), fminf(smn[2][tid], smn[3][tid]));
+        const float mx = fmaxf(fmaxf(smx[0][tid], smx[1][tid]), fmaxf(smx[2][tid], smx[3][tid]));
         float s;
         int z;
         xsv_quant_params(mn, mx, NMAX, s, z, status);
         ss[tid] = s;
+        si[tid] = __frcp_rn(s);
         sz[tid] = z;
         dst.kscale[((size_t)h * dst.capg + gi) * 64 + tid] = s;
         dst.kzero[((size_t)h * dst.capg + gi) * 64 + tid] = z;
     }
     __syncthreads();
-    for (int i = tid; i < cnt * WPR; i += 256) {
-        const int m = i / WPR, j = i % WPR;
-        uint32_t w = 0;
+    if (m < cnt) {
+        uint32_t w[WPQ];
 #pragma unroll
-        for (int e = 0; e < CPW; ++e) {
-            const int c = j * CPW + e;
-            w |= (uint32_t)xsv_quant_code(tile[m][c], ss[c], sz[c], NMAX) << (e * BITS);
-        }
-        *reinterpret_cast<uint32_t*>(dst.kcodes + ((size_t)h * dst.cap + p0 + m) * ROWB + 4 * j) = w;
+        for (int j = 0; j < WPQ; ++j) w[j] = 0u;
+#pragma unroll
+        for (int e = 0; e < 16; ++e)
+            w[e / CPW] |= (uint32_t)xsv_quant_code(x[e], ss[16 * q + e], si[16 * q + e], sz[16 * q + e], NMAX) << ((e % CPW) * BITS);
+        uint8_t* rowp = dst.kcodes + ((size_t)h * dst.cap + p0 + m) * ROWB + q * (ROWB / 4);
+        if (WPQ == 1) *reinterpret_cast<uint32_t*>(rowp) = w[0];
+        else if (WPQ == 2) *reinterpret_cast<uint2*>(rowp) = make_uint2(w[0], w[WPQ - 1]);
+        else *reinterpret_cast<uint4*>(rowp) = make_uint4(w[0], w[1 % WPQ], w[2 % WPQ], w[3 % WPQ]);
     }
 }
 
@@ -407,7 +607,8 @@ __global__ void __launch_bounds__(256) quant_v_kernel(LayerView dst, const T* __
     float s;
     int z;
     xsv_quant_params(mn, mx, NMAX, s, z, status);
-    const uint32_t c0 = (uint32_t)xsv_quant_code(x0, s, z, NMAX), c1 = (uint32_t)xsv_quant_code(x1, s, z, NMAX);
+    const float inv_s = __frcp_rn(s);
+    const uint32_t c0 = (uint32_t)xsv_quant_code(x0, s, inv_s, z, NMAX), c1 = (uint32_t)xsv_quant_code(x1, s, inv_s, z, NMAX);
     uint32_t w = (c0 | (c1 << BITS)) << (2 * BITS * (lane % LPW));
 #pragma unroll
     for (int o = 1; o < LPW; o <<= 1) w |= __shfl_xor_sync(0xFFFFFFFFu, w, o);
@@ -437,8 +638,8 @@ cudaError_t xsv_launch_score(const LayerView& lv, int H, int T_first, int T_c, c
                              float* scores, cudaStream_t st) {
     const int n = T_c - T_first;
     if (n <= 0) return cudaSuccess;
-    const int grid = (n + SCORE_TPB - 1) / SCORE_TPB;
-    const size_t smem = (64 + 2 * (size_t)H * SCORE_MAXG * 64) * sizeof(float);
+    const int grid = (n + SCORE_TOK - 1) / SCORE_TOK;
+    const size_t smem = (64 + (size_t)H * SCORE_MAXG * 65) * sizeof(float);
     cudaError_t e = cudaSuccess;
 #define XSV_SCORE(B)                                                                                       \
     {                                                                                                      \
@@ -474,7 +675,11 @@ cudaError_t xsv_launch_score_raw(const LayerView& lv, int dtype, int H, int T_fi
 
 cudaError_t xsv_launch_select(const float* scores, int n, int k, int T_first, int T_c, int* srcmap, int* dscal,
                               cudaStream_t st) {
-    select_kernel<<<1, 1024, 0, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);
+    if (n <= 1024 * 8) select_reg_kernel<8><<<1, 1024, 0, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);
+    else if (n <= 1024 * 16) select_reg_kernel<16><<<1, 1024, 0, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);
+    else if (n <= 1024 * 24) select_reg_kernel<24><<<1, 1024, 0, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);
+    else if (n <= 1024 * 32) select_reg_kernel<32><<<1, 1024, 0, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);
+    else select_kernel<<<1, 1024, 0, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);
     xsv_count_launch();
     return cudaGetLastError();
 }

@@ -70,10 +70,18 @@ __device__ __forceinline__ void xsv_quant_params(float mn, float mx, int n, floa
     z = __float2int_rn(zf);   // saturates at the int32 limits
 }
 
-// Eq. 9: clamp(round(x / s) + z, 0, n), round = nearest-even.
-__device__ __forceinline__ int xsv_quant_code(float x, float s, int z, int n) {
-    int q = __float2int_rn(__fdiv_rn(x, s));   // saturating
-    long long v = (long long)q + (long long)z;
+// Eq. 9: clamp(round(x / s) + z, 0, n), round = nearest-even, with x / s the
+// IEEE float32 quotient.  inv_s = 1 / s (correctly rounded).  x * inv_s lies
+// within 2^-22 |x / s| of the true quotient, as does the rounded quotient
+// itself; unless x * inv_s comes within 2^-20 |x / s| of a rounding boundary
+// (a half-integer) both therefore round to the same integer, and the division
+// is skipped.  Near a boundary the exact division decides.
+__device__ __forceinline__ int xsv_quant_code(float x, float s, float inv_s, int z, int n) {
+    const float y = __fmul_rn(x, inv_s);
+    float r = rintf(y);
+    if (fabsf(fabsf(y - r) - 0.5f) < fabsf(y) * 9.5367431640625e-7f) r = rintf(__fdiv_rn(x, s));
+    const int q = __float2int_rn(r);   // saturating
+    const long long v = (long long)q + (long long)z;
     return (int)(v < 0 ? 0 : (v > n ? n : v));
 }
 
