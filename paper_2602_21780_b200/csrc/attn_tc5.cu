@@ -37,7 +37,8 @@ constexpr int NSTAGE = 5;          // kv stages in shared memory
 constexpr int NPROD = 7;              // producer warps
 constexpr int NTHREADS = (8 + NPROD + 1) * 32;   // 8 softmax warps, the producers, the MMA issuer
 constexpr uint32_t TILE_BYTES = 128u * 128u;   // 128 rows x 64 fp16
-constexpr int COST_PAIR = 4, COST_SINGLE = 3;  // relative cost of a kv step with two / one active query tile
+constexpr int COST_PAIR = 8, COST_SINGLE = 7;  // relative cost of a kv step with two / one active query tile (measured: the
+                                               // hand-over latencies, not the arithmetic, set the pace of a step)
 constexpr float RESCALE_THRESHOLD = 8.f;       // log2 units; below it the stale row maximum is kept
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
