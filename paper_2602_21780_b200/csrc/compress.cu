@@ -270,38 +270,24 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
 // registers, so the scores are read from memory once.  The four digit
 // histograms are built with warp-aggregated shared-memory atomics (scores
 // share their leading digits, which would otherwise serialise), the bins are
-// scanned by one warp, and the ordered compaction is a block-wide prefix sum
-// over per-thread counts.  Same total order as select_kernel.
+// scanned by one warp, and the ordered compaction works on warp ballots as in
+// select_kernel.  Same total order.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ int block_exclusive_scan_1024(int v, int* warp_sums, int& total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int incl = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t; }
-    __syncthreads();                       // warp_sums may still be read from a previous scan
-    if (lane == 31) warp_sums[warp] = incl;
-    __syncthreads();
-    int ws = warp_sums[lane], wincl = ws;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, wincl, o); if (lane >= o) wincl += t; }
-    total = __shfl_sync(0xFFFFFFFFu, wincl, 31);
-    const int wbase = __shfl_sync(0xFFFFFFFFu, wincl - ws, warp);
-    return wbase + incl - v;
-}
-
 template <int KPT>
 __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restrict__ scores, int n, int k, int T_first,
                                                           int T_c, int* __restrict__ srcmap, int* __restrict__ dscal) {
     __shared__ int hist[256];
-    __shared__ int warp_sums[32];
+    __shared__ int w_gt[32], w_eq[32], w_off[32], w_eqb[32];
     __shared__ uint32_t s_prefix;
     __shared__ int s_remaining;
     __shared__ int s_first_evicted;
-    const int tid = threadIdx.x, lane = tid & 31;
-    const int j0 = tid * KPT;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // warp w owns the contiguous positions [w * 32 * KPT, (w + 1) * 32 * KPT); lane l holds every 32nd of them
+    // (coalesced loads, and the ordered compaction below needs ballots only)
+    const int j0 = warp * 32 * KPT + lane;
     uint32_t key[KPT];
 #pragma unroll
-    for (int i = 0; i < KPT; ++i) key[i] = (j0 + i < n) ? score_key(scores[j0 + i]) : 0u;
+    for (int i = 0; i < KPT; ++i) key[i] = (j0 + 32 * i < n) ? score_key(scores[j0 + 32 * i]) : 0u;
 
     uint32_t thr = 0xFFFFFFFFu;
     int need_eq = 0;
@@ -314,10 +300,12 @@ __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restric
             __syncthreads();
 #pragma unroll
             for (int i = 0; i < KPT; ++i) {
-                const bool act = (j0 + i < n) && (key[i] & mask) == prefix;
-                const uint32_t digit = act ? ((key[i] >> shift) & 255u) : 256u;
-                const uint32_t peers = __match_any_sync(0xFFFFFFFFu, digit);
-                if (act && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+                const bool act = (j0 + 32 * i < n) && (key[i] & mask) == prefix;
+                if (__any_sync(0xFFFFFFFFu, act)) {
+                    const uint32_t digit = act ? ((key[i] >> shift) & 255u) : 256u;
+                    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, digit);
+                    if (act && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+                }
             }
             __syncthreads();
             if (tid < 32) {
@@ -329,8 +317,7 @@ __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restric
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t; }
                 int cum = incl - sum;          // count in the bins above this lane's
-                const bool here = cum < remaining && incl >= remaining;
-                if (here) {
+                if (cum < remaining && incl >= remaining) {
                     int digit = 0;
 #pragma unroll
                     for (int q = 0; q < 8; ++q) {
@@ -353,25 +340,41 @@ __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restric
     int cgt = 0, ceq = 0;
 #pragma unroll
     for (int i = 0; i < KPT; ++i) {
-        const bool valid = j0 + i < n;
-        cgt += (valid && key[i] > thr) ? 1 : 0;
-        ceq += (valid && k > 0 && key[i] == thr) ? 1 : 0;
+        const bool valid = j0 + 32 * i < n;
+        cgt += __popc(__ballot_sync(0xFFFFFFFFu, valid && key[i] > thr));
+        ceq += __popc(__ballot_sync(0xFFFFFFFFu, valid && k > 0 && key[i] == thr));
     }
-    int tot;
-    const int eq_before = block_exclusive_scan_1024(ceq, warp_sums, tot);
-    const int take_eq = max(0, min(ceq, need_eq - eq_before));
-    int off = block_exclusive_scan_1024(cgt + take_eq, warp_sums, tot);
-    int eq_rank = eq_before, first_ev = n;
+    if (lane == 0) { w_gt[warp] = cgt; w_eq[warp] = ceq; }
+    __syncthreads();
+    if (warp == 0) {
+        // exclusive scans over the 32 warps, in warp order
+        const int eq = w_eq[lane], gt = w_gt[lane];
+        int eq_incl = eq;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, eq_incl, o); if (lane >= o) eq_incl += t; }
+        const int eq_before = eq_incl - eq;
+        const int kept = gt + max(0, min(eq, need_eq - eq_before));
+        int k_incl = kept;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, k_incl, o); if (lane >= o) k_incl += t; }
+        w_off[lane] = k_incl - kept;
+        w_eqb[lane] = eq_before;
+    }
+    __syncthreads();
+    int off = w_off[warp], eqb = w_eqb[warp], first_ev = n;
+    const uint32_t lt = (1u << lane) - 1u;
 #pragma unroll
     for (int i = 0; i < KPT; ++i) {
-        const int j = j0 + i;
-        if (j < n) {
-            const bool gt = key[i] > thr, eq = k > 0 && key[i] == thr;
-            const bool keep = gt || (eq && eq_rank < need_eq);
-            if (eq) ++eq_rank;
-            if (keep) srcmap[off++] = T_first + j;
-            else first_ev = min(first_ev, j);
-        }
+        const int j = j0 + 32 * i;
+        const bool valid = j < n;
+        const bool gt = valid && key[i] > thr, eq = valid && k > 0 && key[i] == thr;
+        const uint32_t beq = __ballot_sync(0xFFFFFFFFu, eq);
+        const bool keep = gt || (eq && eqb + __popc(beq & lt) < need_eq);
+        const uint32_t bk = __ballot_sync(0xFFFFFFFFu, keep);
+        if (keep) srcmap[off + __popc(bk & lt)] = T_first + j;
+        if (valid && !keep) first_ev = min(first_ev, j);
+        off += __popc(bk);
+        eqb += __popc(beq);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) first_ev = min(first_ev, __shfl_xor_sync(0xFFFFFFFFu, first_ev, o));
@@ -419,12 +422,12 @@ __global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView
         return;
     }
 
-    __shared__ float tile[XSV_G][XSV_D + 1];
+    __shared__ __align__(16) float tile[XSV_G][XSV_D + 4];   // rows of 68 floats: 16-byte accesses, spread over the banks
     __shared__ float smn[4][64], smx[4][64];
-    __shared__ float ss[64], si[64];
-    __shared__ int sz[64];
-    __shared__ float w_s[RQ_WIN][64];
-    __shared__ int w_z[RQ_WIN][64];
+    __shared__ __align__(16) float ss[64], si[64];
+    __shared__ __align__(16) int sz[64];
+    __shared__ __align__(16) float w_s[RQ_WIN][64];
+    __shared__ __align__(16) int w_z[RQ_WIN][64];
     __shared__ int s_sp[XSV_G];
 
     // old position of every member that comes from the cache (-1: fresh token)
@@ -458,14 +461,25 @@ __global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView
             else if (WPQ == 2) { const uint2 t = *reinterpret_cast<const uint2*>(rowp); w[0] = t.x; w[WPQ - 1] = t.y; }
             else { const uint4 t = *reinterpret_cast<const uint4*>(rowp); w[0] = t.x; w[1 % WPQ] = t.y; w[2 % WPQ] = t.z; w[3 % WPQ] = t.w; }
             const int g = (sp >> 6) - g_lo;
-            const float* ps;
-            const int* pz;
-            if (g < RQ_WIN) { ps = &w_s[g][16 * q]; pz = &w_z[g][16 * q]; }
-            else { ps = src.kscale + ((size_t)h * src.capg + (sp >> 6)) * 64 + 16 * q; pz = src.kzero + ((size_t)h * src.capg + (sp >> 6)) * 64 + 16 * q; }
+            const float4* ps;
+            const int4* pz;
+            if (g < RQ_WIN) { ps = reinterpret_cast<const float4*>(&w_s[g][16 * q]); pz = reinterpret_cast<const int4*>(&w_z[g][16 * q]); }
+            else {
+                ps = reinterpret_cast<const float4*>(src.kscale + ((size_t)h * src.capg + (sp >> 6)) * 64 + 16 * q);
+                pz = reinterpret_cast<const int4*>(src.kzero + ((size_t)h * src.capg + (sp >> 6)) * 64 + 16 * q);
+            }
 #pragma unroll
-            for (int e = 0; e < 16; ++e) {
-                const int code = (int)((w[e / CPW] >> ((e % CPW) * BITS)) & (uint32_t)NMAX);
-                x[e] = xsv_dequant(code, pz[e], ps[e]);
+            for (int e4 = 0; e4 < 4; ++e4) {
+                const float4 s4 = ps[e4];
+                const int4 z4 = pz[e4];
+                const float sv[4] = {s4.x, s4.y, s4.z, s4.w};
+                const int zv[4] = {z4.x, z4.y, z4.z, z4.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int e = 4 * e4 + k;
+                    const int code = (int)((w[e / CPW] >> ((e % CPW) * BITS)) & (uint32_t)NMAX);
+                    x[e] = xsv_dequant(code, zv[k], sv[k]);
+                }
             }
         } else {
             const T* row = Kf + ((size_t)h * F + (p0 + m - n_old_new)) * XSV_D + 16 * q;
@@ -481,7 +495,8 @@ __global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView
             }
         }
 #pragma unroll
-        for (int e = 0; e < 16; ++e) tile[m][16 * q + e] = x[e];
+        for (int e4 = 0; e4 < 4; ++e4)
+            *reinterpret_cast<float4*>(&tile[m][16 * q + 4 * e4]) = make_float4(x[4 * e4], x[4 * e4 + 1], x[4 * e4 + 2], x[4 * e4 + 3]);
     }
     __syncthreads();
     {
@@ -514,8 +529,17 @@ __global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView
 #pragma unroll
         for (int j = 0; j < WPQ; ++j) w[j] = 0u;
 #pragma unroll
-        for (int e = 0; e < 16; ++e)
-            w[e / CPW] |= (uint32_t)xsv_quant_code(x[e], ss[16 * q + e], si[16 * q + e], sz[16 * q + e], NMAX) << ((e % CPW) * BITS);
+        for (int e4 = 0; e4 < 4; ++e4) {
+            const float4 s4 = reinterpret_cast<const float4*>(ss + 16 * q)[e4], i4 = reinterpret_cast<const float4*>(si + 16 * q)[e4];
+            const int4 z4 = reinterpret_cast<const int4*>(sz + 16 * q)[e4];
+            const float sv[4] = {s4.x, s4.y, s4.z, s4.w}, iv[4] = {i4.x, i4.y, i4.z, i4.w};
+            const int zv[4] = {z4.x, z4.y, z4.z, z4.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int e = 4 * e4 + k;
+                w[e / CPW] |= (uint32_t)xsv_quant_code(x[e], sv[k], iv[k], zv[k], NMAX) << ((e % CPW) * BITS);
+            }
+        }
         uint8_t* rowp = dst.kcodes + ((size_t)h * dst.cap + p0 + m) * ROWB + q * (ROWB / 4);
         if (WPQ == 1) *reinterpret_cast<uint32_t*>(rowp) = w[0];
         else if (WPQ == 2) *reinterpret_cast<uint2*>(rowp) = make_uint2(w[0], w[WPQ - 1]);

@@ -55,9 +55,17 @@ template <> __device__ __forceinline__ uint32_t xsv_pack2<__nv_bfloat16>(float a
     return *reinterpret_cast<uint32_t*>(&h);
 }
 
+// Exact int -> float for |v| < 2^22 without the conversion unit: 1.5 * 2^23 + v
+// is exact in float32 and so is the subtraction that follows.
+__device__ __forceinline__ float xsv_small_int_to_float(int v) {
+    return __fadd_rn(__int_as_float(0x4B400000 + v), -12582912.f);
+}
+
 // Eq. 12: x~ = (code - z) * s, one float32 multiply.
 __device__ __forceinline__ float xsv_dequant(int code, int z, float s) {
-    return __fmul_rn(__int2float_rn(code - z), s);
+    const int v = code - z;
+    const float f = (v > -4194304 && v < 4194304) ? xsv_small_int_to_float(v) : __int2float_rn(v);
+    return __fmul_rn(f, s);
 }
 
 // Eq. 10 in float32, one rounding per operation; degenerate groups
@@ -78,9 +86,17 @@ __device__ __forceinline__ void xsv_quant_params(float mn, float mx, int n, floa
 // is skipped.  Near a boundary the exact division decides.
 __device__ __forceinline__ int xsv_quant_code(float x, float s, float inv_s, int z, int n) {
     const float y = __fmul_rn(x, inv_s);
-    float r = rintf(y);
-    if (fabsf(fabsf(y - r) - 0.5f) < fabsf(y) * 9.5367431640625e-7f) r = rintf(__fdiv_rn(x, s));
-    const int q = __float2int_rn(r);   // saturating
+    int q;
+    if (fabsf(y) < 2097152.f) {
+        // round to nearest even by adding and subtracting 1.5 * 2^23 (exact for |y| < 2^21); the integer is
+        // in the low mantissa bits of the sum
+        const float t = __fadd_rn(y, 12582912.f);
+        const float r = __fadd_rn(t, -12582912.f);
+        q = __float_as_int(t) - 0x4B400000;
+        if (fabsf(fabsf(y - r) - 0.5f) < fabsf(y) * 9.5367431640625e-7f) q = __float2int_rn(rintf(__fdiv_rn(x, s)));
+    } else {
+        q = __float2int_rn(rintf(__fdiv_rn(x, s)));   // saturating
+    }
     const long long v = (long long)q + (long long)z;
     return (int)(v < 0 ? 0 : (v > n ? n : v));
 }
