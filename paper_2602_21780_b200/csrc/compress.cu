@@ -57,6 +57,7 @@ __global__ void __launch_bounds__(256) qtilde_partial_kernel(const T* __restrict
 constexpr int SCORE_TPB = 256;             // 64 tokens x 4 slices of the heads
 constexpr int SCORE_TOK = 64;              // tokens per block
 constexpr int SCORE_MAXG = 2;              // key groups a block's 64 tokens can span
+constexpr int SCORE_WS = 66;               // floats per staged weight row
 
 // Sum of the fixed-order partial sums of the pooled queries, scaled: q~[c].
 __device__ __forceinline__ float qtilde_channel(const float* __restrict__ qpart, int n_part, int c, float qnorm) {
@@ -77,8 +78,9 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
     constexpr int CPW = 32 / BITS;             // codes per 32-bit word
     extern __shared__ float sm[];
     float* qt = sm;                             // [64]
-    float* sW = qt + 64;                        // [H][SCORE_MAXG][64] weights q~_c * s_c
-    float* sB = sW + (size_t)H * SCORE_MAXG * 64;   // [H][SCORE_MAXG] bias sum_c q~_c s_c z_c
+    float* sW = qt + 64;                        // [H][SCORE_MAXG][SCORE_WS] weights q~_c * s_c (rows padded: the four
+                                                // heads read at once by a warp fall into different banks)
+    float* sB = sW + (size_t)H * SCORE_MAXG * SCORE_WS;   // [H][SCORE_MAXG] bias sum_c q~_c s_c z_c
 
     const int j0 = blockIdx.x * SCORE_TOK;
     const int p0 = T_first + j0;
@@ -92,7 +94,7 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
         const int k1 = min(np, (part + 1) * per);
 #pragma unroll 8
         for (int k = part * per; k < k1; ++k) s4 += qpart[(size_t)k * 64 + c];
-        sW[part * 64 + c] = s4;            // sW is free until the weights are staged
+        sW[part * 64 + c] = s4;            // sW (at least 256 floats, see the launcher) is free until the weights are staged
         __syncthreads();
         if (threadIdx.x < 64) qt[c] = (((sW[c] + sW[64 + c]) + sW[128 + c]) + sW[192 + c]) * qnorm;
     }
@@ -100,14 +102,14 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
     for (int i = threadIdx.x; i < H * ng * 64; i += SCORE_TPB) {
         const int c = i & 63, gg = (i >> 6) % ng, h = (i >> 6) / ng;
         const size_t m = ((size_t)h * lv.capg + g_lo + gg) * 64 + c;
-        sW[(h * SCORE_MAXG + gg) * 64 + c] = qt[c] * lv.kscale[m];
+        sW[(h * SCORE_MAXG + gg) * SCORE_WS + c] = qt[c] * lv.kscale[m];
     }
     __syncthreads();
     for (int i = threadIdx.x >> 5; i < H * ng; i += SCORE_TPB / 32) {   // one warp per (head, group): the bias
         const int gg = i % ng, h = i / ng, lane = threadIdx.x & 31;
         const size_t m = ((size_t)h * lv.capg + g_lo + gg) * 64;
-        float b = sW[(h * SCORE_MAXG + gg) * 64 + lane] * (float)lv.kzero[m + lane] +
-                  sW[(h * SCORE_MAXG + gg) * 64 + lane + 32] * (float)lv.kzero[m + lane + 32];
+        float b = sW[(h * SCORE_MAXG + gg) * SCORE_WS + lane] * (float)lv.kzero[m + lane] +
+                  sW[(h * SCORE_MAXG + gg) * SCORE_WS + lane + 32] * (float)lv.kzero[m + lane + 32];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) b += __shfl_xor_sync(0xFFFFFFFFu, b, o);
         if (lane == 0) sB[h * SCORE_MAXG + gg] = b;
@@ -121,7 +123,7 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
         const int gg = (p >> 6) - g_lo;
         for (int h = slice; h < H; h += 4) {
             const uint4* row = reinterpret_cast<const uint4*>(lv.kcodes + ((size_t)h * lv.cap + p) * ROWB);
-            const float* w = sW + (h * SCORE_MAXG + gg) * 64;
+            const float* w = sW + (h * SCORE_MAXG + gg) * SCORE_WS;
             float a = 0.f;
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
@@ -663,7 +665,7 @@ cudaError_t xsv_launch_score(const LayerView& lv, int H, int T_first, int T_c, c
     const int n = T_c - T_first;
     if (n <= 0) return cudaSuccess;
     const int grid = (n + SCORE_TOK - 1) / SCORE_TOK;
-    const size_t smem = (64 + (size_t)H * SCORE_MAXG * 65) * sizeof(float);
+    const size_t smem = (64 + ((size_t)H * SCORE_MAXG * (SCORE_WS + 1) > 256 ? (size_t)H * SCORE_MAXG * (SCORE_WS + 1) : 256)) * sizeof(float);
     cudaError_t e = cudaSuccess;
 #define XSV_SCORE(B)                                                                                       \
     {                                                                                                      \
