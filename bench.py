@@ -152,6 +152,23 @@ def oracle_layer_step_seconds(repeats=1):
     return best
 
 
+def replica_seed(base, rank):
+    """Every rank streams its own frames: the path does not shard, ranks are independent replicas."""
+    return base + rank
+
+
+def job_throughput(ms_local, steps, world, dist=None, device=None):
+    """Whole-job frames/s of `world` independent replicas: all ranks' frames over the slowest rank's time.
+    Returns (frames_per_s, ms_max).  `dist` is torch.distributed (initialised) when world > 1."""
+    ms = float(ms_local)
+    if world > 1:
+        import torch
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return world * steps / (ms * 1e-3), ms
+
+
 def blas_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -171,7 +188,7 @@ def run_reference(args, rank):
     sec = sum(times) / len(times)
     fps = 1.0 / (LAYERS * sec)
     cores = blas_threads()
-    line = {"impl": "reference", "metric": METRIC, "value": fps, "unit": "frames/s", "n_gpus": 0,
+    line = {"impl": "reference", "metric": METRIC, "value": fps, "unit": "frames/s", "n_gpus": args.gpus,
             "steps": len(times), "warmup": 1 if args.warmup else 0, "ms_per_step": LAYERS * sec * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic", "config": {"workload": WORKLOAD},
@@ -218,7 +235,7 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    frames = gen_frames(torch, dev, LAYERS, POOL, seed=20260221 + rank)
+    frames = gen_frames(torch, dev, LAYERS, POOL, seed=replica_seed(20260221, rank))
     out = torch.empty(H, F, D, device=dev, dtype=torch.bfloat16)
     stream = torch.cuda.current_stream()
     sp = stream.cuda_stream
@@ -274,11 +291,7 @@ def main():
     kv_layer = cache.layer_kv_bytes(0)
     total_bytes = cache.bytes()
 
-    if world > 1:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = world * args.steps / (ms * 1e-3)
+    value, ms = job_throughput(ms, args.steps, world, dist if world > 1 else None, dev)
 
     # ---- roofline of the dominant kernel (attention), live CUDA-event durations
     peaks = measured_peaks()
@@ -337,12 +350,9 @@ def main():
         torch.cuda.synchronize()
         wall = (time.perf_counter() - t0) * 1e3
         ems = max(e0.elapsed_time(e1), wall)
-        if world > 1:
-            t = torch.tensor([ems], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ems = float(t.item())
+        e2e_value, ems = job_throughput(ems, n_e2e, world, dist if world > 1 else None, dev)
         nb = H * F * D * 2
-        e2e = {"value": world * n_e2e / (ems * 1e-3), "unit": "frames/s", "h2d_bytes_per_step": 3 * nb * LAYERS,
+        e2e = {"value": e2e_value, "unit": "frames/s", "h2d_bytes_per_step": 3 * nb * LAYERS,
                "d2h_bytes_per_step": nb * LAYERS, "steps": n_e2e,
                "api": "xsv_step_host (pinned host Q/K/V in, host out back, per layer)"}
         c2.destroy()
