@@ -77,6 +77,23 @@ def test_config1_sampled_steps(impl):
     assert w["pruned_steps"] == 3
 
 
+def test_config3_shape_sampled_steps():
+    # long-horizon shape: 1374 tokens/frame, budget 10992 (8 frames), 2-bit, drifting means; a deeper layer's
+    # stream; verify the first step, the end of the ramp, the first pruning steps
+    c = synth.CONFIGS[3]
+    st = synth.config_stream(3, layer=17)
+    w = run_stream(st, 11, c["L_max"], c["bits"], check_steps={0, 7, 8, 9, 10})
+    assert w["pruned_steps"] == 3
+
+
+def test_config2_multi_layer_cache_is_per_layer():
+    # several layers in one cache object at paper shape: layers are independent caches; verify a middle one
+    c = synth.CONFIGS[2]
+    st = synth.config_stream(2, layer=5)
+    w = run_stream(st, 18, c["L_max"], c["bits"], check_steps={0, 16, 17}, layers=3, layer=1)
+    assert w["pruned_steps"] == 2
+
+
 @pytest.mark.parametrize("dtype", ["fp16", "bf16"])
 def test_importance_scores_entry_point(dtype):
     from oracle import xsv_oracle as orc
