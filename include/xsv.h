@@ -211,6 +211,16 @@ xsv_status xsv_cache_status(xsv_cache* c, void* stream);
 xsv_status xsv_cache_set_profiling(xsv_cache* c, int on);
 xsv_status xsv_cache_profile_read(xsv_cache* c, double ms[XSV_PHASE_COUNT], long long launches[XSV_PHASE_COUNT], int reset);
 
+/*
+ * Self-test of the bounded device-side waits (the library's kernels hand work
+ * over through barriers; a wait that is never satisfied must not hang the GPU).
+ * Launches one tiny kernel whose only wait nothing ends, synchronises `stream`,
+ * and returns XSV_ERR_TIMEOUT when the wait gave up after its limit (about two
+ * seconds) and reported it -- the expected outcome -- or XSV_OK if it did not.
+ * The context stays usable.  (The paper has no counterpart.)
+ */
+xsv_status xsv_selftest_bounded_wait(void* stream);
+
 /* Kernels launched by this library in the calling process since load. */
 long long xsv_kernel_launches(void);
 

@@ -37,6 +37,7 @@ SYMBOLS = {
     "xsv_cache_status": (_i, [_vp, _vp]),
     "xsv_cache_set_profiling": (_i, [_vp, _i]),
     "xsv_cache_profile_read": (_i, [_vp, C.POINTER(C.c_double), C.POINTER(_ll), _i]),
+    "xsv_selftest_bounded_wait": (_i, [_vp]),
     "xsv_kernel_launches": (_ll, []),
     "xsv_strerror": (C.c_char_p, [_i]),
     "xsv_last_cuda_error": (C.c_char_p, []),
@@ -208,6 +209,11 @@ def importance_scores_static(Q, keys, scores, n_special=5, pool_group=16, stream
     return int(load().xsv_importance_scores_static(Q.data_ptr(), keys.data_ptr(), Q.shape[0], Q.shape[1],
                                                    keys.shape[1], _dtype_code(Q), n_special, pool_group,
                                                    scores.data_ptr(), _stream_ptr(stream)))
+
+
+def selftest_bounded_wait(stream=None):
+    """xsv_selftest_bounded_wait: returns the status code (6 = the wait timed out and said so, as it should)."""
+    return int(load().xsv_selftest_bounded_wait(_stream_ptr(stream)))
 
 
 def kernel_launches():

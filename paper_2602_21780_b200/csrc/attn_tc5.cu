@@ -984,6 +984,20 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const Params p) {
     *dst = make_uint2(xsv_pack2<T>(acc.x * inv, acc.y * inv), xsv_pack2<T>(acc.z * inv, acc.w * inv));
 }
 
+// A wait that nothing ends: one barrier, no arrival.  Exercises the bounded wait of the attention kernel: it must
+// return after WAIT_LIMIT_NS with XSV_DEV_TIMEOUT in *status instead of hanging.
+__global__ void wait_selftest_kernel(int* status) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    mbar_wait(smem_u32(&bar), 0u, &abort_flag, status);
+}
+
 int sm_count() {
     static int n = 0;
     if (n == 0) {
@@ -1009,6 +1023,12 @@ cudaError_t launch(const Params& p, cudaStream_t st) {
 }
 
 }  // namespace
+
+cudaError_t xsv_launch_wait_selftest(int* status, cudaStream_t st) {
+    wait_selftest_kernel<<<1, 64, 0, st>>>(status);
+    xsv_count_launch();
+    return cudaGetLastError();
+}
 
 size_t xsv_attn_tc5_workspace_bytes() { return (size_t)sm_count() * 2 * PART_STRIDE * sizeof(float); }
 

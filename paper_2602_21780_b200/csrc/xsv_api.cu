@@ -409,6 +409,20 @@ xsv_status xsv_importance_scores(const void* Q, const void* keys, int heads, int
     return e == cudaSuccess ? XSV_OK : cuda_fail(e);
 }
 
+xsv_status xsv_selftest_bounded_wait(void* stream) {
+    cudaStream_t st = (cudaStream_t)stream;
+    int* d = nullptr;
+    if (cudaMalloc((void**)&d, sizeof(int)) != cudaSuccess) { cudaGetLastError(); return XSV_ERR_OOM; }
+    int w = 0;
+    cudaError_t e = cudaMemsetAsync(d, 0, sizeof(int), st);
+    if (e == cudaSuccess) e = xsv_launch_wait_selftest(d, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(&w, d, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    cudaFree(d);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return (w & XSV_DEV_TIMEOUT) ? XSV_ERR_TIMEOUT : XSV_OK;
+}
+
 size_t xsv_cache_bytes(const xsv_cache* c) { return c ? c->bytes : 0; }
 
 size_t xsv_cache_layer_kv_bytes(const xsv_cache* c, int layer) {

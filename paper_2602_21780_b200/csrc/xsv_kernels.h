@@ -61,3 +61,7 @@ size_t xsv_attn_tc5_workspace_bytes();
 cudaError_t xsv_launch_attn_tc5(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V,
                                 void* out, int dtype, int H, int F, float* workspace, int* status,
                                 cudaStream_t st);
+
+// One small kernel whose only wait can never be satisfied: it must come back after the
+// attention kernel's wait limit with XSV_DEV_TIMEOUT set in *status (device int).
+cudaError_t xsv_launch_wait_selftest(int* status, cudaStream_t st);

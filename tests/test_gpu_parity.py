@@ -156,3 +156,13 @@ def test_host_step_matches_device_step():
     for key in sa:
         assert np.array_equal(sa[key], sb[key])
     a.destroy(); b.destroy()
+
+
+def test_bounded_wait_times_out_and_reports():
+    # a wait that nothing satisfies returns after its limit with the timeout status; the context stays usable
+    import time
+    t0 = time.time()
+    assert binding.selftest_bounded_wait() == 6
+    assert 1.0 < time.time() - t0 < 30.0
+    x = torch.ones(4, device="cuda")
+    assert float(x.sum()) == 4.0
