@@ -326,8 +326,9 @@ def main():
     e2e = None
     if not args.no_e2e:
         hq = [[tuple(t.cpu().pin_memory() for t in fr) for fr in per[:2]] for per in frames]
-        hout = torch.empty(H, F, D, dtype=torch.bfloat16).pin_memory()
+        houts = [torch.empty(H, F, D, dtype=torch.bfloat16).pin_memory() for _ in range(LAYERS)]
         c2 = make_cache()
+        c2.set_host_pipelining(True)          # results travel back while the next layer computes
         for f in range(PREFILL + 3):
             frame_step(c2, f)
         n_e2e = max(3, min(args.steps, 10))
@@ -335,8 +336,9 @@ def main():
         def host_frame(f):
             for l in range(LAYERS):
                 q, k, v = hq[l][f % 2]
-                c2.step_host(l, q, k, v, hout, stream)
-            torch.cuda.synchronize()       # the frame's result is on the host
+                c2.step_host(l, q, k, v, houts[l], stream)
+            c2.host_flush(stream)
+            torch.cuda.synchronize()       # the frame's results are on the host
 
         host_frame(0)
         if world > 1:
@@ -354,7 +356,7 @@ def main():
         nb = H * F * D * 2
         e2e = {"value": e2e_value, "unit": "frames/s", "h2d_bytes_per_step": 3 * nb * LAYERS,
                "d2h_bytes_per_step": nb * LAYERS, "steps": n_e2e,
-               "api": "xsv_step_host (pinned host Q/K/V in, host out back, per layer)"}
+               "api": "xsv_step_host (pinned host Q/K/V in, host out back, per layer; copies overlap the kernels), xsv_cache_host_flush + synchronise per frame"}
         c2.destroy()
 
     cpu = None

@@ -113,13 +113,29 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
                     int n_tokens, xsv_dtype dtype, void* out, void* stream);
 
 /*
- * Same step with HOST buffers: copies Q, K, V to device staging owned by the
- * cache, runs xsv_step, copies `out` back, all on `stream`, and returns
- * without synchronising.  Pinned host memory makes the copies asynchronous.
+ * Same step with HOST buffers (pinned host memory makes the copies asynchronous).
+ * The inputs are copied to device staging owned by the cache on an internal
+ * stream, so that the copy of one call overlaps the kernels of the previous
+ * one; the step itself runs on `stream`; the call returns without
+ * synchronising.  Q_host, K_host, V_host must stay unchanged until `stream` has
+ * passed the call.
+ *   Default: `out_host` is written on `stream`: it is complete once `stream`
+ *   has passed the call.
+ *   With xsv_cache_set_host_pipelining(c, 1) the result is copied back on a
+ *   second internal stream and the next step does not wait for it: `out_host`
+ *   is complete once `stream` has passed a later xsv_cache_host_flush(c, stream)
+ *   (at most two results are in flight; a third call waits for the first).
  */
 xsv_status xsv_step_host(xsv_cache* c, int layer, const void* Q_host, const void* K_host,
                          const void* V_host, int n_tokens, xsv_dtype dtype, void* out_host,
                          void* stream);
+
+/* Deferred copy-back of xsv_step_host results (see there); off by default.
+ * XSV_ERR_ORDER while results are in flight (flush first). */
+xsv_status xsv_cache_set_host_pipelining(xsv_cache* c, int defer_output);
+
+/* Makes `stream` wait for every result of xsv_step_host still on its way to the host. */
+xsv_status xsv_cache_host_flush(xsv_cache* c, void* stream);
 
 /*
  * Eq. 3-7 on their own: importance scores of `n_keys` keys for one frame's

@@ -25,6 +25,8 @@ SYMBOLS = {
     "xsv_cache_set_attn_impl": (_i, [_vp, _i]),
     "xsv_step": (_i, [_vp, _i, _vp, _vp, _vp, _i, _i, _vp, _vp]),
     "xsv_step_host": (_i, [_vp, _i, _vp, _vp, _vp, _i, _i, _vp, _vp]),
+    "xsv_cache_set_host_pipelining": (_i, [_vp, _i]),
+    "xsv_cache_host_flush": (_i, [_vp, _vp]),
     "xsv_importance_scores": (_i, [_vp, _vp, _i, _i, _ll, _i, _i, _i, _vp, _vp]),
     "xsv_importance_scores_static": (_i, [_vp, _vp, _i, _i, _ll, _i, _i, _i, _vp, _vp]),
     "xsv_cache_bytes": (C.c_size_t, [_vp]),
@@ -125,6 +127,12 @@ class Cache:
                 raise ValueError("xsv.step_host needs contiguous host tensors")
         _check(self._lib.xsv_step_host(self._h, layer, Q.data_ptr(), K.data_ptr(), V.data_ptr(), Q.shape[1],
                                        _dtype_code(Q), out.data_ptr(), _stream_ptr(stream)), "xsv_step_host")
+
+    def set_host_pipelining(self, defer_output):
+        _check(self._lib.xsv_cache_set_host_pipelining(self._h, int(defer_output)), "xsv_cache_set_host_pipelining")
+
+    def host_flush(self, stream=None):
+        _check(self._lib.xsv_cache_host_flush(self._h, _stream_ptr(stream)), "xsv_cache_host_flush")
 
     def bytes(self):
         return int(self._lib.xsv_cache_bytes(self._h))

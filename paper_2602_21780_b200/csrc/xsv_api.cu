@@ -65,9 +65,14 @@ struct xsv_cache {
     void* scratch_slab = nullptr;
     long long last_scores_n = 0;
 
-    // staging for xsv_step_host
+    // staging for xsv_step_host: two slots of (Q, K, V, out), a copy-in and a copy-out stream
     void* stage = nullptr;
     size_t stage_bytes = 0;
+    cudaStream_t cs_in = nullptr, cs_out = nullptr;
+    cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
+    bool slot_used[2] = {false, false}, out_pending[2] = {false, false};
+    bool defer_output = false;
+    unsigned long long host_calls = 0;
 
     size_t bytes = 0;
 
@@ -367,20 +372,69 @@ xsv_status xsv_step_host(xsv_cache* c, int layer, const void* Qh, const void* Kh
     if (c->F != 0 && n_tokens != c->F) return XSV_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
     const size_t nb = (size_t)c->H * n_tokens * c->d * 2;
-    if (c->stage_bytes < 4 * nb) {
+    cudaError_t e = cudaSuccess;
+    if (c->stage_bytes < 8 * nb) {
         cudaSetDevice(c->device);
-        if (c->stage) { cudaStreamSynchronize(st); cudaFree(c->stage); c->bytes -= c->stage_bytes; c->stage = nullptr; c->stage_bytes = 0; }
-        if (cudaMalloc(&c->stage, 4 * nb) != cudaSuccess) { cudaGetLastError(); return XSV_ERR_OOM; }
-        c->stage_bytes = 4 * nb;
+        if (c->stage) { cudaDeviceSynchronize(); cudaFree(c->stage); c->bytes -= c->stage_bytes; c->stage = nullptr; c->stage_bytes = 0; }
+        if (cudaMalloc(&c->stage, 8 * nb) != cudaSuccess) { cudaGetLastError(); return XSV_ERR_OOM; }
+        c->stage_bytes = 8 * nb;
         c->bytes += c->stage_bytes;
+        c->slot_used[0] = c->slot_used[1] = c->out_pending[0] = c->out_pending[1] = false;
     }
-    uint8_t* s = (uint8_t*)c->stage;
-    if (cudaMemcpyAsync(s, Qh, nb, cudaMemcpyHostToDevice, st) != cudaSuccess) return XSV_ERR_CUDA;
-    if (cudaMemcpyAsync(s + nb, Kh, nb, cudaMemcpyHostToDevice, st) != cudaSuccess) return XSV_ERR_CUDA;
-    if (cudaMemcpyAsync(s + 2 * nb, Vh, nb, cudaMemcpyHostToDevice, st) != cudaSuccess) return XSV_ERR_CUDA;
+    if (!c->cs_in) {
+        if ((e = cudaStreamCreateWithFlags(&c->cs_in, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamCreateWithFlags(&c->cs_out, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+        for (int i = 0; i < 2; ++i) {
+            if ((e = cudaEventCreateWithFlags(&c->ev_in[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaEventCreateWithFlags(&c->ev_done[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaEventCreateWithFlags(&c->ev_out[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+        }
+    }
+    // Two staging slots alternate.  The inputs of this call are copied on a stream of their own, as soon as the
+    // step that last used the slot has finished, so the copy overlaps the previous call's kernels.
+    const int slot = (int)(c->host_calls & 1ull);
+    uint8_t* s = (uint8_t*)c->stage + (size_t)slot * 4 * nb;
+    if (c->slot_used[slot] && (e = cudaStreamWaitEvent(c->cs_in, c->ev_done[slot], 0)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(s, Qh, nb, cudaMemcpyHostToDevice, c->cs_in)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(s + nb, Kh, nb, cudaMemcpyHostToDevice, c->cs_in)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(s + 2 * nb, Vh, nb, cudaMemcpyHostToDevice, c->cs_in)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaEventRecord(c->ev_in[slot], c->cs_in)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaStreamWaitEvent(st, c->ev_in[slot], 0)) != cudaSuccess) return cuda_fail(e);
+    if (c->out_pending[slot]) {   // the slot's previous result must have left before the step overwrites it
+        if ((e = cudaStreamWaitEvent(st, c->ev_out[slot], 0)) != cudaSuccess) return cuda_fail(e);
+        c->out_pending[slot] = false;
+    }
     xsv_status r = xsv_step(c, layer, s, s + nb, s + 2 * nb, n_tokens, dtype, s + 3 * nb, stream);
     if (r != XSV_OK) return r;
-    if (cudaMemcpyAsync(out_h, s + 3 * nb, nb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return XSV_ERR_CUDA;
+    ++c->host_calls;
+    c->slot_used[slot] = true;
+    if ((e = cudaEventRecord(c->ev_done[slot], st)) != cudaSuccess) return cuda_fail(e);
+    if (!c->defer_output) {
+        if ((e = cudaMemcpyAsync(out_h, s + 3 * nb, nb, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+    } else {
+        if ((e = cudaStreamWaitEvent(c->cs_out, c->ev_done[slot], 0)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpyAsync(out_h, s + 3 * nb, nb, cudaMemcpyDeviceToHost, c->cs_out)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventRecord(c->ev_out[slot], c->cs_out)) != cudaSuccess) return cuda_fail(e);
+        c->out_pending[slot] = true;
+    }
+    return XSV_OK;
+}
+
+xsv_status xsv_cache_set_host_pipelining(xsv_cache* c, int defer_output) {
+    if (!c) return XSV_ERR_ARG;
+    if (c->out_pending[0] || c->out_pending[1]) return XSV_ERR_ORDER;   // flush first
+    c->defer_output = defer_output != 0;
+    return XSV_OK;
+}
+
+xsv_status xsv_cache_host_flush(xsv_cache* c, void* stream) {
+    if (!c) return XSV_ERR_ARG;
+    for (int i = 0; i < 2; ++i) {
+        if (!c->out_pending[i]) continue;
+        const cudaError_t e = cudaStreamWaitEvent((cudaStream_t)stream, c->ev_out[i], 0);
+        if (e != cudaSuccess) return cuda_fail(e);
+        c->out_pending[i] = false;
+    }
     return XSV_OK;
 }
 
@@ -440,6 +494,13 @@ void xsv_cache_destroy(xsv_cache* c) {
     for (auto& b : c->bufs) if (b.slab) cudaFree(b.slab);
     if (c->scratch_slab) cudaFree(c->scratch_slab);
     if (c->stage) cudaFree(c->stage);
+    for (int i = 0; i < 2; ++i) {
+        if (c->ev_in[i]) cudaEventDestroy(c->ev_in[i]);
+        if (c->ev_done[i]) cudaEventDestroy(c->ev_done[i]);
+        if (c->ev_out[i]) cudaEventDestroy(c->ev_out[i]);
+    }
+    if (c->cs_in) cudaStreamDestroy(c->cs_in);
+    if (c->cs_out) cudaStreamDestroy(c->cs_out);
     for (auto& p : c->pending) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
     for (auto e : c->free_events) cudaEventDestroy(e);
     delete c;

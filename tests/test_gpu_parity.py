@@ -138,19 +138,27 @@ def test_api_errors_and_bytes_constant():
     c.destroy()
 
 
-def test_host_step_matches_device_step():
+@pytest.mark.parametrize("defer", [False, True])
+def test_host_step_matches_device_step(defer):
     st = synth.Stream(H=4, d=64, F=90, dtype="bf16", layer=8)
     a = binding.Cache(1, 4, 64, 300, 4)
     b = binding.Cache(1, 4, 64, 300, 4)
-    for t in range(6):
+    a.set_host_pipelining(defer)
+    hosts, devs = [], []
+    for t in range(7):
         q, k, v = (torch.from_numpy(x).to(torch.bfloat16) for x in st.frame(t))
         Qh, Kh, Vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
         oh = torch.empty_like(Qh).pin_memory()
-        a.step_host(0, Qh, Kh, Vh, oh)
+        a.step_host(0, Qh, Kh, Vh, oh)              # no synchronisation between calls: copies and kernels overlap
+        hosts.append((Qh, Kh, Vh, oh))
         Q, K, V = q.cuda(), k.cuda(), v.cuda()
         od = torch.empty_like(Q)
         b.step(0, Q, K, V, od)
-        torch.cuda.synchronize()
+        devs.append(od)
+    if defer:
+        a.host_flush()
+    torch.cuda.synchronize()
+    for (_, _, _, oh), od in zip(hosts, devs):
         assert torch.equal(oh, od.cpu())
     sa, sb = a.export_layer(0), b.export_layer(0)
     for key in sa:
