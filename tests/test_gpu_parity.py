@@ -174,3 +174,36 @@ def test_bounded_wait_times_out_and_reports():
     assert 1.0 < time.time() - t0 < 30.0
     x = torch.ones(4, device="cuda")
     assert float(x.sum()) == 4.0
+
+
+def test_long_horizon_stream_stays_flat():
+    # config-3 shape (1374 tokens/frame, budget 10992, 2-bit), fewer layers and frames than the full run:
+    # once pruning has started the cache bytes, the cache length and the per-frame time must stay flat
+    H, F, L, bits, layers, frames = 16, 1374, 10992, 2, 4, 300
+    g = torch.Generator(device="cuda")
+    g.manual_seed(3)
+    pool = [tuple(torch.randn(H, F, 64, device="cuda", generator=g).to(torch.bfloat16) for _ in range(3)) for _ in range(5)]
+    out = torch.empty(H, F, 64, device="cuda", dtype=torch.bfloat16)
+    c = binding.Cache(layers, H, 64, L, bits)
+    times, ev = [], [torch.cuda.Event(enable_timing=True) for _ in range(frames + 1)]
+    bytes_seen = set()
+    ev[0].record()
+    for t in range(frames):
+        q, k, v = pool[t % len(pool)]
+        for l in range(layers):
+            c.step(l, q, k, v, out)
+        ev[t + 1].record()
+        if t >= 9:
+            bytes_seen.add(c.bytes())
+            assert c.len(layers - 1) == L
+    torch.cuda.synchronize()
+    assert c.status() == 0
+    assert len(bytes_seen) == 1                                   # constant device memory
+    assert torch.isfinite(out.float()).all()
+    times = [ev[t].elapsed_time(ev[t + 1]) for t in range(frames)]
+    steady = sorted(times[20:])
+    p50, p99 = steady[len(steady) // 2], steady[int(len(steady) * 0.99)]
+    first, last = sum(times[20:60]) / 40, sum(times[-40:]) / 40
+    assert p99 < 1.5 * p50, (p50, p99)
+    assert abs(last - first) < 0.15 * first, (first, last)        # no drift of the per-frame time
+    c.destroy()
