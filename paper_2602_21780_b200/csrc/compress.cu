@@ -426,9 +426,9 @@ __global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView
 
     __shared__ __align__(16) float tile[XSV_G][XSV_D + 4];   // rows of 68 floats: 16-byte accesses, spread over the banks
     __shared__ float smn[4][64], smx[4][64];
-    __shared__ __align__(16) float ss[64], si[64];
+    __shared__ __align__(16) float ss[64], si[64], szf[64];   // new scale, its reciprocal, the zero-point as a float (NaN: too large)
     __shared__ __align__(16) int sz[64];
-    __shared__ __align__(16) float w_s[RQ_WIN][64];
+    __shared__ __align__(16) float w_s[RQ_WIN][64], w_zc[RQ_WIN][64];   // old scale; -(2^23 + z) as a float (NaN: |z| too large)
     __shared__ __align__(16) int w_z[RQ_WIN][64];
     __shared__ int s_sp[XSV_G];
 
@@ -445,8 +445,10 @@ __global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView
         for (int i = tid; i < RQ_WIN * 64; i += 256) {
             const int g = g_lo + (i >> 6);
             if (g < src.capg) {
+                const int z = src.kzero[((size_t)h * src.capg + g) * 64 + (i & 63)];
                 w_s[i >> 6][i & 63] = src.kscale[((size_t)h * src.capg + g) * 64 + (i & 63)];
-                w_z[i >> 6][i & 63] = src.kzero[((size_t)h * src.capg + g) * 64 + (i & 63)];
+                w_z[i >> 6][i & 63] = z;
+                w_zc[i >> 6][i & 63] = (z > -4194304 && z < 4194304) ? -(float)(8388608 + z) : __int_as_float(0x7FC00000);
             }
         }
     }
@@ -463,24 +465,29 @@ __global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView
             else if (WPQ == 2) { const uint2 t = *reinterpret_cast<const uint2*>(rowp); w[0] = t.x; w[WPQ - 1] = t.y; }
             else { const uint4 t = *reinterpret_cast<const uint4*>(rowp); w[0] = t.x; w[1 % WPQ] = t.y; w[2 % WPQ] = t.z; w[3 % WPQ] = t.w; }
             const int g = (sp >> 6) - g_lo;
-            const float4* ps;
-            const int4* pz;
-            if (g < RQ_WIN) { ps = reinterpret_cast<const float4*>(&w_s[g][16 * q]); pz = reinterpret_cast<const int4*>(&w_z[g][16 * q]); }
-            else {
-                ps = reinterpret_cast<const float4*>(src.kscale + ((size_t)h * src.capg + (sp >> 6)) * 64 + 16 * q);
-                pz = reinterpret_cast<const int4*>(src.kzero + ((size_t)h * src.capg + (sp >> 6)) * 64 + 16 * q);
-            }
+            if (g < RQ_WIN) {
+                // float(code - z) without the conversion unit: (2^23 + code) + (-(2^23 + z)), both exact
+                const float4* ps = reinterpret_cast<const float4*>(&w_s[g][16 * q]);
+                const float4* pc = reinterpret_cast<const float4*>(&w_zc[g][16 * q]);
 #pragma unroll
-            for (int e4 = 0; e4 < 4; ++e4) {
-                const float4 s4 = ps[e4];
-                const int4 z4 = pz[e4];
-                const float sv[4] = {s4.x, s4.y, s4.z, s4.w};
-                const int zv[4] = {z4.x, z4.y, z4.z, z4.w};
+                for (int e4 = 0; e4 < 4; ++e4) {
+                    const float4 s4 = ps[e4], c4 = pc[e4];
+                    const float sv[4] = {s4.x, s4.y, s4.z, s4.w}, cv[4] = {c4.x, c4.y, c4.z, c4.w};
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int e = 4 * e4 + k;
+                    for (int k = 0; k < 4; ++k) {
+                        const int e = 4 * e4 + k;
+                        const uint32_t code = (w[e / CPW] >> ((e % CPW) * BITS)) & (uint32_t)NMAX;
+                        if (cv[k] == cv[k]) x[e] = __fmul_rn(__fadd_rn(__uint_as_float(0x4B000000u | code), cv[k]), sv[k]);
+                        else x[e] = xsv_dequant((int)code, w_z[g][16 * q + e], sv[k]);
+                    }
+                }
+            } else {
+                const float* ps = src.kscale + ((size_t)h * src.capg + (sp >> 6)) * 64 + 16 * q;
+                const int* pz = src.kzero + ((size_t)h * src.capg + (sp >> 6)) * 64 + 16 * q;
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
                     const int code = (int)((w[e / CPW] >> ((e % CPW) * BITS)) & (uint32_t)NMAX);
-                    x[e] = xsv_dequant(code, zv[k], sv[k]);
+                    x[e] = xsv_dequant(code, pz[e], ps[e]);
                 }
             }
         } else {
@@ -522,6 +529,7 @@ __global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView
         ss[tid] = s;
         si[tid] = __frcp_rn(s);
         sz[tid] = z;
+        szf[tid] = (z > -2097152 && z < 2097152) ? (float)z : __int_as_float(0x7FC00000);
         dst.kscale[((size_t)h * dst.capg + gi) * 64 + tid] = s;
         dst.kzero[((size_t)h * dst.capg + gi) * 64 + tid] = z;
     }
@@ -532,14 +540,26 @@ __global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView
         for (int j = 0; j < WPQ; ++j) w[j] = 0u;
 #pragma unroll
         for (int e4 = 0; e4 < 4; ++e4) {
-            const float4 s4 = reinterpret_cast<const float4*>(ss + 16 * q)[e4], i4 = reinterpret_cast<const float4*>(si + 16 * q)[e4];
-            const int4 z4 = reinterpret_cast<const int4*>(sz + 16 * q)[e4];
-            const float sv[4] = {s4.x, s4.y, s4.z, s4.w}, iv[4] = {i4.x, i4.y, i4.z, i4.w};
-            const int zv[4] = {z4.x, z4.y, z4.z, z4.w};
+            const float4 s4 = reinterpret_cast<const float4*>(ss + 16 * q)[e4], i4 = reinterpret_cast<const float4*>(si + 16 * q)[e4],
+                         f4 = reinterpret_cast<const float4*>(szf + 16 * q)[e4];
+            const float sv[4] = {s4.x, s4.y, s4.z, s4.w}, iv[4] = {i4.x, i4.y, i4.z, i4.w}, fv[4] = {f4.x, f4.y, f4.z, f4.w};
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const int e = 4 * e4 + k;
-                w[e / CPW] |= (uint32_t)xsv_quant_code(x[e], sv[k], iv[k], zv[k], NMAX) << ((e % CPW) * BITS);
+                // Eq. 9 in the float domain (see xsv_quant_code for why x * (1/s) may stand in for x / s): round by
+                // adding 1.5 * 2^23, add the zero-point (exact: both are integers below 2^22), clamp, and read the code
+                // off the mantissa.  Near a rounding boundary, for huge quotients or zero-points: the general routine.
+                const float y = __fmul_rn(x[e], iv[k]);
+                const float t = __fadd_rn(y, 12582912.f);
+                const float r = __fadd_rn(t, -12582912.f);
+                uint32_t code;
+                if (fabsf(y - r) > fmaf(fabsf(y), -9.5367431640625e-7f, 0.5f) || fv[k] != fv[k]) {
+                    code = (uint32_t)xsv_quant_code(x[e], sv[k], iv[k], sz[16 * q + e], NMAX);
+                } else {
+                    const float c = fminf(fmaxf(__fadd_rn(r, fv[k]), 0.f), (float)NMAX);
+                    code = __float_as_uint(__fadd_rn(c, 12582912.f)) & 0xFFu;
+                }
+                w[e / CPW] |= code << ((e % CPW) * BITS);
             }
         }
         uint8_t* rowp = dst.kcodes + ((size_t)h * dst.cap + p0 + m) * ROWB + q * (ROWB / 4);
