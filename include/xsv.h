@@ -209,6 +209,25 @@ xsv_status xsv_cache_export_layer(xsv_cache* c, int layer, unsigned char* k_code
                                   void* stream);
 
 /*
+ * The inverse of xsv_cache_export_layer: load one layer's logical state from
+ * HOST arrays (checkpoint restore; also the way to continue a stream on another
+ * cache object).  Synchronises `stream`.
+ *   n_cached     : T, tokens in the arrays; at most the cache's capacity
+ *                  (max(budget, 2 * frame_tokens), or max_cache_tokens when unbounded).
+ *   frames_done  : frames this layer has been stepped with (the next step is
+ *                  frame frames_done + 1; all layers must agree before stepping on).
+ *   frame_tokens, dtype : F and the element type of the stream (fixed per cache).
+ *   arrays       : as in xsv_cache_export_layer (codes one per byte, < 2^bits;
+ *                  k_raw / v_raw instead when bits == 16); `origin` is required.
+ * Errors leave the cache unchanged, except XSV_ERR_CUDA.
+ */
+xsv_status xsv_cache_import_layer(xsv_cache* c, int layer, long long n_cached, long long frames_done,
+                                  int frame_tokens, xsv_dtype dtype, const unsigned char* k_codes,
+                                  const float* k_scale, const int* k_zero, const unsigned char* v_codes,
+                                  const float* v_scale, const int* v_zero, const long long* origin,
+                                  const unsigned short* k_raw, const unsigned short* v_raw, void* stream);
+
+/*
  * Importance scores (Eq. 7) of the last pruning step of any layer, copied to
  * a HOST array of capacity `cap` floats; *n receives their count (the length
  * of the prunable middle segment), 0 if the last step did not prune.

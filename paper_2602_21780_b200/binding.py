@@ -35,6 +35,7 @@ SYMBOLS = {
     "xsv_cache_len": (_ll, [_vp, _i]),
     "xsv_cache_frames": (_ll, [_vp, _i]),
     "xsv_cache_export_layer": (_i, [_vp, _i] + [_vp] * 9 + [_vp]),
+    "xsv_cache_import_layer": (_i, [_vp, _i, _ll, _ll, _i, _i] + [_vp] * 9 + [_vp]),
     "xsv_last_scores": (_i, [_vp, _vp, _ll, C.POINTER(_ll), _vp]),
     "xsv_cache_status": (_i, [_vp, _vp]),
     "xsv_cache_set_profiling": (_i, [_vp, _i]),
@@ -165,6 +166,17 @@ class Cache:
         _check(self._lib.xsv_cache_export_layer(self._h, layer, *args, _stream_ptr(stream)),
                "xsv_cache_export_layer")
         return st
+
+    def import_layer(self, layer, st, frames_done, frame_tokens, dtype_code, stream=None):
+        """Load a state dict as returned by export_layer (see xsv_cache_import_layer)."""
+        def ptr(name):
+            a = st.get(name)
+            return np.ascontiguousarray(a).ctypes.data_as(C.c_void_p) if a is not None else None
+        keep = {k: np.ascontiguousarray(v) for k, v in st.items() if isinstance(v, np.ndarray)}   # alive during the call
+        args = [keep[k].ctypes.data_as(C.c_void_p) if k in keep else None
+                for k in ("Kc", "Ks", "Kz", "Vc", "Vs", "Vz", "origin", "Kraw", "Vraw")]
+        _check(self._lib.xsv_cache_import_layer(self._h, layer, int(st["T"]), int(frames_done), int(frame_tokens),
+                                                int(dtype_code), *args, _stream_ptr(stream)), "xsv_cache_import_layer")
 
     def last_scores(self, stream=None):
         """Importance scores (Eq. 7) of the most recent pruning step; empty if it did not prune."""

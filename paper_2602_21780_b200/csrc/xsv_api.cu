@@ -560,6 +560,71 @@ xsv_status xsv_cache_export_layer(xsv_cache* c, int layer, unsigned char* k_code
     return XSV_OK;
 }
 
+xsv_status xsv_cache_import_layer(xsv_cache* c, int layer, long long n_cached, long long frames_done, int frame_tokens,
+                                  xsv_dtype dtype, const unsigned char* k_codes, const float* k_scale, const int* k_zero,
+                                  const unsigned char* v_codes, const float* v_scale, const int* v_zero,
+                                  const long long* origin, const unsigned short* k_raw, const unsigned short* v_raw,
+                                  void* stream) {
+    if (!c || layer < 0 || layer >= c->layers || n_cached < 0 || frames_done < 0 || frame_tokens <= 0 || !origin) return XSV_ERR_ARG;
+    if (dtype != XSV_F16 && dtype != XSV_BF16) return XSV_ERR_ARG;
+    if (c->bits == 16 ? (!k_raw || !v_raw) : (!k_codes || !k_scale || !k_zero || !v_codes || !v_scale || !v_zero)) return XSV_ERR_ARG;
+    if (c->F != 0 && frame_tokens != c->F) return XSV_ERR_SHAPE;
+    if (c->dtype >= 0 && (int)dtype != c->dtype) return XSV_ERR_SHAPE;
+    if (c->n_special > frame_tokens) return XSV_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!c->allocated) {
+        c->F = frame_tokens;
+        cudaSetDevice(c->device);
+        const xsv_status s = allocate(c);
+        if (s != XSV_OK) { c->F = 0; return s; }
+    }
+    if (n_cached > c->cap) return XSV_ERR_CAPACITY;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return XSV_ERR_CUDA;
+    const LayerView& lv = c->bufs[c->buf_of_layer[layer]].view;
+    const int H = c->H, d = c->d, rowb = lv.rowb, bits = c->bits;
+    const long long T = n_cached, groups = (T + XSV_G - 1) / XSV_G;
+    cudaError_t e = cudaSuccess;
+    if (T > 0) {
+        std::vector<uint8_t> tmp((size_t)T * rowb);
+        for (int pass = 0; pass < 2 && e == cudaSuccess; ++pass) {
+            uint8_t* dev = pass == 0 ? lv.kcodes : lv.vcodes;
+            const unsigned char* codes = pass == 0 ? k_codes : v_codes;
+            const unsigned short* raw = pass == 0 ? k_raw : v_raw;
+            for (int h = 0; h < H && e == cudaSuccess; ++h) {
+                if (bits == 16) {
+                    memcpy(tmp.data(), raw + (size_t)h * T * d, (size_t)T * rowb);
+                } else {
+                    memset(tmp.data(), 0, tmp.size());
+                    const unsigned mask = (1u << bits) - 1u;
+                    for (long long p = 0; p < T; ++p)
+                        for (int ch = 0; ch < d; ++ch) {
+                            const unsigned code = codes[((size_t)h * T + p) * d + ch];
+                            if (code > mask) return XSV_ERR_ARG;
+                            const int bit = ch * bits;
+                            tmp[(size_t)p * rowb + bit / 8] |= (uint8_t)(code << (bit % 8));
+                        }
+                }
+                e = cudaMemcpy(dev + (size_t)h * lv.cap * rowb, tmp.data(), (size_t)T * rowb, cudaMemcpyHostToDevice);
+            }
+        }
+        if (bits < 16) {
+            for (int h = 0; h < H && e == cudaSuccess; ++h) {
+                e = cudaMemcpy(lv.kscale + (size_t)h * lv.capg * 64, k_scale + (size_t)h * groups * 64, (size_t)groups * 64 * 4, cudaMemcpyHostToDevice);
+                if (e == cudaSuccess) e = cudaMemcpy(lv.kzero + (size_t)h * lv.capg * 64, k_zero + (size_t)h * groups * 64, (size_t)groups * 64 * 4, cudaMemcpyHostToDevice);
+                if (e == cudaSuccess) e = cudaMemcpy(lv.vscale + (size_t)h * lv.cap, v_scale + (size_t)h * T, (size_t)T * 4, cudaMemcpyHostToDevice);
+                if (e == cudaSuccess) e = cudaMemcpy(lv.vzero + (size_t)h * lv.cap, v_zero + (size_t)h * T, (size_t)T * 4, cudaMemcpyHostToDevice);
+            }
+        }
+        if (e == cudaSuccess) e = cudaMemcpy(lv.origin, origin, (size_t)T * 8, cudaMemcpyHostToDevice);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    c->len[layer] = T;
+    c->frames[layer] = frames_done;
+    c->dtype = (int)dtype;
+    c->stepped = true;
+    return XSV_OK;
+}
+
 xsv_status xsv_last_scores(xsv_cache* c, float* scores_host, long long cap, long long* n, void* stream) {
     if (!c || !n) return XSV_ERR_ARG;
     *n = c->last_scores_n;

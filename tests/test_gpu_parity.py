@@ -56,6 +56,41 @@ def test_quantisation_off(L_max):
     run_stream(st, 6, L_max, 16, max_cache_tokens=400 if L_max == 0 else -1)
 
 
+def test_quantise_only_unbounded_cache():
+    # ablation "quantisation without pruning": no budget, 4-bit cache growing up to its capacity
+    st = synth.Stream(H=2, d=64, F=50, dtype="bf16", layer=10)
+    w = run_stream(st, 6, 0, 4, max_cache_tokens=400)
+    assert w["pruned_steps"] == 0
+
+
+@pytest.mark.parametrize("bits", [4, 16])
+def test_checkpoint_restore_continues_the_stream(bits):
+    # export after 5 frames, import into a fresh cache, step both on: same outputs, same state
+    st = synth.Stream(H=4, d=64, F=70, dtype="bf16", layer=11)
+    a = binding.Cache(2, 4, 64, 260, bits)
+    frames = [tuple(torch.from_numpy(x).to("cuda:0", torch.bfloat16).contiguous() for x in st.frame(t)) for t in range(8)]
+    out_a, out_b = torch.empty_like(frames[0][0]), torch.empty_like(frames[0][0])
+    for t in range(5):
+        for l in range(2):
+            a.step(l, *frames[t], out_a)
+    b = binding.Cache(2, 4, 64, 260, bits)
+    for l in range(2):
+        b.import_layer(l, a.export_layer(l), frames_done=5, frame_tokens=70, dtype_code=binding.BF16)
+    assert b.len(0) == a.len(0) and b.frames(1) == 5
+    for t in range(5, 8):
+        for l in range(2):
+            a.step(l, *frames[t], out_a)
+            b.step(l, *frames[t], out_b)
+            torch.cuda.synchronize()
+            assert torch.equal(out_a, out_b)
+    for l in range(2):
+        sa, sb = a.export_layer(l), b.export_layer(l)
+        for key in sa:
+            assert np.array_equal(sa[key], sb[key])
+    assert a.status() == 0 and b.status() == 0
+    a.destroy(); b.destroy()
+
+
 def test_pooling_options_and_multi_layer():
     st = synth.Stream(H=4, d=64, F=37, dtype="fp16", layer=7)
     run_stream(st, 6, 100, 4, n_special=1, g=4, layers=3, layer=2)
