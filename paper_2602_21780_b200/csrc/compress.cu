@@ -386,186 +386,355 @@ __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restric
 }
 
 // ---------------------------------------------------------------------------
-// Eq. 9-11 for keys.  One block per (new 64-token group, head), 256 threads =
-// 64 member tokens x 4 quarters of 16 channels.  A thread fetches the 16 codes
-// of its (token, quarter) with one vector load and dequantises them (Eq. 12)
-// with the parameters of the token's old group, which the block stages in
-// shared memory (kept tokens stay in order, so a new group draws on a short
-// run of old groups); fresh tokens are widened from the frame's 16-bit keys.
-// The values stay in registers; a shared-memory tile serves only the
-// per-channel min/max over the 64 tokens.  Then parameters, codes, pack.
+// Eq. 9-11 for keys.  One warp per (new 64-token group, head), no block-level
+// synchronisation; warps walk the (group, head) items with a stride of the
+// whole grid.  A warp first copies the packed rows of the group's 64 members
+// into its slice of shared memory (all loads in flight at once) together with
+// the parameters of the old groups they come from (kept tokens stay in order,
+// so a new group draws on a short run of old groups).  Lane (tq, w) owns the
+// 8 channels [8w, 8w + 8) of the members tq, tq + 4, ..., tq + 60: eight lanes
+// cover one packed row, and a row's 8 new codes are one store of 8 * bits bits.
+// Pass 1 dequantises (Eq. 12) or widens the frame's 16-bit keys and keeps a
+// running min / max per channel; two shuffles finish the reduction over the 64
+// tokens.  Each lane derives the parameters of two channels (Eq. 10) and
+// publishes them through shared memory.  Pass 2 re-derives the values and
+// writes the codes (Eq. 9).
+//
+// The arithmetic is arranged for the pipes it runs on (integer and min/max
+// instructions issue at half the rate of float multiply-adds):
+//  * a code is not shifted down before it is widened: (word & mask_k) | 2^23,
+//    read as a float, is 2^23 + code * 2^(bits k); the staged constants are
+//    -(2^23 + z * 2^(bits k)) and s * 2^-(bits k), so one add and one multiply
+//    give (code - z) * s with the same single rounding as Eq. 12;
+//  * the clamp of Eq. 9 is a saturating multiply by 1/n, and a row's codes are
+//    summed into 16-bit sub-words by multiply-adds (n * 2^(bits k) each) and
+//    converted once per sub-word.
 // ---------------------------------------------------------------------------
-constexpr int RQ_WIN = 4;   // old groups whose parameters are staged; tokens from further on read global memory
+constexpr int RQ_WIN = 4;                  // old groups whose parameters are staged; tokens from further on read global memory
+constexpr int RQ_THREADS = 256;
+
+template <int BITS>
+struct RqCfg {
+    static constexpr int ROWB = XSV_D * BITS / 8;
+    static constexpr int SUB = (BITS == 8) ? 2 : (BITS == 4 ? 4 : 8);   // codes per 16-bit sub-word
+    static constexpr int NSUB = 8 / SUB;                                // sub-words per lane (8 codes)
+    static constexpr int ZLIM = 1 << (22 - BITS * (SUB - 1));           // |z| below this: 2^23 + z * 2^(bits k) is exact
+    static constexpr int CODE_WORDS = XSV_G * ROWB / 4;
+    // per warp, in 4-byte words: old scale and offset constants, new scale / reciprocal / z as float / z,
+    // old positions, packed rows
+    static constexpr int WORDS = 2 * RQ_WIN * 64 + 4 * 64 + 64 + CODE_WORDS;
+    static constexpr int OFF_CODES = 2 * RQ_WIN * 64 + 4 * 64 + 64;
+};
+
+__device__ __forceinline__ float rq_min3(float a, float b, float c) {
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float rq_max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float rq_mul_sat(float a, float b) {
+    float d;
+    asm("mul.rn.sat.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+
+// 16-bit sub-word j of a lane's 8 codes (the upper half of the register is ignored by the masks).
+template <int BITS>
+__device__ __forceinline__ uint32_t rq_sub(uint64_t ch, int j) { return (uint32_t)(ch >> (16 * j)); }
+
+// General form of Eq. 12 for a row whose old group is outside the staged window or has parameters the fast
+// form cannot take: parameters from memory, one conversion per code.
+template <int BITS>
+__device__ __forceinline__ void rq_fetch_slow(const float* __restrict__ ks, const int* __restrict__ kz, uint64_t ch, float (&x)[8]) {
+    constexpr uint32_t NMAX = (1u << BITS) - 1u;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) x[e] = xsv_dequant((int)((uint32_t)(ch >> (e * BITS)) & NMAX), kz[e], ks[e]);
+}
+
+template <typename T>
+__device__ __forceinline__ void rq_fetch_fresh(const T* __restrict__ row, float (&x)[8]) {
+    const uint4 a = *reinterpret_cast<const uint4*>(row);
+    const uint32_t u[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        T lo, hi;
+        *reinterpret_cast<uint16_t*>(&lo) = (uint16_t)(u[e] & 0xFFFFu);
+        *reinterpret_cast<uint16_t*>(&hi) = (uint16_t)(u[e] >> 16);
+        x[2 * e] = xsv_to_float<T>(lo);
+        x[2 * e + 1] = xsv_to_float<T>(hi);
+    }
+}
+
+// General form of Eq. 9 for the 8 codes of one (token, channel octet).
+template <int BITS>
+__device__ __forceinline__ uint64_t rq_codes_slow(const float (&x)[8], const float* ns, const float* ni, const int* nz) {
+    uint64_t out = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+        out |= (uint64_t)(uint32_t)xsv_quant_code(x[e], ns[e], ni[e], nz[e], (1 << BITS) - 1) << (e * BITS);
+    return out;
+}
 
 template <typename T, int BITS>
-__global__ void __launch_bounds__(256) requant_k_kernel(LayerView src, LayerView dst, const T* __restrict__ Kf,
-                                                        int F, int n_old_new, int T_new, int T_first,
-                                                        const int* __restrict__ srcmap,
-                                                        const int* __restrict__ fz_dev, int fz_host,
-                                                        int g_base, int* __restrict__ status) {
-    constexpr int ROWB = XSV_D * BITS / 8;
-    constexpr int WPR = ROWB / 4;              // 32-bit words per row
-    constexpr int CPW = 32 / BITS;             // codes per word
-    constexpr int WPQ = WPR / 4;               // words per 16-channel quarter
+__global__ void __launch_bounds__(RQ_THREADS, 3) requant_k_kernel(LayerView src, LayerView dst, const T* __restrict__ Kf,
+                                                               int H, int F, int n_old_new, int T_new, int T_first,
+                                                               const int* __restrict__ srcmap,
+                                                               const int* __restrict__ fz_dev, int fz_host,
+                                                               int g_base, int n_items, int* __restrict__ status) {
+    using C = RqCfg<BITS>;
+    constexpr int ROWB = C::ROWB, SUB = C::SUB, NSUB = C::NSUB;
     constexpr int NMAX = (1 << BITS) - 1;
-    const int gi = g_base + blockIdx.x, h = blockIdx.y, tid = threadIdx.x;
+    constexpr uint32_t FULL = 0xFFFFFFFFu;
+    constexpr float KINV = 1.f / (float)NMAX;
+    extern __shared__ __align__(16) float rq_sm[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
+    const int tq = lane >> 3, w = lane & 7;
+    float* w_s = rq_sm + (size_t)warp * C::WORDS;
+    float* w_zc = w_s + RQ_WIN * 64;
+    float* n_s = w_zc + RQ_WIN * 64;
+    float* n_i = n_s + 64;
+    float* n_zf = n_i + 64;
+    int* n_z = reinterpret_cast<int*>(n_zf + 64);
+    int* s_sp = n_z + 64;
+    uint8_t* s_codes = reinterpret_cast<uint8_t*>(w_s + C::OFF_CODES);
     const int fz = fz_dev ? *fz_dev : fz_host;
     const bool same = (src.kcodes == dst.kcodes);
-    const int p0 = gi * XSV_G;
-    const int cnt = min(XSV_G, T_new - p0);
+    // position of this lane's staging channels (lane and lane + 32: same position) inside their 16-bit sub-word
+    const int pos_shift = BITS * ((lane & 7) % SUB);
+    const float pos_scale = __int_as_float((127 - pos_shift) << 23);
 
-    if (gi < fz) {   // frozen: the group keeps its members, positions, codes and parameters
-        if (same) return;
-        const uint32_t* s = reinterpret_cast<const uint32_t*>(src.kcodes + ((size_t)h * src.cap + p0) * ROWB);
-        uint32_t* d = reinterpret_cast<uint32_t*>(dst.kcodes + ((size_t)h * dst.cap + p0) * ROWB);
-        for (int i = tid; i < XSV_G * WPR; i += 256) d[i] = s[i];
-        if (tid < 64) dst.kscale[((size_t)h * dst.capg + gi) * 64 + tid] = src.kscale[((size_t)h * src.capg + gi) * 64 + tid];
-        else if (tid < 128) dst.kzero[((size_t)h * dst.capg + gi) * 64 + tid - 64] = src.kzero[((size_t)h * src.capg + gi) * 64 + tid - 64];
-        return;
-    }
+    // item of round r: r * (warps of the grid) + warp * (blocks) + block, so that a last, partial round is spread over
+    // all blocks (and so over all multiprocessors)
+    for (int it = warp * gridDim.x + blockIdx.x; it < n_items; it += gridDim.x * wpb) {
+        const int gi = g_base + it / H, h = it % H;
+        const int p0 = gi * XSV_G;
+        const int cnt = min(XSV_G, T_new - p0);
+        const size_t prm = ((size_t)h * dst.capg + gi) * 64;
 
-    __shared__ __align__(16) float tile[XSV_G][XSV_D + 4];   // rows of 68 floats: 16-byte accesses, spread over the banks
-    __shared__ float smn[4][64], smx[4][64];
-    __shared__ __align__(16) float ss[64], si[64], szf[64];   // new scale, its reciprocal, the zero-point as a float (NaN: too large)
-    __shared__ __align__(16) int sz[64];
-    __shared__ __align__(16) float w_s[RQ_WIN][64], w_zc[RQ_WIN][64];   // old scale; -(2^23 + z) as a float (NaN: |z| too large)
-    __shared__ __align__(16) int w_z[RQ_WIN][64];
-    __shared__ int s_sp[XSV_G];
-
-    // old position of every member that comes from the cache (-1: fresh token)
-    if (tid < XSV_G) {
-        const int p = p0 + tid;
-        int sp = -1;
-        if (tid < cnt && p < n_old_new) sp = (srcmap != nullptr && p >= T_first) ? srcmap[p - T_first] : p;
-        s_sp[tid] = sp;
-    }
-    __syncthreads();
-    const int g_lo = s_sp[0] >> 6;             // members are in ascending old position; -1 >> 6 == -1: no cached member
-    if (g_lo >= 0) {
-        for (int i = tid; i < RQ_WIN * 64; i += 256) {
-            const int g = g_lo + (i >> 6);
-            if (g < src.capg) {
-                const int z = src.kzero[((size_t)h * src.capg + g) * 64 + (i & 63)];
-                w_s[i >> 6][i & 63] = src.kscale[((size_t)h * src.capg + g) * 64 + (i & 63)];
-                w_z[i >> 6][i & 63] = z;
-                w_zc[i >> 6][i & 63] = (z > -4194304 && z < 4194304) ? -(float)(8388608 + z) : __int_as_float(0x7FC00000);
-            }
+        if (gi < fz) {   // frozen: the group keeps its members, positions, codes and parameters
+            if (same) continue;
+            const uint32_t* s = reinterpret_cast<const uint32_t*>(src.kcodes + ((size_t)h * src.cap + p0) * ROWB);
+            uint32_t* d = reinterpret_cast<uint32_t*>(dst.kcodes + ((size_t)h * dst.cap + p0) * ROWB);
+#pragma unroll 4
+            for (int i = lane; i < XSV_G * ROWB / 4; i += 32) d[i] = s[i];
+            const size_t sprm = ((size_t)h * src.capg + gi) * 64;
+            dst.kscale[prm + lane] = src.kscale[sprm + lane];
+            dst.kscale[prm + lane + 32] = src.kscale[sprm + lane + 32];
+            dst.kzero[prm + lane] = src.kzero[sprm + lane];
+            dst.kzero[prm + lane + 32] = src.kzero[sprm + lane + 32];
+            continue;
         }
-    }
-    __syncthreads();
 
-    const int m = tid >> 2, q = tid & 3;       // member token, quarter of 16 channels
-    float x[16];
-    if (m < cnt) {
-        const int sp = s_sp[m];
-        if (sp >= 0) {
-            uint32_t w[WPQ];
-            const uint8_t* rowp = src.kcodes + ((size_t)h * src.cap + sp) * ROWB + q * (ROWB / 4);
-            if (WPQ == 1) w[0] = *reinterpret_cast<const uint32_t*>(rowp);
-            else if (WPQ == 2) { const uint2 t = *reinterpret_cast<const uint2*>(rowp); w[0] = t.x; w[WPQ - 1] = t.y; }
-            else { const uint4 t = *reinterpret_cast<const uint4*>(rowp); w[0] = t.x; w[1 % WPQ] = t.y; w[2 % WPQ] = t.z; w[3 % WPQ] = t.w; }
-            const int g = (sp >> 6) - g_lo;
-            if (g < RQ_WIN) {
-                // float(code - z) without the conversion unit: (2^23 + code) + (-(2^23 + z)), both exact
-                const float4* ps = reinterpret_cast<const float4*>(&w_s[g][16 * q]);
-                const float4* pc = reinterpret_cast<const float4*>(&w_zc[g][16 * q]);
+        // old position of every member (-1: a token of the frame, -2: past the end)
+        int spv[2];
 #pragma unroll
-                for (int e4 = 0; e4 < 4; ++e4) {
-                    const float4 s4 = ps[e4], c4 = pc[e4];
-                    const float sv[4] = {s4.x, s4.y, s4.z, s4.w}, cv[4] = {c4.x, c4.y, c4.z, c4.w};
+        for (int k = 0; k < 2; ++k) {
+            const int tk = lane + 32 * k, p = p0 + tk;
+            int sp = -2;
+            if (tk < cnt) sp = (p >= n_old_new) ? -1 : ((srcmap != nullptr && p >= T_first) ? srcmap[p - T_first] : p);
+            s_sp[tk] = sp;
+            spv[k] = sp;
+        }
+        __syncwarp();
+        const int g_lo = s_sp[0] >> 6;     // members are in ascending old position; -1 >> 6 == -1: none cached
+        uint32_t slow_rows = 0;
+        if (g_lo >= 0) {
+            // packed rows of the cached members
+            constexpr int PPR = ROWB / 16;
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        const int e = 4 * e4 + k;
-                        const uint32_t code = (w[e / CPW] >> ((e % CPW) * BITS)) & (uint32_t)NMAX;
-                        if (cv[k] == cv[k]) x[e] = __fmul_rn(__fadd_rn(__uint_as_float(0x4B000000u | code), cv[k]), sv[k]);
-                        else x[e] = xsv_dequant((int)code, w_z[g][16 * q + e], sv[k]);
+            for (int j = 0; j < 2 * PPR; ++j) {
+                const int idx = lane + 32 * j, row = idx / PPR, piece = idx % PPR;
+                const int sp = s_sp[row];
+                if (sp >= 0)
+                    reinterpret_cast<uint4*>(s_codes)[idx] =
+                        *reinterpret_cast<const uint4*>(src.kcodes + ((size_t)h * src.cap + sp) * ROWB + 16 * piece);
+            }
+            // parameters of the staged old groups: lane l takes channels l and l + 32 of each row
+            bool slow[RQ_WIN];
+            const float* ksp = src.kscale + ((size_t)h * src.capg + g_lo) * 64 + lane;
+            const int* kzp = src.kzero + ((size_t)h * src.capg + g_lo) * 64 + lane;
+#pragma unroll
+            for (int r = 0; r < RQ_WIN; ++r) {
+                slow[r] = false;
+                if (g_lo + r < src.capg) {
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        const int z = kzp[r * 64 + 32 * k];
+                        const float sc = ksp[r * 64 + 32 * k];
+                        const bool ok = z > -C::ZLIM && z < C::ZLIM && sc >= 7.8886090522101181e-31f /* 2^-100 */;
+                        w_s[r * 64 + 32 * k + lane] = sc * pos_scale;
+                        w_zc[r * 64 + 32 * k + lane] = -(float)(8388608 + (ok ? (z << pos_shift) : 0));
+                        slow[r] |= !ok;
                     }
                 }
-            } else {
-                const float* ps = src.kscale + ((size_t)h * src.capg + (sp >> 6)) * 64 + 16 * q;
-                const int* pz = src.kzero + ((size_t)h * src.capg + (sp >> 6)) * 64 + 16 * q;
+            }
 #pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const int code = (int)((w[e / CPW] >> ((e % CPW) * BITS)) & (uint32_t)NMAX);
-                    x[e] = xsv_dequant(code, pz[e], ps[e]);
+            for (int r = 0; r < RQ_WIN; ++r) slow_rows |= __any_sync(FULL, slow[r]) ? (1u << r) : 0u;
+        }
+        __syncwarp();
+
+        // members whose old group lies in the first g + 1 staged rows (they are the first nb[g] members)
+        int nb[RQ_WIN];
+#pragma unroll
+        for (int g = 0; g < RQ_WIN; ++g) {
+            const bool a = spv[0] >= 0 && (spv[0] >> 6) - g_lo <= g, b = spv[1] >= 0 && (spv[1] >> 6) - g_lo <= g;
+            nb[g] = __popc(__ballot_sync(FULL, a)) + __popc(__ballot_sync(FULL, b));
+        }
+
+        const uint8_t* const cbase = s_codes + tq * ROWB + w * BITS;   // this lane's octet of member tq; member tq + 4 i is 4 i rows on
+        auto chunk_of = [&](int i) -> uint64_t {
+            const uint8_t* cp = cbase + i * (4 * ROWB);
+            if (BITS == 2) return *reinterpret_cast<const uint16_t*>(cp);
+            if (BITS == 4) return *reinterpret_cast<const uint32_t*>(cp);
+            const uint2 t = *reinterpret_cast<const uint2*>(cp);
+            return (uint64_t)t.x | ((uint64_t)t.y << 32);
+        };
+        // Walks this lane's members tq, tq + 4, ...: run by run of members that share a staged old group (the group's
+        // constants are loaded once per run; two members per step where the run allows), then whatever is left -- old
+        // groups outside the window or with parameters the fast form cannot take, and the frame's tokens -- one by one
+        // in the general form.  one(i, x) / two(i, x0, x1) receive the values of member tq + 4 i (and tq + 4 i + 4).
+        auto walk = [&](auto&& one, auto&& two) {
+            int i = 0;
+            if (g_lo >= 0) {
+#pragma unroll 1
+                for (int g = 0; g < RQ_WIN; ++g) {
+                    const int i_end = min(16, max(0, (nb[g] - tq + 3) >> 2));
+                    if (i >= i_end) continue;
+                    if ((slow_rows >> g) & 1u) break;
+                    const float4 s0 = *reinterpret_cast<const float4*>(w_s + g * 64 + 8 * w), s1 = *reinterpret_cast<const float4*>(w_s + g * 64 + 8 * w + 4);
+                    const float4 c0 = *reinterpret_cast<const float4*>(w_zc + g * 64 + 8 * w), c1 = *reinterpret_cast<const float4*>(w_zc + g * 64 + 8 * w + 4);
+                    const float sv[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+                    const float cv[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+                    auto deq = [&](uint64_t ch, float (&x)[8]) {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const uint32_t m = (rq_sub<BITS>(ch, e / SUB) & ((uint32_t)NMAX << (BITS * (e % SUB)))) | 0x4B000000u;
+                            x[e] = __fmul_rn(__fadd_rn(__uint_as_float(m), cv[e]), sv[e]);
+                        }
+                    };
+#pragma unroll 1
+                    for (; i + 1 < i_end; i += 2) {
+                        const uint64_t ch0 = chunk_of(i), ch1 = chunk_of(i + 1);
+                        float x0[8], x1[8];
+                        deq(ch0, x0);
+                        deq(ch1, x1);
+                        two(i, x0, x1);
+                    }
+                    if (i < i_end) {
+                        float x0[8];
+                        deq(chunk_of(i), x0);
+                        one(i, x0);
+                        ++i;
+                    }
                 }
             }
-        } else {
-            const T* row = Kf + ((size_t)h * F + (p0 + m - n_old_new)) * XSV_D + 16 * q;
-            const uint4 a = reinterpret_cast<const uint4*>(row)[0], b = reinterpret_cast<const uint4*>(row)[1];
-            const uint32_t u[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                T lo, hi;
-                *reinterpret_cast<uint16_t*>(&lo) = (uint16_t)(u[e] & 0xFFFFu);
-                *reinterpret_cast<uint16_t*>(&hi) = (uint16_t)(u[e] >> 16);
-                x[2 * e] = xsv_to_float<T>(lo);
-                x[2 * e + 1] = xsv_to_float<T>(hi);
-            }
-        }
-#pragma unroll
-        for (int e4 = 0; e4 < 4; ++e4)
-            *reinterpret_cast<float4*>(&tile[m][16 * q + 4 * e4]) = make_float4(x[4 * e4], x[4 * e4 + 1], x[4 * e4 + 2], x[4 * e4 + 3]);
-    }
-    __syncthreads();
-    {
-        const int c = tid & 63, part = tid >> 6;
-        float mn = INFINITY, mx = -INFINITY;
-        for (int mm = part; mm < cnt; mm += 4) {
-            const float v = tile[mm][c];
-            mn = fminf(mn, v);
-            mx = fmaxf(mx, v);
-        }
-        smn[part][c] = mn;
-        smx[part][c] = mx;
-    }
-    __syncthreads();
-    if (tid < 64) {
-        const float mn = fminf(fminf(smn[0][tid], smn[1][tid]), fminf(smn[2][tid], smn[3][tid]));
-        const float mx = fmaxf(fmaxf(smx[0][tid], smx[1][tid]), fmaxf(smx[2][tid], smx[3][tid]));
-        float s;
-        int z;
-        xsv_quant_params(mn, mx, NMAX, s, z, status);
-        ss[tid] = s;
-        si[tid] = __frcp_rn(s);
-        sz[tid] = z;
-        szf[tid] = (z > -2097152 && z < 2097152) ? (float)z : __int_as_float(0x7FC00000);
-        dst.kscale[((size_t)h * dst.capg + gi) * 64 + tid] = s;
-        dst.kzero[((size_t)h * dst.capg + gi) * 64 + tid] = z;
-    }
-    __syncthreads();
-    if (m < cnt) {
-        uint32_t w[WPQ];
-#pragma unroll
-        for (int j = 0; j < WPQ; ++j) w[j] = 0u;
-#pragma unroll
-        for (int e4 = 0; e4 < 4; ++e4) {
-            const float4 s4 = reinterpret_cast<const float4*>(ss + 16 * q)[e4], i4 = reinterpret_cast<const float4*>(si + 16 * q)[e4],
-                         f4 = reinterpret_cast<const float4*>(szf + 16 * q)[e4];
-            const float sv[4] = {s4.x, s4.y, s4.z, s4.w}, iv[4] = {i4.x, i4.y, i4.z, i4.w}, fv[4] = {f4.x, f4.y, f4.z, f4.w};
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int e = 4 * e4 + k;
-                // Eq. 9 in the float domain (see xsv_quant_code for why x * (1/s) may stand in for x / s): round by
-                // adding 1.5 * 2^23, add the zero-point (exact: both are integers below 2^22), clamp, and read the code
-                // off the mantissa.  Near a rounding boundary, for huge quotients or zero-points: the general routine.
-                const float y = __fmul_rn(x[e], iv[k]);
-                const float t = __fadd_rn(y, 12582912.f);
-                const float r = __fadd_rn(t, -12582912.f);
-                uint32_t code;
-                if (fabsf(y - r) > fmaf(fabsf(y), -9.5367431640625e-7f, 0.5f) || fv[k] != fv[k]) {
-                    code = (uint32_t)xsv_quant_code(x[e], sv[k], iv[k], sz[16 * q + e], NMAX);
+#pragma unroll 1
+            for (; i < 16; ++i) {
+                const int tk = tq + 4 * i;
+                const int sp = s_sp[tk];
+                if (sp == -2) break;
+                float x[8];
+                if (sp >= 0) {
+                    const size_t m = ((size_t)h * src.capg + (sp >> 6)) * 64 + 8 * w;
+                    rq_fetch_slow<BITS>(src.kscale + m, src.kzero + m, chunk_of(i), x);
                 } else {
-                    const float c = fminf(fmaxf(__fadd_rn(r, fv[k]), 0.f), (float)NMAX);
-                    code = __float_as_uint(__fadd_rn(c, 12582912.f)) & 0xFFu;
+                    rq_fetch_fresh<T>(Kf + ((size_t)h * F + (p0 + tk - n_old_new)) * XSV_D + 8 * w, x);
                 }
-                w[e / CPW] |= code << ((e % CPW) * BITS);
+                one(i, x);
             }
+        };
+
+        float mn[8], mx[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { mn[e] = INFINITY; mx[e] = -INFINITY; }
+        walk(
+            [&](int, const float (&x)[8]) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) { mn[e] = fminf(mn[e], x[e]); mx[e] = fmaxf(mx[e], x[e]); }
+            },
+            [&](int, const float (&x0)[8], const float (&x1)[8]) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) { mn[e] = rq_min3(mn[e], x0[e], x1[e]); mx[e] = rq_max3(mx[e], x0[e], x1[e]); }
+            });
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            mn[e] = fminf(mn[e], __shfl_xor_sync(FULL, mn[e], 8));
+            mx[e] = fmaxf(mx[e], __shfl_xor_sync(FULL, mx[e], 8));
+            mn[e] = fminf(mn[e], __shfl_xor_sync(FULL, mn[e], 16));
+            mx[e] = fmaxf(mx[e], __shfl_xor_sync(FULL, mx[e], 16));
         }
-        uint8_t* rowp = dst.kcodes + ((size_t)h * dst.cap + p0 + m) * ROWB + q * (ROWB / 4);
-        if (WPQ == 1) *reinterpret_cast<uint32_t*>(rowp) = w[0];
-        else if (WPQ == 2) *reinterpret_cast<uint2*>(rowp) = make_uint2(w[0], w[WPQ - 1]);
-        else *reinterpret_cast<uint4*>(rowp) = make_uint4(w[0], w[1 % WPQ], w[2 % WPQ], w[3 % WPQ]);
+        // Eq. 10: this lane derives the parameters of channels 8w + 2tq and 8w + 2tq + 1
+        float s2[2];
+        int z2[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const float a = tq == 0 ? mn[k] : tq == 1 ? mn[2 + k] : tq == 2 ? mn[4 + k] : mn[6 + k];
+            const float b = tq == 0 ? mx[k] : tq == 1 ? mx[2 + k] : tq == 2 ? mx[4 + k] : mx[6 + k];
+            xsv_quant_params(a, b, NMAX, s2[k], z2[k], status);
+            const int c = 8 * w + 2 * tq + k;
+            n_s[c] = s2[k];
+            n_i[c] = __frcp_rn(s2[k]);
+            n_z[c] = z2[k];
+            n_zf[c] = (z2[k] > -2097152 && z2[k] < 2097152) ? (float)z2[k] : __int_as_float(0x7FC00000);
+        }
+        __syncwarp();
+        float iv[8], fv[8], ns[8];
+        bool slow_lane = false;
+        {
+            const float4 i0 = *reinterpret_cast<const float4*>(n_i + 8 * w), i1 = *reinterpret_cast<const float4*>(n_i + 8 * w + 4);
+            const float4 f0 = *reinterpret_cast<const float4*>(n_zf + 8 * w), f1 = *reinterpret_cast<const float4*>(n_zf + 8 * w + 4);
+            const float4 a0 = *reinterpret_cast<const float4*>(n_s + 8 * w), a1 = *reinterpret_cast<const float4*>(n_s + 8 * w + 4);
+            iv[0] = i0.x; iv[1] = i0.y; iv[2] = i0.z; iv[3] = i0.w; iv[4] = i1.x; iv[5] = i1.y; iv[6] = i1.z; iv[7] = i1.w;
+            fv[0] = f0.x; fv[1] = f0.y; fv[2] = f0.z; fv[3] = f0.w; fv[4] = f1.x; fv[5] = f1.y; fv[6] = f1.z; fv[7] = f1.w;
+            ns[0] = -a0.x; ns[1] = -a0.y; ns[2] = -a0.z; ns[3] = -a0.w; ns[4] = -a1.x; ns[5] = -a1.y; ns[6] = -a1.z; ns[7] = -a1.w;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) slow_lane |= (fv[e] != fv[e]);
+        }
+        uint8_t* const obase = dst.kcodes + ((size_t)h * dst.cap + p0 + tq) * ROWB + w * BITS;
+        auto put = [&](int i, const float (&x)[8]) {
+            // Eq. 9 in the float domain.  Re-quantised values sit on rounding boundaries of the new grid whenever the
+            // old and new scales are in a small rational ratio, so the quotient must be the IEEE one every time: with
+            // 1/s correctly rounded, y0 = x (1/s) followed by two remainder corrections y += (x - y s) (1/s), each one
+            // fused multiply-add pair, is the correctly rounded x / s (the first correction makes y faithful, the
+            // second exact).  Then: round to nearest even by adding and subtracting 1.5 * 2^23, add the zero-point
+            // (exact: both are integers below 2^22), clamp to [0, n] by a saturating multiply with 1/n, and sum
+            // n * u * 2^(bits k) into the sub-word (the sum is within 2^-6 of the integer it stands for, so the
+            // conversion restores it).  A lane whose zero-points are too large for this takes the general routine
+            // (quotients beyond 2^21 imply such a zero-point, since code = quotient + z lies in [0, n]).
+            uint64_t out;
+            if (slow_lane) {
+                out = rq_codes_slow<BITS>(x, n_s + 8 * w, n_i + 8 * w, n_z + 8 * w);
+            } else {
+                float acc[NSUB];
+#pragma unroll
+                for (int j = 0; j < NSUB; ++j) acc[j] = 0.f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    float y = __fmul_rn(x[e], iv[e]);
+                    y = __fmaf_rn(__fmaf_rn(y, ns[e], x[e]), iv[e], y);
+                    y = __fmaf_rn(__fmaf_rn(y, ns[e], x[e]), iv[e], y);
+                    const float r = __fadd_rn(__fadd_rn(y, 12582912.f), -12582912.f);
+                    const float u = rq_mul_sat(__fadd_rn(r, fv[e]), KINV);
+                    acc[e / SUB] = __fmaf_rn(u, (float)(NMAX << (BITS * (e % SUB))), acc[e / SUB]);
+                }
+                out = 0;
+#pragma unroll
+                for (int j = 0; j < NSUB; ++j) out |= (uint64_t)__float2uint_rn(acc[j]) << (16 * j);
+            }
+            uint8_t* rowp = obase + i * (4 * ROWB);
+            if (BITS == 2) *reinterpret_cast<uint16_t*>(rowp) = (uint16_t)out;
+            else if (BITS == 4) *reinterpret_cast<uint32_t*>(rowp) = (uint32_t)out;
+            else *reinterpret_cast<uint2*>(rowp) = make_uint2((uint32_t)out, (uint32_t)(out >> 32));
+        };
+        walk(put, [&](int i, const float (&x0)[8], const float (&x1)[8]) { put(i, x0); put(i + 1, x1); });
+        // the parameters go out last: in place, the group's old parameters may still have been read from memory above
+        *reinterpret_cast<float2*>(dst.kscale + prm + 8 * w + 2 * tq) = make_float2(s2[0], s2[1]);
+        *reinterpret_cast<int2*>(dst.kzero + prm + 8 * w + 2 * tq) = make_int2(z2[0], z2[1]);
+        __syncwarp();   // the staged rows are rewritten by the next item
     }
 }
 
@@ -671,6 +840,17 @@ __global__ void __launch_bounds__(256) quant_v_kernel(LayerView dst, const T* __
 }  // namespace
 
 // ------------------------------ launchers ----------------------------------
+int xsv_sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
+}
+
 cudaError_t xsv_launch_qtilde(const void* Q, int dtype, int H, int F, int n_special, int g, float* qpart,
                               cudaStream_t st) {
     dim3 grid(XSV_QCHUNKS, H);
@@ -736,10 +916,22 @@ cudaError_t xsv_launch_requant_k(const LayerView& src, const LayerView& dst, con
     const int ngroups = (T_new + XSV_G - 1) / XSV_G;
     const int g0 = (fz_dev == nullptr && src.kcodes == dst.kcodes) ? fz_host : 0;   // in place: skip the frozen prefix
     if (ngroups - g0 <= 0) return cudaSuccess;
-    dim3 grid(ngroups - g0, H);
-#define XSV_RQ(TT, B)                                                                                         \
-    requant_k_kernel<TT, B><<<grid, 256, 0, st>>>(src, dst, (const TT*)Kf, F, n_old_new, T_new, T_first, srcmap, \
-                                                  fz_dev, fz_host, g0, status)
+    const int n_items = (ngroups - g0) * H, wpb = RQ_THREADS / 32;
+#define XSV_RQ(TT, B)                                                                                                \
+    {                                                                                                                \
+        const size_t smem = (size_t)wpb * RqCfg<B>::WORDS * 4;                                                       \
+        static int per_sm = 0;   /* resident blocks per multiprocessor: the grid is one wave of them */              \
+        if (per_sm == 0) {                                                                                           \
+            cudaFuncSetAttribute(requant_k_kernel<TT, B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);   \
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, requant_k_kernel<TT, B>, RQ_THREADS, smem) != \
+                    cudaSuccess || per_sm <= 0)                                                                      \
+                per_sm = 2;                                                                                          \
+        }                                                                                                            \
+        const int grid = min((n_items + wpb - 1) / wpb, xsv_sm_count() * per_sm);                                    \
+        requant_k_kernel<TT, B><<<grid, RQ_THREADS, smem, st>>>(src, dst, (const TT*)Kf, H, F, n_old_new, T_new,      \
+                                                                T_first, srcmap, fz_dev, fz_host, g0, n_items,       \
+                                                                status);                                             \
+    }
     if (dtype == 0) {
         switch (src.bits) {
             case 2: XSV_RQ(__half, 2); break;

@@ -4,6 +4,9 @@
 
 // dtype: 0 = fp16, 1 = bf16 (xsv_dtype).
 
+// Multiprocessors of the current device (queried once).
+int xsv_sm_count();
+
 // Eq. 3-4 folded by linearity: per-(head, chunk) partial sums of the pooling-weighted
 // queries; qpart [H * XSV_QCHUNKS][64].
 #define XSV_QCHUNKS 8
