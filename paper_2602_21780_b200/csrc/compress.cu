@@ -17,134 +17,165 @@ __global__ void __launch_bounds__(256) qtilde_partial_kernel(const T* __restrict
     const int h = blockIdx.y, chunk = blockIdx.x;
     const int per = (F + XSV_QCHUNKS - 1) / XSV_QCHUNKS;
     const int i0 = chunk * per, i1 = min(F, i0 + per);
-    const int c4 = threadIdx.x & 15, r = threadIdx.x >> 4;     // 4 channels (one 8-byte load), 16 rows in flight
+    const int c8 = threadIdx.x & 7, r = threadIdx.x >> 3;      // 8 channels (one 16-byte load), 32 rows in flight
     const int n_patch = F - n_special;
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll 4
-    for (int i = i0 + r; i < i1; i += 16) {
+    float a[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) a[e] = 0.f;
+#pragma unroll 6
+    for (int i = i0 + r; i < i1; i += 32) {
         float w = 1.f;
         if (i >= n_special) {
             const int gi = (i - n_special) / g;
             w = 1.f / (float)min(g, n_patch - gi * g);
         }
-        const uint2 v = *reinterpret_cast<const uint2*>(Q + ((size_t)h * F + i) * XSV_D + 4 * c4);
-        T e[4];
-        *reinterpret_cast<uint2*>(e) = v;
-        a0 = fmaf(w, xsv_to_float<T>(e[0]), a0);
-        a1 = fmaf(w, xsv_to_float<T>(e[1]), a1);
-        a2 = fmaf(w, xsv_to_float<T>(e[2]), a2);
-        a3 = fmaf(w, xsv_to_float<T>(e[3]), a3);
+        const uint4 v = *reinterpret_cast<const uint4*>(Q + ((size_t)h * F + i) * XSV_D + 8 * c8);
+        T e8[8];
+        *reinterpret_cast<uint4*>(e8) = v;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) a[e] = fmaf(w, xsv_to_float<T>(e8[e]), a[e]);
     }
-    __shared__ float red[16][64];
-    red[r][4 * c4] = a0;
-    red[r][4 * c4 + 1] = a1;
-    red[r][4 * c4 + 2] = a2;
-    red[r][4 * c4 + 3] = a3;
+    // the four row lanes of a warp, then the eight warps, in a fixed order
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        a[e] += __shfl_xor_sync(0xFFFFFFFFu, a[e], 8);
+        a[e] += __shfl_xor_sync(0xFFFFFFFFu, a[e], 16);
+    }
+    __shared__ float red[8][64];
+    if ((threadIdx.x & 31) < 8) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) red[threadIdx.x >> 5][8 * c8 + e] = a[e];
+    }
     __syncthreads();
     if (threadIdx.x < 64) {
         float s = 0.f;
 #pragma unroll
-        for (int k = 0; k < 16; ++k) s += red[k][threadIdx.x];
+        for (int k = 0; k < 8; ++k) s += red[k][threadIdx.x];
         qpart[((size_t)h * XSV_QCHUNKS + chunk) * 64 + threadIdx.x] = s;
     }
 }
 
-// ---------------------------------------------------------------------------
-// Eq. 5-7: S[j] = (1/H) sum_h q~ . K~[h, T_first + j, :] over the middle segment.
-// One thread per token; the (scale, zero-point) rows of the key groups a block
-// touches are staged in shared memory.
-// ---------------------------------------------------------------------------
-constexpr int SCORE_TPB = 256;             // 64 tokens x 4 slices of the heads
-constexpr int SCORE_TOK = 64;              // tokens per block
-constexpr int SCORE_MAXG = 2;              // key groups a block's 64 tokens can span
-constexpr int SCORE_WS = 66;               // floats per staged weight row
-
-// Sum of the fixed-order partial sums of the pooled queries, scaled: q~[c].
-__device__ __forceinline__ float qtilde_channel(const float* __restrict__ qpart, int n_part, int c, float qnorm) {
-    float s = 0.f;
+// Fixed-order sum of the n_part partial rows, written over the first row: qpart[0..64) = sum_h sum_i w_i Q[h,i,:].
+__global__ void __launch_bounds__(256) qtilde_final_kernel(float* __restrict__ qpart, int n_part) {
+    __shared__ float red[4][64];
+    const int c = threadIdx.x & 63, part = threadIdx.x >> 6, per = (n_part + 3) / 4;
+    float s4 = 0.f;
+    const int k1 = min(n_part, (part + 1) * per);
 #pragma unroll 8
-    for (int k = 0; k < n_part; ++k) s += qpart[(size_t)k * 64 + c];
-    return s * qnorm;
+    for (int k = part * per; k < k1; ++k) s4 += qpart[(size_t)k * 64 + c];
+    red[part][c] = s4;
+    __syncthreads();       // every partial row has been read
+    if (threadIdx.x < 64) qpart[c] = ((red[0][c] + red[1][c]) + red[2][c]) + red[3][c];
 }
 
-// By linearity q~ . K~[h,j,:] = sum_c (q~_c s_c) code_c - sum_c q~_c s_c z_c: the weights q~_c s_c and the
-// bias are prepared once per (head, key group) of the block; a token then costs one multiply-add per code.
+// ---------------------------------------------------------------------------
+// Eq. 5-7: S[j] = (1/H) sum_h q~ . K~[h, T_first + j, :] over the middle segment.
+// By linearity q~ . K~[h,p,:] = sum_c (q~_c s_c) code_c - sum_c q~_c s_c z_c, with
+// (s, z) the parameters of the key group of p: one block per key group, so the
+// weights q~_c s_c and the bias are prepared once per head and a token costs one
+// multiply-add per code.  256 threads = 64 tokens x 4 head slices; a warp reads
+// 32 consecutive packed rows of one head.  A thread first issues the loads of
+// its (up to four) rows, then helps with the weights, so the two round trips to
+// memory overlap.  Codes are widened without the conversion unit:
+// (word & mask_k) | 2^23 read as a float, minus 2^23, is code * 2^(bits k); the
+// weight carries the 2^-(bits k).
+// ---------------------------------------------------------------------------
+constexpr int SCORE_TPB = 256;             // 64 tokens x 4 slices of the heads
+constexpr int SCORE_ROWS = 4;              // rows a thread holds in registers at a time
+
 template <int BITS>
 __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, int T_first, int T_c,
-                                                          const float* __restrict__ qpart, float qnorm,
+                                                          const float* __restrict__ qfinal, float qnorm,
                                                           float* __restrict__ scores) {
     constexpr int ROWB = XSV_D * BITS / 8;
     constexpr int NV = ROWB / 16;              // 16-byte loads per row
-    constexpr int CPW = 32 / BITS;             // codes per 32-bit word
-    extern __shared__ float sm[];
-    float* qt = sm;                             // [64]
-    float* sW = qt + 64;                        // [H][SCORE_MAXG][SCORE_WS] weights q~_c * s_c (rows padded: the four
-                                                // heads read at once by a warp fall into different banks)
-    float* sB = sW + (size_t)H * SCORE_MAXG * SCORE_WS;   // [H][SCORE_MAXG] bias sum_c q~_c s_c z_c
+    constexpr int SUB = (BITS == 8) ? 2 : (BITS == 4 ? 4 : 8);   // codes per 16-bit sub-word
+    constexpr uint32_t NMAX = (1u << BITS) - 1u;
+    extern __shared__ __align__(16) float sm[];
+    float* sW = sm;                             // [H][64] weights q~_c * s_c * 2^-(bits * position of c in its sub-word)
+    float* sB = sW + (size_t)H * 64;            // [H] bias sum_c q~_c s_c z_c
+    float* part = sB + ((H + 3) & ~3);          // [4][64] per-slice sums
 
-    const int j0 = blockIdx.x * SCORE_TOK;
-    const int p0 = T_first + j0;
-    const int g_lo = p0 >> 6;
-    const int p_last = min(T_c - 1, p0 + SCORE_TOK - 1);
-    const int ng = (p_last >> 6) - g_lo + 1;
+    const int g = (T_first >> 6) + blockIdx.x;  // key group of this block
+    const int tok = threadIdx.x & 63, slice = threadIdx.x >> 6, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int p = g * 64 + tok;
+    const bool valid = p >= T_first && p < T_c;
 
-    {   // q~: four threads per channel sum a quarter of the partial sums each, then a fixed-order sum of the four
-        const int c = threadIdx.x & 63, part = threadIdx.x >> 6, np = H * XSV_QCHUNKS, per = (np + 3) / 4;
-        float s4 = 0.f;
-        const int k1 = min(np, (part + 1) * per);
-#pragma unroll 8
-        for (int k = part * per; k < k1; ++k) s4 += qpart[(size_t)k * 64 + c];
-        sW[part * 64 + c] = s4;            // sW (at least 256 floats, see the launcher) is free until the weights are staged
-        __syncthreads();
-        if (threadIdx.x < 64) qt[c] = (((sW[c] + sW[64 + c]) + sW[128 + c]) + sW[192 + c]) * qnorm;
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < H * ng * 64; i += SCORE_TPB) {
-        const int c = i & 63, gg = (i >> 6) % ng, h = (i >> 6) / ng;
-        const size_t m = ((size_t)h * lv.capg + g_lo + gg) * 64 + c;
-        sW[(h * SCORE_MAXG + gg) * SCORE_WS + c] = qt[c] * lv.kscale[m];
-    }
-    __syncthreads();
-    for (int i = threadIdx.x >> 5; i < H * ng; i += SCORE_TPB / 32) {   // one warp per (head, group): the bias
-        const int gg = i % ng, h = i / ng, lane = threadIdx.x & 31;
-        const size_t m = ((size_t)h * lv.capg + g_lo + gg) * 64;
-        float b = sW[(h * SCORE_MAXG + gg) * SCORE_WS + lane] * (float)lv.kzero[m + lane] +
-                  sW[(h * SCORE_MAXG + gg) * SCORE_WS + lane + 32] * (float)lv.kzero[m + lane + 32];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) b += __shfl_xor_sync(0xFFFFFFFFu, b, o);
-        if (lane == 0) sB[h * SCORE_MAXG + gg] = b;
-    }
-    __syncthreads();
-
-    const int tok = threadIdx.x >> 2, slice = threadIdx.x & 3;
-    const int p = p0 + tok;
     float acc = 0.f;
-    if (p < T_c) {
-        const int gg = (p >> 6) - g_lo;
-        for (int h = slice; h < H; h += 4) {
-            const uint4* row = reinterpret_cast<const uint4*>(lv.kcodes + ((size_t)h * lv.cap + p) * ROWB);
-            const float* w = sW + (h * SCORE_MAXG + gg) * SCORE_WS;
-            float a = 0.f;
+    for (int hb = 0; hb < H; hb += 4 * SCORE_ROWS) {
+        uint4 rows[SCORE_ROWS][NV];
 #pragma unroll
-            for (int v = 0; v < NV; ++v) {
-                const uint4 q = row[v];
-                const uint32_t ww[4] = {q.x, q.y, q.z, q.w};
+        for (int r = 0; r < SCORE_ROWS; ++r) {
+            const int h = hb + slice + 4 * r;
+            if (valid && h < H) {
+                const uint4* row = reinterpret_cast<const uint4*>(lv.kcodes + ((size_t)h * lv.cap + p) * ROWB);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
+                for (int v = 0; v < NV; ++v) rows[r][v] = row[v];
+            } else {
 #pragma unroll
-                    for (int e = 0; e < CPW; ++e) {
-                        const int c = (v * 4 + k) * CPW + e;
-                        a = fmaf(w[c], (float)((ww[k] >> (e * BITS)) & ((1u << BITS) - 1u)), a);
+                for (int v = 0; v < NV; ++v) rows[r][v] = make_uint4(0u, 0u, 0u, 0u);
+            }
+        }
+        if (hb == 0) {
+            // weights and bias: one warp per head at a time, lane l takes channels l and l + 32 (same position in
+            // their sub-words)
+            const float q0 = qfinal[lane] * qnorm, q1 = qfinal[lane + 32] * qnorm;
+            const float pos = __int_as_float((127 - BITS * ((lane & 7) % SUB)) << 23);
+            for (int h = warp; h < H; h += SCORE_TPB / 32) {
+                const size_t m = ((size_t)h * lv.capg + g) * 64;
+                const float w0 = q0 * lv.kscale[m + lane], w1 = q1 * lv.kscale[m + lane + 32];
+                float b = w0 * (float)lv.kzero[m + lane] + w1 * (float)lv.kzero[m + lane + 32];
+                sW[h * 64 + lane] = w0 * pos;
+                sW[h * 64 + lane + 32] = w1 * pos;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) b += __shfl_xor_sync(0xFFFFFFFFu, b, o);
+                if (lane == 0) sB[h] = b;
+            }
+            __syncthreads();
+        }
+#pragma unroll
+        for (int r = 0; r < SCORE_ROWS; ++r) {
+            const int h = hb + slice + 4 * r;
+            if (h < H) {
+                const float4* w4 = reinterpret_cast<const float4*>(sW + h * 64);
+                float a = 0.f;
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    const uint32_t ww[4] = {rows[r][v].x, rows[r][v].y, rows[r][v].z, rows[r][v].w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {           // the word's two 16-bit sub-words
+                            const uint32_t sub = ww[k] >> (16 * j);
+#pragma unroll
+                            for (int e4 = 0; e4 < SUB / 4; ++e4) {
+                                const int c = ((v * 4 + k) * 2 + j) * SUB + 4 * e4;   // channel of the first of four codes
+                                const float4 wv = w4[c / 4];
+                                const float wq[4] = {wv.x, wv.y, wv.z, wv.w};
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const uint32_t mk = (sub & (NMAX << (BITS * (4 * e4 + e)))) | 0x4B000000u;
+                                    a = fmaf(wq[e], __uint_as_float(mk) - 8388608.f, a);
+                                }
+                            }
+                            if (SUB == 2) {
+                                // 8-bit codes: two per sub-word, weights read in pairs
+                                const int c = ((v * 4 + k) * 2 + j) * 2;
+                                const float2 wv = reinterpret_cast<const float2*>(sW + h * 64)[c / 2];
+                                a = fmaf(wv.x, __uint_as_float((sub & 0xFFu) | 0x4B000000u) - 8388608.f, a);
+                                a = fmaf(wv.y, __uint_as_float((sub & 0xFF00u) | 0x4B000000u) - 8388608.f, a);
+                            }
+                        }
                     }
                 }
+                acc += a - sB[h];
             }
-            acc += a - sB[h * SCORE_MAXG + gg];
         }
     }
-    // the four slices of a token sit in adjacent lanes: fixed-order sum
-    acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 1);
-    acc += __shfl_xor_sync(0xFFFFFFFFu, acc, 2);
-    if (slice == 0 && p < T_c) scores[j0 + tok] = acc / (float)H;
+    part[slice * 64 + tok] = acc;
+    __syncthreads();
+    if (threadIdx.x < 64 && valid)
+        scores[p - T_first] = (((part[tok] + part[64 + tok]) + part[128 + tok]) + part[192 + tok]) / (float)H;
 }
 
 // bits == 16: keys are raw 16-bit values.
@@ -153,7 +184,7 @@ __global__ void __launch_bounds__(SCORE_TPB) score_raw_kernel(LayerView lv, int 
                                                               const float* __restrict__ qpart, float qnorm,
                                                               float* __restrict__ scores) {
     __shared__ float qt[64];
-    if (threadIdx.x < 64) qt[threadIdx.x] = qtilde_channel(qpart, H * XSV_QCHUNKS, threadIdx.x, qnorm);
+    if (threadIdx.x < 64) qt[threadIdx.x] = qpart[threadIdx.x] * qnorm;
     __syncthreads();
     const int j = blockIdx.x * SCORE_TPB + threadIdx.x;
     const int p = T_first + j;
@@ -268,120 +299,199 @@ __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ 
 }
 
 // ---------------------------------------------------------------------------
-// Eq. 8 again, for n <= 1024 * KPT: every thread keeps KPT consecutive keys in
-// registers, so the scores are read from memory once.  The four digit
-// histograms are built with warp-aggregated shared-memory atomics (scores
-// share their leading digits, which would otherwise serialise), the bins are
-// scanned by one warp, and the ordered compaction works on warp ballots as in
-// select_kernel.  Same total order.
+// Eq. 8 again, for n <= 1024 * KPT: thread t keeps the keys of the KPT
+// consecutive positions [t KPT, (t + 1) KPT) in registers (16-byte loads), so
+// the scores are read from memory once.
+//
+// The k-th largest key is found by bisection on its bits, from the highest bit
+// in which the keys differ downwards.  A step counts the keys >= (prefix | bit)
+// -- one warp reduction, one shared-memory atomic per warp, one barrier -- and
+// the search stops as soon as a candidate splits off exactly k keys, which for
+// scores without ties happens after about log2(n) + a few steps.  Only the keys
+// inside the current interval [prefix, prefix + 2^(b+1)) are still undecided;
+// once they number at most 2048 they are copied to shared memory and the
+// remaining steps look at one or two keys per thread instead of KPT.
+//
+// Ordered compaction: block-wide exclusive scans of the per-thread counts give
+// every thread the output offset of its first kept position; the kept
+// positions are staged in shared memory and copied out coalesced.  Same total
+// order as select_kernel (score descending, position ascending).
 // ---------------------------------------------------------------------------
+constexpr int SEL_ACT = 2048;             // undecided keys that fit the shared-memory stage of the bisection
+
+// Exclusive prefix sum of v over the 1024 threads of the block; *total receives the sum.  ws: 33 ints.
+__device__ __forceinline__ int sel_block_scan(int v, int* ws, int* total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t; }
+    __syncthreads();               // ws may still be read from an earlier scan
+    if (lane == 31) ws[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        const int x = ws[lane];
+        int xi = x;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, xi, o); if (lane >= o) xi += t; }
+        ws[lane] = xi - x;
+        if (lane == 31) ws[32] = xi;
+    }
+    __syncthreads();
+    *total = ws[32];
+    return ws[warp] + incl - v;
+}
+
 template <int KPT>
 __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restrict__ scores, int n, int k, int T_first,
                                                           int T_c, int* __restrict__ srcmap, int* __restrict__ dscal) {
-    __shared__ int hist[256];
-    __shared__ int w_gt[32], w_eq[32], w_off[32], w_eqb[32];
-    __shared__ uint32_t s_prefix;
-    __shared__ int s_remaining;
+    extern __shared__ __align__(16) int sel_sm[];     // [1024 * KPT]: undecided keys, later the kept positions
+    __shared__ int cnt[36];
+    __shared__ uint32_t s_lo, s_hi;
+    __shared__ int s_nact;
+    __shared__ int ws[33];
     __shared__ int s_first_evicted;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // warp w owns the contiguous positions [w * 32 * KPT, (w + 1) * 32 * KPT); lane l holds every 32nd of them
-    // (coalesced loads, and the ordered compaction below needs ballots only)
-    const int j0 = warp * 32 * KPT + lane;
-    uint32_t key[KPT];
+    constexpr uint32_t FULL = 0xFFFFFFFFu;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int j0 = tid * KPT;
+    uint32_t key[KPT];                    // positions past n hold key 0
+    if ((reinterpret_cast<uintptr_t>(scores) & 15) == 0) {
 #pragma unroll
-    for (int i = 0; i < KPT; ++i) key[i] = (j0 + 32 * i < n) ? score_key(scores[j0 + 32 * i]) : 0u;
+        for (int v = 0; v < KPT / 4; ++v) {
+            const int j = j0 + 4 * v;
+            if (j + 3 < n) {
+                const float4 f = *reinterpret_cast<const float4*>(scores + j);
+                key[4 * v] = score_key(f.x); key[4 * v + 1] = score_key(f.y);
+                key[4 * v + 2] = score_key(f.z); key[4 * v + 3] = score_key(f.w);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) key[4 * v + e] = (j + e < n) ? score_key(scores[j + e]) : 0u;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < KPT; ++i) key[i] = (j0 + i < n) ? score_key(scores[j0 + i]) : 0u;
+    }
 
     uint32_t thr = 0xFFFFFFFFu;
     int need_eq = 0;
-    if (k > 0) {
-        uint32_t prefix = 0, mask = 0;
-        int remaining = k;
-        for (int pass = 3; pass >= 0; --pass) {
-            const int shift = pass * 8;
-            if (tid < 256) hist[tid] = 0;
-            __syncthreads();
+    if (k >= n) {
+        thr = 0u;                  // every key is kept
+        need_eq = n;
+    } else if (k > 0) {
+        if (tid < 36) cnt[tid] = 0;
+        if (tid == 0) { s_lo = 0xFFFFFFFFu; s_hi = 0u; s_nact = 0; }
+        __syncthreads();
+        uint32_t lo = 0xFFFFFFFFu, hi = 0u;
 #pragma unroll
-            for (int i = 0; i < KPT; ++i) {
-                const bool act = (j0 + 32 * i < n) && (key[i] & mask) == prefix;
-                if (__any_sync(0xFFFFFFFFu, act)) {
-                    const uint32_t digit = act ? ((key[i] >> shift) & 255u) : 256u;
-                    const uint32_t peers = __match_any_sync(0xFFFFFFFFu, digit);
-                    if (act && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+        for (int i = 0; i < KPT; ++i)
+            if (j0 + i < n) { lo = min(lo, key[i]); hi = max(hi, key[i]); }
+        lo = __reduce_min_sync(FULL, lo);
+        hi = __reduce_max_sync(FULL, hi);
+        if (lane == 0) { atomicMin(&s_lo, lo); atomicMax(&s_hi, hi); }
+        __syncthreads();
+        lo = s_lo;
+        hi = s_hi;
+        if (lo == hi) {            // all keys equal: the k lowest positions
+            thr = lo;
+            need_eq = k;
+        } else {
+            int b = 31 - __clz(lo ^ hi);
+            uint32_t v = (b == 31) ? 0u : (lo & ~((2u << b) - 1u));     // the leading bits all keys share
+            // Invariants: ge_v keys are >= v, `above` of them are >= v + 2^(b+1) (the end of the undecided interval),
+            // above < k <= ge_v.
+            int ge_v = n, above = 0, step = 0;
+            bool exact = false;
+            // stage 1: all keys, in registers
+            for (; b >= 0 && ge_v - above > SEL_ACT; --b, ++step) {
+                const uint32_t cand = v | (1u << b);
+                int c = 0;
+#pragma unroll
+                for (int i = 0; i < KPT; ++i) c += (key[i] >= cand) ? 1 : 0;
+                c = __reduce_add_sync(FULL, c);
+                if (lane == 0 && c != 0) atomicAdd(&cnt[step], c);
+                __syncthreads();
+                c = cnt[step];
+                if (c >= k) {
+                    v = cand;
+                    ge_v = c;
+                    if (c == k) { exact = true; break; }
+                } else {
+                    above = c;
                 }
             }
-            __syncthreads();
-            if (tid < 32) {
-                // bins from the top: find the digit at which the cumulated count reaches `remaining`
-                int c[8], sum = 0;
+            if (!exact && b >= 0) {
+                // stage 2: the undecided keys (v <= key < v + 2^(b+1)), one or two per thread, from shared memory
+                const uint32_t width = (b == 31) ? 0xFFFFFFFFu : ((2u << b) - 1u);      // interval length - 1
+                int mine = 0;
 #pragma unroll
-                for (int q = 0; q < 8; ++q) { c[q] = hist[255 - (tid * 8 + q)]; sum += c[q]; }
-                int incl = sum;
+                for (int i = 0; i < KPT; ++i) mine += (j0 + i < n && key[i] - v <= width && key[i] >= v) ? 1 : 0;
+                int incl = mine;
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o); if (lane >= o) incl += t; }
-                int cum = incl - sum;          // count in the bins above this lane's
-                if (cum < remaining && incl >= remaining) {
-                    int digit = 0;
+                for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(FULL, incl, o); if (lane >= o) incl += t; }
+                int base = 0;
+                if (lane == 31 && incl != 0) base = atomicAdd(&s_nact, incl);
+                base = __shfl_sync(FULL, base, 31) + incl - mine;
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        if (cum + c[q] >= remaining) { digit = 255 - (tid * 8 + q); break; }
-                        cum += c[q];
+                for (int i = 0; i < KPT; ++i)
+                    if (j0 + i < n && key[i] - v <= width && key[i] >= v) sel_sm[base++] = (int)key[i];
+                __syncthreads();
+                const int n_act = s_nact;          // == ge_v - above
+                const uint32_t a0 = tid < n_act ? (uint32_t)sel_sm[tid] : 0u;
+                const uint32_t a1 = tid + 1024 < n_act ? (uint32_t)sel_sm[tid + 1024] : 0u;
+                const int above0 = above;          // keys beyond the staged interval
+                for (; b >= 0; --b, ++step) {
+                    const uint32_t cand = v | (1u << b);
+                    int c = ((a0 >= cand) ? 1 : 0) + ((a1 >= cand) ? 1 : 0);
+                    c = __reduce_add_sync(FULL, c);
+                    if (lane == 0 && c != 0) atomicAdd(&cnt[step], c);
+                    __syncthreads();
+                    c = cnt[step] + above0;       // all keys >= cand
+                    if (c >= k) {
+                        v = cand;
+                        if (c == k) { exact = true; break; }
+                    } else {
+                        above = c;
                     }
-                    s_remaining = remaining - cum;
-                    s_prefix = prefix | ((uint32_t)digit << shift);
                 }
             }
-            __syncthreads();
-            prefix = s_prefix;
-            remaining = s_remaining;
-            mask |= 255u << shift;
+            if (exact) {           // exactly k keys are >= v
+                thr = v - 1u;
+                need_eq = 0;
+            } else {               // v is the k-th largest key; `above` keys are larger
+                thr = v;
+                need_eq = k - above;
+            }
         }
-        thr = prefix;
-        need_eq = remaining;       // how many of the keys equal to thr are taken (lowest positions)
     }
     if (tid == 0) s_first_evicted = n;
-    int cgt = 0, ceq = 0;
+
+    // ordered compaction
+    int n_gt = 0, n_eq = 0;
 #pragma unroll
     for (int i = 0; i < KPT; ++i) {
-        const bool valid = j0 + 32 * i < n;
-        cgt += __popc(__ballot_sync(0xFFFFFFFFu, valid && key[i] > thr));
-        ceq += __popc(__ballot_sync(0xFFFFFFFFu, valid && k > 0 && key[i] == thr));
+        const bool valid = j0 + i < n;
+        n_gt += (valid && key[i] > thr) ? 1 : 0;
+        n_eq += (valid && k > 0 && key[i] == thr) ? 1 : 0;
     }
-    if (lane == 0) { w_gt[warp] = cgt; w_eq[warp] = ceq; }
-    __syncthreads();
-    if (warp == 0) {
-        // exclusive scans over the 32 warps, in warp order
-        const int eq = w_eq[lane], gt = w_gt[lane];
-        int eq_incl = eq;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, eq_incl, o); if (lane >= o) eq_incl += t; }
-        const int eq_before = eq_incl - eq;
-        const int kept = gt + max(0, min(eq, need_eq - eq_before));
-        int k_incl = kept;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xFFFFFFFFu, k_incl, o); if (lane >= o) k_incl += t; }
-        w_off[lane] = k_incl - kept;
-        w_eqb[lane] = eq_before;
-    }
-    __syncthreads();
-    int off = w_off[warp], eqb = w_eqb[warp], first_ev = n;
-    const uint32_t lt = (1u << lane) - 1u;
+    int total = 0, eq_before = 0;
+    if (need_eq > 0) eq_before = sel_block_scan(n_eq, ws, &total);       // need_eq is the same in every thread
+    const int take_eq = max(0, min(n_eq, need_eq - eq_before));
+    int off = sel_block_scan(n_gt + take_eq, ws, &total);
+    int first_ev = n, eq_rank = eq_before;
 #pragma unroll
     for (int i = 0; i < KPT; ++i) {
-        const int j = j0 + 32 * i;
+        const int j = j0 + i;
         const bool valid = j < n;
-        const bool gt = valid && key[i] > thr, eq = valid && k > 0 && key[i] == thr;
-        const uint32_t beq = __ballot_sync(0xFFFFFFFFu, eq);
-        const bool keep = gt || (eq && eqb + __popc(beq & lt) < need_eq);
-        const uint32_t bk = __ballot_sync(0xFFFFFFFFu, keep);
-        if (keep) srcmap[off + __popc(bk & lt)] = T_first + j;
+        const bool eq = valid && k > 0 && key[i] == thr;
+        const bool keep = (valid && key[i] > thr) || (eq && eq_rank < need_eq);
+        eq_rank += eq ? 1 : 0;
+        if (keep) sel_sm[off++] = T_first + j;
         if (valid && !keep) first_ev = min(first_ev, j);
-        off += __popc(bk);
-        eqb += __popc(beq);
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) first_ev = min(first_ev, __shfl_xor_sync(0xFFFFFFFFu, first_ev, o));
+    first_ev = __reduce_min_sync(FULL, first_ev);
     if (lane == 0 && first_ev < n) atomicMin(&s_first_evicted, first_ev);
     __syncthreads();
+    for (int i = tid; i < total; i += 1024) srcmap[i] = sel_sm[i];
     if (tid == 0) dscal[0] = min(T_first + s_first_evicted, T_c) >> 6;
 }
 
@@ -479,12 +589,95 @@ __device__ __forceinline__ uint64_t rq_codes_slow(const float (&x)[8], const flo
     return out;
 }
 
+// Values of kept tokens move verbatim (codes row, scale, zero-point, origin): one warp per (64 new positions, head).
+template <int BITS>
+__device__ __forceinline__ void rq_gather_v_item(const LayerView& src, const LayerView& dst, int H, int n_old_new,
+                                                 int T_first, const int* __restrict__ srcmap, int item, int lane) {
+    constexpr int ROWB = XSV_D * BITS / 8, PPR = ROWB / 16;
+    const int h = item % H, p0 = (item / H) * 64;
+    int spv[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const int p = p0 + lane + 32 * k;
+        spv[k] = p < n_old_new ? ((srcmap != nullptr && p >= T_first) ? srcmap[p - T_first] : p) : -1;
+    }
+    uint4 v[2 * PPR];
+#pragma unroll
+    for (int j = 0; j < 2 * PPR; ++j) {
+        const int idx = lane + 32 * j, row = idx / PPR, piece = idx % PPR;
+        const int sp = __shfl_sync(0xFFFFFFFFu, spv[row >> 5], row & 31);
+        v[j] = make_uint4(0u, 0u, 0u, 0u);
+        if (sp >= 0) v[j] = *reinterpret_cast<const uint4*>(src.vcodes + ((size_t)h * src.cap + sp) * ROWB + 16 * piece);
+    }
+#pragma unroll
+    for (int j = 0; j < 2 * PPR; ++j) {
+        const int idx = lane + 32 * j, row = idx / PPR, piece = idx % PPR;
+        if (p0 + row < n_old_new)
+            *reinterpret_cast<uint4*>(dst.vcodes + ((size_t)h * dst.cap + p0 + row) * ROWB + 16 * piece) = v[j];
+    }
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const int p = p0 + lane + 32 * k;
+        if (spv[k] >= 0) {
+            dst.vscale[(size_t)h * dst.cap + p] = src.vscale[(size_t)h * src.cap + spv[k]];
+            dst.vzero[(size_t)h * dst.cap + p] = src.vzero[(size_t)h * src.cap + spv[k]];
+            if (h == 0) dst.origin[p] = src.origin[spv[k]];
+        }
+    }
+}
+
+// Eq. 9-11 for the frame's values: one warp per (16 tokens, head); a row of 64 channels at a time, two channels per
+// lane, shuffle reductions for min / max.
+constexpr int RQ_VROWS = 16;
+template <typename T, int BITS>
+__device__ __forceinline__ void rq_quant_v_item(const LayerView& dst, const T* __restrict__ Vf, int H, int F,
+                                                int n_old_new, long long origin0, int* __restrict__ status, int item,
+                                                int lane) {
+    constexpr int ROWB = XSV_D * BITS / 8;
+    constexpr int NMAX = (1 << BITS) - 1;
+    constexpr int LPW = 16 / BITS;            // lanes that share one 32-bit word
+    const int h = item % H, f0 = (item / H) * RQ_VROWS;
+#pragma unroll 4
+    for (int i = 0; i < RQ_VROWS; ++i) {
+        const int f = f0 + i;
+        if (f >= F) break;
+        const uint32_t raw = *reinterpret_cast<const uint32_t*>(Vf + ((size_t)h * F + f) * XSV_D + 2 * lane);
+        T lo, hi;
+        *reinterpret_cast<uint16_t*>(&lo) = (uint16_t)(raw & 0xFFFFu);
+        *reinterpret_cast<uint16_t*>(&hi) = (uint16_t)(raw >> 16);
+        const float x0 = xsv_to_float<T>(lo), x1 = xsv_to_float<T>(hi);
+        float mn = fminf(x0, x1), mx = fmaxf(x0, x1);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
+            mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+        }
+        float s;
+        int z;
+        xsv_quant_params(mn, mx, NMAX, s, z, status);
+        const float inv_s = __frcp_rn(s);
+        const uint32_t c0 = (uint32_t)xsv_quant_code(x0, s, inv_s, z, NMAX), c1 = (uint32_t)xsv_quant_code(x1, s, inv_s, z, NMAX);
+        uint32_t w = (c0 | (c1 << BITS)) << (2 * BITS * (lane % LPW));
+#pragma unroll
+        for (int o = 1; o < LPW; o <<= 1) w |= __shfl_xor_sync(0xFFFFFFFFu, w, o);
+        const int p = n_old_new + f;
+        if (lane % LPW == 0)
+            *reinterpret_cast<uint32_t*>(dst.vcodes + ((size_t)h * dst.cap + p) * ROWB + 4 * (lane / LPW)) = w;
+        if (lane == 0) {
+            dst.vscale[(size_t)h * dst.cap + p] = s;
+            dst.vzero[(size_t)h * dst.cap + p] = z;
+            if (h == 0) dst.origin[p] = origin0 + f;
+        }
+    }
+}
+
 template <typename T, int BITS>
 __global__ void __launch_bounds__(RQ_THREADS, 3) requant_k_kernel(LayerView src, LayerView dst, const T* __restrict__ Kf,
-                                                               int H, int F, int n_old_new, int T_new, int T_first,
-                                                               const int* __restrict__ srcmap,
+                                                               const T* __restrict__ Vf, int H, int F, int n_old_new,
+                                                               int T_new, int T_first, const int* __restrict__ srcmap,
                                                                const int* __restrict__ fz_dev, int fz_host,
-                                                               int g_base, int n_items, int* __restrict__ status) {
+                                                               int g_base, int n_items, int n_vg, int n_vq,
+                                                               long long origin0, int* __restrict__ status) {
     using C = RqCfg<BITS>;
     constexpr int ROWB = C::ROWB, SUB = C::SUB, NSUB = C::NSUB;
     constexpr int NMAX = (1 << BITS) - 1;
@@ -507,9 +700,21 @@ __global__ void __launch_bounds__(RQ_THREADS, 3) requant_k_kernel(LayerView src,
     const int pos_shift = BITS * ((lane & 7) % SUB);
     const float pos_scale = __int_as_float((127 - pos_shift) << 23);
 
-    // item of round r: r * (warps of the grid) + warp * (blocks) + block, so that a last, partial round is spread over
-    // all blocks (and so over all multiprocessors)
-    for (int it = warp * gridDim.x + blockIdx.x; it < n_items; it += gridDim.x * wpb) {
+    // Warp slot: warp * (blocks) + block, so that a partial round of items is spread over all blocks (and so over all
+    // multiprocessors).  The heavy key-group items are dealt out first, round by round; the short value items then go
+    // to the slots that received one key item fewer (to all slots if the key items came out even).
+    const int slot = warp * gridDim.x + blockIdx.x, n_slots = gridDim.x * wpb;
+    {
+        const int extra = n_items % n_slots;                  // slots [0, extra) hold one more key item
+        const int first = (extra == 0) ? 0 : extra;
+        if (slot >= first) {
+            for (int j = slot - first; j < n_vg + n_vq; j += n_slots - first) {
+                if (j < n_vg) rq_gather_v_item<BITS>(src, dst, H, n_old_new, T_first, srcmap, j, lane);
+                else rq_quant_v_item<T, BITS>(dst, Vf, H, F, n_old_new, origin0, status, j - n_vg, lane);
+            }
+        }
+    }
+    for (int it = slot; it < n_items; it += n_slots) {
         const int gi = g_base + it / H, h = it % H;
         const int p0 = gi * XSV_G;
         const int cnt = min(XSV_G, T_new - p0);
@@ -797,46 +1002,6 @@ __global__ void __launch_bounds__(256) append_raw_kernel(LayerView dst, const ui
     if (h == 0 && piece == 0) dst.origin[n_old_new + f] = origin0 + f;
 }
 
-// ---------------------------------------------------------------------------
-// Eq. 9-11 for the fresh frame's values: one warp per (head, token) row of 64
-// channels, two channels per lane, shuffle reductions for min / max.
-// ---------------------------------------------------------------------------
-template <typename T, int BITS>
-__global__ void __launch_bounds__(256) quant_v_kernel(LayerView dst, const T* __restrict__ Vf, int H, int F,
-                                                      int n_old_new, long long origin0, int* __restrict__ status) {
-    constexpr int ROWB = XSV_D * BITS / 8;
-    constexpr int NMAX = (1 << BITS) - 1;
-    constexpr int LPW = 16 / BITS;            // lanes that share one 32-bit word
-    const int lane = threadIdx.x & 31;
-    const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (row >= (long long)H * F) return;
-    const int f = (int)(row % F), h = (int)(row / F);
-    const T* src = Vf + ((size_t)h * F + f) * XSV_D + 2 * lane;
-    const float x0 = xsv_to_float<T>(src[0]), x1 = xsv_to_float<T>(src[1]);
-    float mn = fminf(x0, x1), mx = fmaxf(x0, x1);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
-        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-    }
-    float s;
-    int z;
-    xsv_quant_params(mn, mx, NMAX, s, z, status);
-    const float inv_s = __frcp_rn(s);
-    const uint32_t c0 = (uint32_t)xsv_quant_code(x0, s, inv_s, z, NMAX), c1 = (uint32_t)xsv_quant_code(x1, s, inv_s, z, NMAX);
-    uint32_t w = (c0 | (c1 << BITS)) << (2 * BITS * (lane % LPW));
-#pragma unroll
-    for (int o = 1; o < LPW; o <<= 1) w |= __shfl_xor_sync(0xFFFFFFFFu, w, o);
-    const int p = n_old_new + f;
-    if (lane % LPW == 0)
-        *reinterpret_cast<uint32_t*>(dst.vcodes + ((size_t)h * dst.cap + p) * ROWB + 4 * (lane / LPW)) = w;
-    if (lane == 0) {
-        dst.vscale[(size_t)h * dst.cap + p] = s;
-        dst.vzero[(size_t)h * dst.cap + p] = z;
-        if (h == 0) dst.origin[p] = origin0 + f;
-    }
-}
-
 }  // namespace
 
 // ------------------------------ launchers ----------------------------------
@@ -856,7 +1021,8 @@ cudaError_t xsv_launch_qtilde(const void* Q, int dtype, int H, int F, int n_spec
     dim3 grid(XSV_QCHUNKS, H);
     if (dtype == 0) qtilde_partial_kernel<__half><<<grid, 256, 0, st>>>((const __half*)Q, F, n_special, g, qpart);
     else qtilde_partial_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)Q, F, n_special, g, qpart);
-    xsv_count_launch();
+    qtilde_final_kernel<<<1, 256, 0, st>>>(qpart, H * XSV_QCHUNKS);
+    xsv_count_launch(2);
     return cudaGetLastError();
 }
 
@@ -864,8 +1030,8 @@ cudaError_t xsv_launch_score(const LayerView& lv, int H, int T_first, int T_c, c
                              float* scores, cudaStream_t st) {
     const int n = T_c - T_first;
     if (n <= 0) return cudaSuccess;
-    const int grid = (n + SCORE_TOK - 1) / SCORE_TOK;
-    const size_t smem = (64 + ((size_t)H * SCORE_MAXG * (SCORE_WS + 1) > 256 ? (size_t)H * SCORE_MAXG * (SCORE_WS + 1) : 256)) * sizeof(float);
+    const int grid = ((T_c - 1) >> 6) - (T_first >> 6) + 1;      // key groups that hold a middle token
+    const size_t smem = ((size_t)H * 64 + ((H + 3) & ~3) + 4 * 64) * sizeof(float);
     cudaError_t e = cudaSuccess;
 #define XSV_SCORE(B)                                                                                       \
     {                                                                                                      \
@@ -901,22 +1067,38 @@ cudaError_t xsv_launch_score_raw(const LayerView& lv, int dtype, int H, int T_fi
 
 cudaError_t xsv_launch_select(const float* scores, int n, int k, int T_first, int T_c, int* srcmap, int* dscal,
                               cudaStream_t st) {
-    if (n <= 1024 * 8) select_reg_kernel<8><<<1, 1024, 0, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);
-    else if (n <= 1024 * 16) select_reg_kernel<16><<<1, 1024, 0, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);
-    else if (n <= 1024 * 24) select_reg_kernel<24><<<1, 1024, 0, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);
-    else if (n <= 1024 * 32) select_reg_kernel<32><<<1, 1024, 0, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);
+#define XSV_SEL(KPT)                                                                                             \
+    {                                                                                                            \
+        static bool attr_set = false;                                                                            \
+        if (!attr_set) {                                                                                         \
+            cudaError_t e = cudaFuncSetAttribute(select_reg_kernel<KPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                                 1024 * KPT * 4);                                                \
+            if (e != cudaSuccess) return e;                                                                      \
+            attr_set = true;                                                                                     \
+        }                                                                                                        \
+        select_reg_kernel<KPT><<<1, 1024, 1024 * KPT * 4, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);      \
+    }
+    if (n <= 1024 * 8) XSV_SEL(8)
+    else if (n <= 1024 * 16) XSV_SEL(16)
+    else if (n <= 1024 * 24) XSV_SEL(24)
+    else if (n <= 1024 * 32) XSV_SEL(32)
     else select_kernel<<<1, 1024, 0, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);
+#undef XSV_SEL
     xsv_count_launch();
     return cudaGetLastError();
 }
 
-cudaError_t xsv_launch_requant_k(const LayerView& src, const LayerView& dst, const void* Kf, int dtype, int H,
-                                 int F, int n_old_new, int T_new, int T_first, const int* srcmap,
-                                 const int* fz_dev, int fz_host, int* status, cudaStream_t st) {
+cudaError_t xsv_launch_compress(const LayerView& src, const LayerView& dst, const void* Kf, const void* Vf, int dtype,
+                                int H, int F, int n_old_new, int T_new, int T_first, const int* srcmap,
+                                const int* fz_dev, int fz_host, long long origin0, int* status, cudaStream_t st) {
     const int ngroups = (T_new + XSV_G - 1) / XSV_G;
-    const int g0 = (fz_dev == nullptr && src.kcodes == dst.kcodes) ? fz_host : 0;   // in place: skip the frozen prefix
-    if (ngroups - g0 <= 0) return cudaSuccess;
-    const int n_items = (ngroups - g0) * H, wpb = RQ_THREADS / 32;
+    const bool same = src.kcodes == dst.kcodes;
+    const int g0 = (fz_dev == nullptr && same) ? fz_host : 0;   // in place: skip the frozen prefix
+    const int n_items = max(0, ngroups - g0) * H, wpb = RQ_THREADS / 32;
+    const int n_vg = same ? 0 : ((n_old_new + 63) / 64) * H;     // value rows that move
+    const int n_vq = ((F + RQ_VROWS - 1) / RQ_VROWS) * H;        // value rows of the frame
+    const int n_all = n_items + n_vg + n_vq;
+    if (n_all <= 0) return cudaSuccess;
 #define XSV_RQ(TT, B)                                                                                                \
     {                                                                                                                \
         const size_t smem = (size_t)wpb * RqCfg<B>::WORDS * 4;                                                       \
@@ -927,10 +1109,10 @@ cudaError_t xsv_launch_requant_k(const LayerView& src, const LayerView& dst, con
                     cudaSuccess || per_sm <= 0)                                                                      \
                 per_sm = 2;                                                                                          \
         }                                                                                                            \
-        const int grid = min((n_items + wpb - 1) / wpb, xsv_sm_count() * per_sm);                                    \
-        requant_k_kernel<TT, B><<<grid, RQ_THREADS, smem, st>>>(src, dst, (const TT*)Kf, H, F, n_old_new, T_new,      \
-                                                                T_first, srcmap, fz_dev, fz_host, g0, n_items,       \
-                                                                status);                                             \
+        const int grid = min((n_all + wpb - 1) / wpb, xsv_sm_count() * per_sm);                                      \
+        requant_k_kernel<TT, B><<<grid, RQ_THREADS, smem, st>>>(src, dst, (const TT*)Kf, (const TT*)Vf, H, F,        \
+                                                                n_old_new, T_new, T_first, srcmap, fz_dev, fz_host,  \
+                                                                g0, n_items, n_vg, n_vq, origin0, status);           \
     }
     if (dtype == 0) {
         switch (src.bits) {
@@ -948,46 +1130,6 @@ cudaError_t xsv_launch_requant_k(const LayerView& src, const LayerView& dst, con
         }
     }
 #undef XSV_RQ
-    xsv_count_launch();
-    return cudaGetLastError();
-}
-
-cudaError_t xsv_launch_gather_v(const LayerView& src, const LayerView& dst, int H, int n_old_new, int T_first,
-                                const int* srcmap, cudaStream_t st) {
-    if (n_old_new <= 0) return cudaSuccess;
-    const long long total = (long long)H * n_old_new * (src.rowb / 16);
-    const int grid = (int)((total + 255) / 256);
-    switch (src.rowb) {
-        case 16: gather_v_kernel<16><<<grid, 256, 0, st>>>(src, dst, H, n_old_new, T_first, srcmap); break;
-        case 32: gather_v_kernel<32><<<grid, 256, 0, st>>>(src, dst, H, n_old_new, T_first, srcmap); break;
-        case 64: gather_v_kernel<64><<<grid, 256, 0, st>>>(src, dst, H, n_old_new, T_first, srcmap); break;
-        case 128: gather_v_kernel<128><<<grid, 256, 0, st>>>(src, dst, H, n_old_new, T_first, srcmap); break;
-        default: return cudaErrorInvalidValue;
-    }
-    xsv_count_launch();
-    return cudaGetLastError();
-}
-
-cudaError_t xsv_launch_quant_v(const LayerView& dst, const void* Vf, int dtype, int H, int F, int n_old_new,
-                               long long origin0, int* status, cudaStream_t st) {
-    const int grid = (int)(((long long)H * F + 7) / 8);
-#define XSV_QV(TT, B) quant_v_kernel<TT, B><<<grid, 256, 0, st>>>(dst, (const TT*)Vf, H, F, n_old_new, origin0, status)
-    if (dtype == 0) {
-        switch (dst.bits) {
-            case 2: XSV_QV(__half, 2); break;
-            case 4: XSV_QV(__half, 4); break;
-            case 8: XSV_QV(__half, 8); break;
-            default: return cudaErrorInvalidValue;
-        }
-    } else {
-        switch (dst.bits) {
-            case 2: XSV_QV(__nv_bfloat16, 2); break;
-            case 4: XSV_QV(__nv_bfloat16, 4); break;
-            case 8: XSV_QV(__nv_bfloat16, 8); break;
-            default: return cudaErrorInvalidValue;
-        }
-    }
-#undef XSV_QV
     xsv_count_launch();
     return cudaGetLastError();
 }

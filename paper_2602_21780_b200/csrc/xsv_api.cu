@@ -334,11 +334,8 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
             if (c->bits == 16) {
                 e = xsv_launch_raw_update(lv, dv, K, V, H, F, n_old_new, T_first, c->srcmap, origin0, st);
             } else {
-                e = xsv_launch_gather_v(lv, dv, H, n_old_new, T_first, c->srcmap, st);
-                if (e == cudaSuccess) e = xsv_launch_quant_v(dv, V, (int)dtype, H, F, n_old_new, origin0, c->status, st);
-                if (e == cudaSuccess)
-                    e = xsv_launch_requant_k(lv, dv, K, (int)dtype, H, F, n_old_new, T_new, T_first, c->srcmap, c->dscal, 0,
-                                             c->status, st);
+                e = xsv_launch_compress(lv, dv, K, V, (int)dtype, H, F, n_old_new, T_new, T_first, c->srcmap, c->dscal, 0,
+                                        origin0, c->status, st);
             }
             if (e != cudaSuccess) return cuda_fail(e);
         }
@@ -353,10 +350,8 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
         if (c->bits == 16) {
             e = xsv_launch_raw_update(lv, lv, K, V, H, F, (int)T_c, F, nullptr, origin0, st);
         } else {
-            e = xsv_launch_quant_v(lv, V, (int)dtype, H, F, (int)T_c, origin0, c->status, st);
-            if (e == cudaSuccess)
-                e = xsv_launch_requant_k(lv, lv, K, (int)dtype, H, F, (int)T_c, (int)T, F, nullptr, nullptr,
-                                         (int)(T_c / XSV_G), c->status, st);
+            e = xsv_launch_compress(lv, lv, K, V, (int)dtype, H, F, (int)T_c, (int)T, F, nullptr, nullptr,
+                                    (int)(T_c / XSV_G), origin0, c->status, st);
         }
         if (e != cudaSuccess) return cuda_fail(e);
         c->len[layer] = T;

@@ -27,24 +27,18 @@ cudaError_t xsv_launch_score_raw(const LayerView& lv, int dtype, int H, int T_fi
 cudaError_t xsv_launch_select(const float* scores, int n, int k, int T_first, int T_c, int* srcmap,
                               int* dscal, cudaStream_t st);
 
-// Eq. 9-11 for keys: rebuild the key groups of the new cache order.
-//   new position p < n_old_new comes from cache position (p < T_first ? p : srcmap[p - T_first])
-//   (srcmap == nullptr: identity); p >= n_old_new is fresh token p - n_old_new.
-//   Groups below the frozen count (fz_dev ? *fz_dev : fz_host) are copied verbatim
-//   (skipped when src and dst are the same buffer).
-cudaError_t xsv_launch_requant_k(const LayerView& src, const LayerView& dst, const void* Kf, int dtype,
-                                 int H, int F, int n_old_new, int T_new, int T_first, const int* srcmap,
-                                 const int* fz_dev, int fz_host, int* status, cudaStream_t st);
-
-// Values: gather kept rows (codes, scale, zero-point, origin) into dst for new
-// positions [0, n_old_new); only needed when dst != src.
-cudaError_t xsv_launch_gather_v(const LayerView& src, const LayerView& dst, int H, int n_old_new,
-                                int T_first, const int* srcmap, cudaStream_t st);
-
-// Values: Eq. 9-11 per token for the fresh frame, written at new positions
-// [n_old_new, n_old_new + F); also writes their origin ids.
-cudaError_t xsv_launch_quant_v(const LayerView& dst, const void* Vf, int dtype, int H, int F,
-                               int n_old_new, long long origin0, int* status, cudaStream_t st);
+// Eq. 9-11 for the new cache order, one launch (bits < 16).
+// Keys: the key groups are rebuilt.  New position p < n_old_new comes from cache position
+//   (p < T_first ? p : srcmap[p - T_first]) (srcmap == nullptr: identity); p >= n_old_new is token
+//   p - n_old_new of the frame.  Groups below the frozen count (fz_dev ? *fz_dev : fz_host) are copied
+//   verbatim (skipped when src and dst are the same buffer).
+// Values: kept rows move verbatim (codes, scale, zero-point, origin) to new positions [0, n_old_new) when
+//   dst != src; the frame's rows are quantised per token into [n_old_new, n_old_new + F), with their origins
+//   origin0 + token index.
+cudaError_t xsv_launch_compress(const LayerView& src, const LayerView& dst, const void* Kf, const void* Vf,
+                                int dtype, int H, int F, int n_old_new, int T_new, int T_first,
+                                const int* srcmap, const int* fz_dev, int fz_host, long long origin0,
+                                int* status, cudaStream_t st);
 
 // bits == 16: gather / append raw 16-bit rows of K and V (no quantisation).
 cudaError_t xsv_launch_raw_update(const LayerView& src, const LayerView& dst, const void* Kf,
