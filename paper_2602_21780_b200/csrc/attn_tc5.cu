@@ -940,7 +940,8 @@ constexpr int MAX_PARTS = 256;         // a unit can be shared by as many CTAs a
 template <typename T>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const Params p) {
     __shared__ int s_slot[MAX_PARTS];
-    __shared__ int s_n;
+    __shared__ int s_cand[MAX_PARTS];      // per candidate CTA: -1 nothing of this unit, -2 the whole unit, else its slot
+    __shared__ int s_n, s_b0, s_nb;
     const int u = blockIdx.y;
     if (threadIdx.x == 0) {
         long long base;
@@ -950,12 +951,25 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const Params p) {
         int b0 = (int)(base * p.G / p.total), b1 = (int)((base + (long long)cost * (p.nkv - 1)) * p.G / p.total);
         b0 = max(0, b0 - 1);
         b1 = min(p.G - 1, b1 + 1);
+        s_b0 = b0;
+        s_nb = min(b1 - b0 + 1, MAX_PARTS);
+    }
+    __syncthreads();
+    if (threadIdx.x < s_nb) {              // one candidate per thread: the span arithmetic is long-latency integer work
+        const int b = s_b0 + threadIdx.x;
+        const Span sp = cta_span(p, b, u);
+        int v = -1;
+        if (sp.kv0 < sp.kv1) v = (sp.kv0 == 0 && sp.kv1 == p.nkv) ? -2 : b * 2 + (sp.kv0 > 0 ? 0 : 1);
+        s_cand[threadIdx.x] = v;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
         int n = 0;
-        for (int b = b0; b <= b1; ++b) {
-            const Span sp = cta_span(p, b, u);
-            if (sp.kv0 >= sp.kv1) continue;
-            if (sp.kv0 == 0 && sp.kv1 == p.nkv) { n = 0; break; }   // whole unit in one CTA: already written
-            if (n < MAX_PARTS) s_slot[n++] = b * 2 + (sp.kv0 > 0 ? 0 : 1);
+        for (int i = 0; i < s_nb; ++i) {
+            const int v = s_cand[i];
+            if (v == -1) continue;
+            if (v == -2) { n = 0; break; }   // whole unit in one CTA: already written
+            s_slot[n++] = v;
         }
         s_n = n;
     }

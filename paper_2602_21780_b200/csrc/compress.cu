@@ -465,29 +465,32 @@ __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restric
     }
     if (tid == 0) s_first_evicted = n;
 
-    // ordered compaction
-    int n_gt = 0, n_eq = 0;
+    // ordered compaction.  Positions past n hold key 0, which is never above the threshold; they can only tie with it,
+    // and ties are looked at only when some are to be kept (need_eq is the same in every thread).
+    uint32_t keep = 0;                    // bit i: position j0 + i is kept
 #pragma unroll
-    for (int i = 0; i < KPT; ++i) {
-        const bool valid = j0 + i < n;
-        n_gt += (valid && key[i] > thr) ? 1 : 0;
-        n_eq += (valid && k > 0 && key[i] == thr) ? 1 : 0;
-    }
-    int total = 0, eq_before = 0;
-    if (need_eq > 0) eq_before = sel_block_scan(n_eq, ws, &total);       // need_eq is the same in every thread
-    const int take_eq = max(0, min(n_eq, need_eq - eq_before));
-    int off = sel_block_scan(n_gt + take_eq, ws, &total);
-    int first_ev = n, eq_rank = eq_before;
+    for (int i = 0; i < KPT; ++i) keep |= (key[i] > thr) ? (1u << i) : 0u;
+    int total = 0;
+    if (need_eq > 0) {
+        uint32_t eqm = 0;
 #pragma unroll
-    for (int i = 0; i < KPT; ++i) {
-        const int j = j0 + i;
-        const bool valid = j < n;
-        const bool eq = valid && k > 0 && key[i] == thr;
-        const bool keep = (valid && key[i] > thr) || (eq && eq_rank < need_eq);
-        eq_rank += eq ? 1 : 0;
-        if (keep) sel_sm[off++] = T_first + j;
-        if (valid && !keep) first_ev = min(first_ev, j);
+        for (int i = 0; i < KPT; ++i) eqm |= (j0 + i < n && key[i] == thr) ? (1u << i) : 0u;
+        const int eq_before = sel_block_scan(__popc(eqm), ws, &total);
+        int take = max(0, min(__popc(eqm), need_eq - eq_before));
+        while (take > 0) {                // the lowest positions among the ties
+            const uint32_t low = eqm & (0u - eqm);
+            keep |= low;
+            eqm ^= low;
+            --take;
+        }
     }
+    int off = sel_block_scan(__popc(keep), ws, &total);
+#pragma unroll
+    for (int i = 0; i < KPT; ++i)
+        if (keep & (1u << i)) sel_sm[off++] = T_first + j0 + i;
+    const uint32_t owned = (j0 >= n) ? 0u : ((n - j0 >= KPT) ? ((KPT == 32) ? 0xFFFFFFFFu : ((1u << (KPT & 31)) - 1u)) : ((1u << (n - j0)) - 1u));
+    const uint32_t dropped = owned & ~keep;
+    int first_ev = dropped ? j0 + __ffs(dropped) - 1 : n;
     first_ev = __reduce_min_sync(FULL, first_ev);
     if (lane == 0 && first_ev < n) atomicMin(&s_first_evicted, first_ev);
     __syncthreads();
