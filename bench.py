@@ -265,7 +265,7 @@ def main():
     assert cache.len(0) == L_MAX
     bytes_before = cache.bytes()
 
-    cache.set_profiling(True)
+    cache.set_profiling(2)                 # events around the attention kernel only: its live duration for the roofline
     cache.profile_read(reset=True)
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -285,7 +285,14 @@ def main():
     launches = binding.kernel_launches() - launches0
     clocks = sampler.stop()
     prof = cache.profile_read(reset=True)
-    cache.set_profiling(False)
+    # the other phases, in a short pass of their own after the timed region (events around every phase slow the step)
+    cache.set_profiling(1)
+    n_phase_frames = max(1, min(3, args.steps))
+    for f in range(n_phase_frames):
+        frame_step(cache, PREFILL + args.warmup + args.steps + f)
+    torch.cuda.synchronize()
+    prof_all = cache.profile_read(reset=True)
+    cache.set_profiling(0)
     assert cache.status() == 0, "device status word set"
     assert cache.bytes() == bytes_before, "cache bytes changed in steady state"
     kv_layer = cache.layer_kv_bytes(0)
@@ -313,13 +320,14 @@ def main():
     quant_bytes = n_mid * tok_b + 2 * H * F * D * 2 + (L_MAX - F) * tok_b
     phases = {}
     for name, nbytes in (("score", score_bytes), ("select", n_mid * 4 + k_keep * 4), ("quant", quant_bytes)):
-        pms, pn = prof[name]
-        steps_n = attn_n
+        pms, pn = prof_all[name]
+        steps_n = n_phase_frames * LAYERS
         if steps_n and pms > 0:
             per = pms / steps_n
             phases[name] = {"avg_ms": per, "algorithmic_bytes": nbytes, "GB/s": nbytes / (per * 1e-3) / 1e9,
                             "frac_of_hbm": nbytes / (per * 1e-3) / 1e9 / peaks["hbm"], "launches_per_step": pn / steps_n}
     phases["attn"] = {"avg_ms": attn_ms / attn_n if attn_n else None}
+    phases["note"] = f"score/select/quant: events around every phase, {n_phase_frames} frames after the timed region"
     cache.destroy()
 
     # ---- end to end: same metric through the C ABI with HOST buffers (copies inside the timed region)

@@ -239,10 +239,13 @@ xsv_status xsv_last_scores(xsv_cache* c, float* scores_host, long long cap, long
  * XSV_OK, XSV_ERR_TIMEOUT or XSV_ERR_RANGE. */
 xsv_status xsv_cache_status(xsv_cache* c, void* stream);
 
-/* Per-phase CUDA-event timing.  When on, every step records events around
- * each phase on the step's stream.  xsv_cache_profile_read synchronises the
- * recorded events, adds their durations to per-phase totals, and returns the
- * totals (milliseconds) and launch counts accumulated since the last reset. */
+/* Per-phase CUDA-event timing.  on = 1: every step records events around each
+ * phase on the step's stream; on = 2: around the attention phase only (each
+ * pair of events costs the stream a few microseconds, which matters when the
+ * whole step is being timed as well); on = 0: none.  xsv_cache_profile_read
+ * synchronises the recorded events, adds their durations to per-phase totals,
+ * and returns the totals (milliseconds) and launch counts accumulated since
+ * the last reset. */
 xsv_status xsv_cache_set_profiling(xsv_cache* c, int on);
 xsv_status xsv_cache_profile_read(xsv_cache* c, double ms[XSV_PHASE_COUNT], long long launches[XSV_PHASE_COUNT], int reset);
 

@@ -22,18 +22,31 @@ __global__ void __launch_bounds__(256) qtilde_partial_kernel(const T* __restrict
     float a[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) a[e] = 0.f;
-#pragma unroll 6
-    for (int i = i0 + r; i < i1; i += 32) {
-        float w = 1.f;
-        if (i >= n_special) {
-            const int gi = (i - n_special) / g;
-            w = 1.f / (float)min(g, n_patch - gi * g);
-        }
-        const uint4 v = *reinterpret_cast<const uint4*>(Q + ((size_t)h * F + i) * XSV_D + 8 * c8);
-        T e8[8];
-        *reinterpret_cast<uint4*>(e8) = v;
+    // six rows per thread at a time, all loads issued before the first use
+    for (int base = i0 + r; base < i1; base += 32 * 6) {
+        uint4 v[6];
+        float w[6];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) a[e] = fmaf(w, xsv_to_float<T>(e8[e]), a[e]);
+        for (int k = 0; k < 6; ++k) {
+            const int i = base + 32 * k;
+            v[k] = make_uint4(0u, 0u, 0u, 0u);
+            w[k] = 0.f;
+            if (i < i1) {
+                v[k] = *reinterpret_cast<const uint4*>(Q + ((size_t)h * F + i) * XSV_D + 8 * c8);
+                w[k] = 1.f;
+                if (i >= n_special) {
+                    const int gi = (i - n_special) / g;
+                    w[k] = 1.f / (float)min(g, n_patch - gi * g);
+                }
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 6; ++k) {
+            T e8[8];
+            *reinterpret_cast<uint4*>(e8) = v[k];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) a[e] = fmaf(w[k], xsv_to_float<T>(e8[e]), a[e]);
+        }
     }
     // the four row lanes of a warp, then the eight warps, in a fixed order
 #pragma unroll
@@ -56,16 +69,26 @@ __global__ void __launch_bounds__(256) qtilde_partial_kernel(const T* __restrict
 }
 
 // Fixed-order sum of the n_part partial rows, written over the first row: qpart[0..64) = sum_h sum_i w_i Q[h,i,:].
-__global__ void __launch_bounds__(256) qtilde_final_kernel(float* __restrict__ qpart, int n_part) {
-    __shared__ float red[4][64];
-    const int c = threadIdx.x & 63, part = threadIdx.x >> 6, per = (n_part + 3) / 4;
-    float s4 = 0.f;
-    const int k1 = min(n_part, (part + 1) * per);
-#pragma unroll 8
-    for (int k = part * per; k < k1; ++k) s4 += qpart[(size_t)k * 64 + c];
-    red[part][c] = s4;
+// 1024 threads: 16 per channel, each sums every 16th row (loads issued eight at a time), then a fixed-order sum of the 16.
+__global__ void __launch_bounds__(1024) qtilde_final_kernel(float* __restrict__ qpart, int n_part) {
+    __shared__ float red[16][64];
+    const int c = threadIdx.x & 63, part = threadIdx.x >> 6;
+    float s = 0.f;
+    for (int k0 = part; k0 < n_part; k0 += 16 * 8) {
+        float v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = (k0 + 16 * j < n_part) ? qpart[(size_t)(k0 + 16 * j) * 64 + c] : 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) s += v[j];
+    }
+    red[part][c] = s;
     __syncthreads();       // every partial row has been read
-    if (threadIdx.x < 64) qpart[c] = ((red[0][c] + red[1][c]) + red[2][c]) + red[3][c];
+    if (threadIdx.x < 64) {
+        float t = 0.f;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) t += red[k][c];
+        qpart[c] = t;
+    }
 }
 
 // ---------------------------------------------------------------------------
@@ -121,15 +144,29 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
             // their sub-words)
             const float q0 = qfinal[lane] * qnorm, q1 = qfinal[lane + 32] * qnorm;
             const float pos = __int_as_float((127 - BITS * ((lane & 7) % SUB)) << 23);
-            for (int h = warp; h < H; h += SCORE_TPB / 32) {
-                const size_t m = ((size_t)h * lv.capg + g) * 64;
-                const float w0 = q0 * lv.kscale[m + lane], w1 = q1 * lv.kscale[m + lane + 32];
-                float b = w0 * (float)lv.kzero[m + lane] + w1 * (float)lv.kzero[m + lane + 32];
-                sW[h * 64 + lane] = w0 * pos;
-                sW[h * 64 + lane + 32] = w1 * pos;
+            for (int h0 = warp; h0 < H; h0 += 2 * (SCORE_TPB / 32)) {     // two heads per pass: eight loads in flight
+                float sc[2][2];
+                int zz[2][2];
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) b += __shfl_xor_sync(0xFFFFFFFFu, b, o);
-                if (lane == 0) sB[h] = b;
+                for (int t = 0; t < 2; ++t) {
+                    const int h = h0 + t * (SCORE_TPB / 32);
+                    const size_t m = ((size_t)min(h, H - 1) * lv.capg + g) * 64;
+                    sc[t][0] = lv.kscale[m + lane]; sc[t][1] = lv.kscale[m + lane + 32];
+                    zz[t][0] = lv.kzero[m + lane]; zz[t][1] = lv.kzero[m + lane + 32];
+                }
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    const int h = h0 + t * (SCORE_TPB / 32);
+                    const float w0 = q0 * sc[t][0], w1 = q1 * sc[t][1];
+                    float b = w0 * (float)zz[t][0] + w1 * (float)zz[t][1];
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) b += __shfl_xor_sync(0xFFFFFFFFu, b, o);
+                    if (h < H) {
+                        sW[h * 64 + lane] = w0 * pos;
+                        sW[h * 64 + lane + 32] = w1 * pos;
+                        if (lane == 0) sB[h] = b;
+                    }
+                }
             }
             __syncthreads();
         }
@@ -1024,7 +1061,7 @@ cudaError_t xsv_launch_qtilde(const void* Q, int dtype, int H, int F, int n_spec
     dim3 grid(XSV_QCHUNKS, H);
     if (dtype == 0) qtilde_partial_kernel<__half><<<grid, 256, 0, st>>>((const __half*)Q, F, n_special, g, qpart);
     else qtilde_partial_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)Q, F, n_special, g, qpart);
-    qtilde_final_kernel<<<1, 256, 0, st>>>(qpart, H * XSV_QCHUNKS);
+    qtilde_final_kernel<<<1, 1024, 0, st>>>(qpart, H * XSV_QCHUNKS);
     xsv_count_launch(2);
     return cudaGetLastError();
 }

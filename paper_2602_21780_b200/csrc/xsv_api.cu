@@ -76,7 +76,7 @@ struct xsv_cache {
 
     size_t bytes = 0;
 
-    bool profiling = false;
+    int profiling = 0;          // 0 off, 1 events around every phase, 2 around the attention phase only
     std::vector<PendingEvent> pending;
     std::vector<cudaEvent_t> free_events;
     double prof_ms[XSV_PHASE_COUNT] = {0, 0, 0, 0};
@@ -175,16 +175,18 @@ struct PhaseTimer {
     int phase;
     cudaEvent_t a = nullptr, b = nullptr;
     long long launches0;
+    bool on;
     PhaseTimer(xsv_cache* c_, cudaStream_t st_, int phase_) : c(c_), st(st_), phase(phase_) {
         launches0 = g_launches.load(std::memory_order_relaxed);
-        if (c->profiling) {
+        on = c->profiling == 1 || (c->profiling == 2 && phase == XSV_PHASE_ATTN);
+        if (on) {
             a = get_event(c);
             b = get_event(c);
             cudaEventRecord(a, st);
         }
     }
     ~PhaseTimer() {
-        if (c->profiling) {
+        if (on) {
             cudaEventRecord(b, st);
             c->pending.push_back({phase, a, b});
             c->prof_launches[phase] += g_launches.load(std::memory_order_relaxed) - launches0;
@@ -643,7 +645,8 @@ xsv_status xsv_cache_status(xsv_cache* c, void* stream) {
 
 xsv_status xsv_cache_set_profiling(xsv_cache* c, int on) {
     if (!c) return XSV_ERR_ARG;
-    c->profiling = on != 0;
+    if (on < 0 || on > 2) return XSV_ERR_ARG;
+    c->profiling = on;
     return XSV_OK;
 }
 
