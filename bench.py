@@ -200,7 +200,7 @@ def run_reference(args, rank):
 
 
 def main():
-    global LAYERS, WORKLOAD
+    global LAYERS, WORKLOAD, L_MAX, BITS, PREFILL
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=40)
@@ -211,6 +211,10 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--layers", type=int, default=LAYERS,
                     help="layers in the stack (default 24 = the benchmark; fewer only for profiling a small case)")
+    ap.add_argument("--budget-frames", type=int, default=L_MAX // F,
+                    help="cache budget in frames (default 16 = the benchmark; other values: the cache-length sweep)")
+    ap.add_argument("--bits", type=int, default=BITS, choices=[2, 4, 8, 16],
+                    help="bits per cached element (default 4 = the benchmark; 16 = quantisation off, pruning only)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -221,6 +225,16 @@ def main():
     if args.layers != LAYERS:
         WORKLOAD = WORKLOAD.replace("24 layers", f"{args.layers} layers (profiling case, not the benchmark)")
         LAYERS = args.layers
+    sweep = args.budget_frames * F != L_MAX or args.bits != BITS
+    if sweep:
+        if args.budget_frames < 3:
+            ap.error("--budget-frames must be at least 3")
+        WORKLOAD = (WORKLOAD.replace("config2:", "sweep case (not the benchmark), config2 with")
+                    .replace(f"budget {L_MAX} tokens/layer", f"budget {args.budget_frames * F} tokens/layer")
+                    .replace(f"{BITS}-bit KV", f"{args.bits}-bit KV")
+                    .replace(f"{PREFILL}-frame prefill", f"{args.budget_frames}-frame prefill"))
+        L_MAX, BITS, PREFILL = args.budget_frames * F, args.bits, args.budget_frames
+        args.no_cpu_baseline = True
     if args.warmup < 3:
         args.warmup = 3
 
@@ -309,7 +323,7 @@ def main():
     achieved = flops / (attn_ms / attn_n * 1e-3) / 1e12 if attn_n else None
     roofline = {"bound": "tensor", "kernel": "fused dequant+attention", "achieved": achieved,
                 "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"] if achieved else None,
-                "traffic": attn_traffic_bytes(), "peak_source": peaks["source"],
+                "traffic": None if sweep else attn_traffic_bytes(), "peak_source": peaks["source"],
                 "flops_per_launch": flops, "avg_launch_ms": attn_ms / attn_n if attn_n else None,
                 "kernels_per_launch": attn_launches / attn_n if attn_n else None}
     # the bandwidth-bound phases: algorithmic bytes per layer-step / live duration

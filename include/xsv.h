@@ -152,6 +152,21 @@ xsv_status xsv_importance_scores(const void* Q, const void* keys, int heads, int
                                  float* scores, void* stream);
 
 /*
+ * Quantisation error of the two granularities of Eq. 11, the quantity Table 1
+ * compares: the tensor x [heads][n_tokens][64] (DEVICE, 16-bit elements) is
+ * quantised with Eq. 9-10 -- per channel over groups of 64 consecutive tokens
+ * (per_channel != 0: the scheme Eq. 11 gives to keys; a last, partial group
+ * holds the remaining tokens) or per token over its 64 channels (per_channel
+ * == 0: the scheme for values) -- dequantised with Eq. 12, and the mean of
+ * (x - x~)^2 over all elements, accumulated in float64, is written to
+ * *mse_host (HOST).  bits: 2, 4 or 8.  Allocates and frees its scratch on
+ * `stream` (stream-ordered allocator) and synchronises `stream`.
+ * XSV_ERR_RANGE: a zero-point left the int32 range.
+ */
+xsv_status xsv_quantization_mse(const void* x, int heads, long long n_tokens, xsv_dtype dtype, int bits,
+                                int per_channel, double* mse_host, void* stream);
+
+/*
  * xsv_importance_scores for callers that must not allocate.  (The paper has no
  * counterpart: this is a property of the library, not of the method.)
  *

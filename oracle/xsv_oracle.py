@@ -74,6 +74,31 @@ def dequantize(codes, s, z):
     return (diff.astype(F32) * np.asarray(s, dtype=F32)).astype(F32)
 
 
+def quantization_mse(x, bits, granularity, G=64):
+    """Mean squared error of Eq. 9-12 under one of the two granularities of Eq. 11 (the quantity of Table 1).
+
+    x [H, T, d] (d == G).  granularity "channel": one (s, z) per channel per group of G consecutive tokens (the
+    scheme Eq. 11 assigns to keys; a last, partial group holds the remaining tokens); "token": one (s, z) per token
+    over its d channels (the scheme for values).  Quantise, dequantise, and average (x - x~)^2 over all elements
+    in float64.
+    """
+    x = np.asarray(x, dtype=F32)
+    H, T, d = x.shape
+    if granularity == "token":
+        c, s, z = quantize_groups(x, bits)                       # groups along the channel axis
+        xh = dequantize(c, s[..., None], z[..., None])
+    elif granularity == "channel":
+        xh = np.empty_like(x)
+        for t0 in range(0, T, G):
+            blk = x[:, t0:t0 + G, :].transpose(0, 2, 1)           # [H, d, tokens of the group]
+            c, s, z = quantize_groups(blk, bits)
+            xh[:, t0:t0 + G, :] = dequantize(c, s[..., None], z[..., None]).transpose(0, 2, 1)
+    else:
+        raise ValueError(granularity)
+    e = x.astype(np.float64) - xh.astype(np.float64)
+    return float(np.mean(e * e))
+
+
 # --------------------------------------------------------------------------
 # Eq. 2: attention of one frame's queries over [cache ; current frame].
 # --------------------------------------------------------------------------

@@ -35,6 +35,7 @@ SYMBOLS = {
     "xsv_cache_len": (_ll, [_vp, _i]),
     "xsv_cache_frames": (_ll, [_vp, _i]),
     "xsv_cache_export_layer": (_i, [_vp, _i] + [_vp] * 9 + [_vp]),
+    "xsv_quantization_mse": (_i, [_vp, _i, _ll, _i, _i, _i, C.POINTER(C.c_double), _vp]),
     "xsv_cache_import_layer": (_i, [_vp, _i, _ll, _ll, _i, _i] + [_vp] * 9 + [_vp]),
     "xsv_last_scores": (_i, [_vp, _vp, _ll, C.POINTER(_ll), _vp]),
     "xsv_cache_status": (_i, [_vp, _vp]),
@@ -229,6 +230,15 @@ def importance_scores_static(Q, keys, scores, n_special=5, pool_group=16, stream
     return int(load().xsv_importance_scores_static(Q.data_ptr(), keys.data_ptr(), Q.shape[0], Q.shape[1],
                                                    keys.shape[1], _dtype_code(Q), n_special, pool_group,
                                                    scores.data_ptr(), _stream_ptr(stream)))
+
+
+def quantization_mse(x, bits, per_channel, stream=None):
+    """xsv_quantization_mse: mean squared quantisation error of x [heads, tokens, 64] (fp16/bf16 CUDA tensor)."""
+    out = C.c_double(0.0)
+    _check(load().xsv_quantization_mse(x.data_ptr(), x.shape[0], x.shape[1], _dtype_code(x), int(bits),
+                                       1 if per_channel else 0, C.byref(out), _stream_ptr(stream)),
+           "xsv_quantization_mse")
+    return out.value
 
 
 def selftest_bounded_wait(stream=None):

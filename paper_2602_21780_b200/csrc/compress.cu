@@ -215,24 +215,58 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
         scores[p - T_first] = (((part[tok] + part[64 + tok]) + part[128 + tok]) + part[192 + tok]) / (float)H;
 }
 
-// bits == 16: keys are raw 16-bit values.
+// bits == 16: keys are raw 16-bit values.  64 tokens x 4 head slices per block as above; a warp reads 32 consecutive
+// rows (4 KB) of one head, a thread one 128-byte row at a time with the next one already in flight.
 template <typename T>
 __global__ void __launch_bounds__(SCORE_TPB) score_raw_kernel(LayerView lv, int H, int T_first, int T_c,
                                                               const float* __restrict__ qpart, float qnorm,
                                                               float* __restrict__ scores) {
-    __shared__ float qt[64];
+    __shared__ __align__(16) float qt[64];
+    __shared__ float part[4][64];
     if (threadIdx.x < 64) qt[threadIdx.x] = qpart[threadIdx.x] * qnorm;
-    __syncthreads();
-    const int j = blockIdx.x * SCORE_TPB + threadIdx.x;
+    const int tok = threadIdx.x & 63, slice = threadIdx.x >> 6;
+    const int j = blockIdx.x * 64 + tok;
     const int p = T_first + j;
-    if (p >= T_c) return;
+    const bool valid = p < T_c;
+    uint4 cur[8], nxt[8];
+    auto load_row = [&](int h, uint4 (&r)[8]) {
+        if (valid && h < H) {
+            const uint4* row = reinterpret_cast<const uint4*>(lv.kcodes + ((size_t)h * lv.cap + p) * (XSV_D * 2));
+#pragma unroll
+            for (int v = 0; v < 8; ++v) r[v] = row[v];
+        } else {
+#pragma unroll
+            for (int v = 0; v < 8; ++v) r[v] = make_uint4(0u, 0u, 0u, 0u);
+        }
+    };
+    load_row(slice, cur);
+    __syncthreads();
     float acc = 0.f;
-    for (int h = 0; h < H; ++h) {
-        const T* row = reinterpret_cast<const T*>(lv.kcodes + ((size_t)h * lv.cap + p) * (XSV_D * 2));
-#pragma unroll 8
-        for (int c = 0; c < XSV_D; ++c) acc = fmaf(qt[c], xsv_to_float<T>(row[c]), acc);
+    for (int h = slice; h < H; h += 4) {
+        load_row(h + 4, nxt);
+        float a = 0.f;
+#pragma unroll
+        for (int v = 0; v < 8; ++v) {
+            const uint32_t u[4] = {cur[v].x, cur[v].y, cur[v].z, cur[v].w};
+            const float4 q0 = reinterpret_cast<const float4*>(qt)[2 * v], q1 = reinterpret_cast<const float4*>(qt)[2 * v + 1];
+            const float qq[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                T lo, hi;
+                *reinterpret_cast<uint16_t*>(&lo) = (uint16_t)(u[e] & 0xFFFFu);
+                *reinterpret_cast<uint16_t*>(&hi) = (uint16_t)(u[e] >> 16);
+                a = fmaf(qq[2 * e], xsv_to_float<T>(lo), a);
+                a = fmaf(qq[2 * e + 1], xsv_to_float<T>(hi), a);
+            }
+        }
+        acc += a;
+#pragma unroll
+        for (int v = 0; v < 8; ++v) cur[v] = nxt[v];
     }
-    scores[j] = acc / (float)H;
+    part[slice][tok] = acc;
+    __syncthreads();
+    if (threadIdx.x < 64 && valid)
+        scores[j] = (((part[0][tok] + part[1][tok]) + part[2][tok]) + part[3][tok]) / (float)H;
 }
 
 // ---------------------------------------------------------------------------
@@ -1098,7 +1132,7 @@ cudaError_t xsv_launch_score_raw(const LayerView& lv, int dtype, int H, int T_fi
                                  float qnorm, float* scores, cudaStream_t st) {
     const int n = T_c - T_first;
     if (n <= 0) return cudaSuccess;
-    const int grid = (n + SCORE_TPB - 1) / SCORE_TPB;
+    const int grid = (n + 63) / 64;
     if (dtype == 0) score_raw_kernel<__half><<<grid, SCORE_TPB, 0, st>>>(lv, H, T_first, T_c, qpart, qnorm, scores);
     else score_raw_kernel<__nv_bfloat16><<<grid, SCORE_TPB, 0, st>>>(lv, H, T_first, T_c, qpart, qnorm, scores);
     xsv_count_launch();

@@ -3,6 +3,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import xsv_oracle as orc
 from paper_2602_21780_b200 import binding, synth
 from tests.gpu_harness import run_stream
 
@@ -89,6 +90,22 @@ def test_checkpoint_restore_continues_the_stream(bits):
             assert np.array_equal(sa[key], sb[key])
     assert a.status() == 0 and b.status() == 0
     a.destroy(); b.destroy()
+
+
+@pytest.mark.parametrize("dtype", ["fp16", "bf16"])
+def test_quantization_mse_matches_oracle(dtype):
+    # the granularity study of Table 1 on the synthetic keys (outlier channels) and values; 300 tokens = 4 full groups
+    # and a partial one
+    st = synth.Stream(H=3, d=64, F=300, dtype=dtype, layer=12)
+    _, K, V = st.frame(0)
+    tdt = torch.float16 if dtype == "fp16" else torch.bfloat16
+    for name, x in (("K", K), ("V", V)):
+        xd = torch.from_numpy(x).to("cuda:0", tdt).contiguous()
+        for bits in (2, 4, 8):
+            for gran in ("channel", "token"):
+                got = binding.quantization_mse(xd, bits, gran == "channel")
+                want = orc.quantization_mse(x, bits, gran)
+                assert got == pytest.approx(want, rel=1e-9), (name, bits, gran)
 
 
 def test_pooling_options_and_multi_layer():

@@ -5,6 +5,7 @@ import numpy as np
 import pytest
 
 from oracle import xsv_oracle as orc
+from paper_2602_21780_b200 import synth
 
 
 def _rows(path):
@@ -120,3 +121,64 @@ def test_granularity_direction_matches_table1():
         assert mse(K, False, bits) > factor * mse(K, True, bits)
         rv = mse(V, False, bits) / mse(V, True, bits)
         assert 0.5 < rv < 2.0
+
+
+# --------------------------------------------------------------------------
+# quantization_mse (Eq. 11 granularities, the quantity of Table 1)
+# --------------------------------------------------------------------------
+def test_mse_is_zero_for_values_on_the_grid():
+    rng = np.random.default_rng(3)
+    for bits in (2, 4, 8):
+        n = (1 << bits) - 1
+        # per token: every token's 64 channels lie on a grid with step 2^-3 that contains both ends
+        c = rng.integers(0, n + 1, size=(2, 70, 64))
+        c[..., 0], c[..., 1] = 0, n
+        z = rng.integers(-5, 6, size=(2, 70, 1))
+        x = ((c - z) * 0.125).astype(np.float32)
+        assert orc.quantization_mse(x, bits, "token") == 0.0
+        # per channel: the same construction along the token axis, groups of 64 tokens (the second group is partial)
+        c = rng.integers(0, n + 1, size=(2, 70, 64))
+        c[:, 0, :], c[:, 1, :], c[:, 64, :], c[:, 65, :] = 0, n, 0, n
+        x = ((c - 3) * 0.25).astype(np.float32)
+        assert orc.quantization_mse(x, bits, "channel") == 0.0
+
+
+def test_mse_hand_worked_example():
+    # 2 bits (n = 3).  Token 0: [0, 1, 3] -> s = 1, z = 0, exact.  Token 1: [0, 0.4, 3] -> s = 1, 0.4 rounds to 0.
+    x = np.array([[[0.0, 1.0, 3.0], [0.0, 0.4, 3.0]]], dtype=np.float32)
+    want = float(np.float64(np.float32(0.4)) ** 2) / 6.0
+    assert orc.quantization_mse(x, 2, "token") == pytest.approx(want, rel=1e-12)
+    # per channel over the (partial) group of the two tokens: channel 1 is [1, 0.4] -> s = 0.2, z = round(-0.4/0.2) = -2,
+    # codes 3 and 0, dequantised (3+2)*0.2 = 1.0 and 0.4 up to float32 rounding; channels 0 and 2 are constant
+    got = orc.quantization_mse(x, 2, "channel")
+    assert got < 1e-14
+
+
+def test_mse_per_channel_is_per_token_of_the_transpose():
+    rng = np.random.default_rng(4)
+    x = rng.normal(size=(3, 64, 64)).astype(np.float32)
+    for bits in (2, 4):
+        a, b = orc.quantization_mse(x, bits, "channel"), orc.quantization_mse(x.transpose(0, 2, 1).copy(), bits, "token")
+        assert a == pytest.approx(b, rel=1e-12)      # same groups, same errors; only the order of the float64 sum differs
+
+
+def test_mse_of_uniform_data_is_step_squared_over_twelve():
+    rng = np.random.default_rng(5)
+    x = rng.uniform(-1.0, 1.0, size=(4, 256, 64)).astype(np.float32)
+    for bits in (4, 8):
+        n = (1 << bits) - 1
+        step = 2.0 / n                       # groups of 64 uniform samples span almost the whole interval
+        got = orc.quantization_mse(x, bits, "token")
+        assert 0.8 * step * step / 12 < got < 1.05 * step * step / 12
+
+
+def test_mse_direction_of_table_1_on_outlier_channels():
+    # keys with a few channels of ten-fold magnitude (Fig. 4): per-channel groups keep the outliers apart, per-token
+    # groups stretch every token's range over them; values without outliers show no such gap
+    st = synth.Stream(H=4, d=64, F=256, dtype="bf16", layer=2)
+    _, K, V = st.frame(0)
+    for bits, gap in ((2, 1.0), (4, 0.3), (8, 0.3)):
+        k_ch, k_tok = orc.quantization_mse(K, bits, "channel"), orc.quantization_mse(K, bits, "token")
+        v_ch, v_tok = orc.quantization_mse(V, bits, "channel"), orc.quantization_mse(V, bits, "token")
+        assert k_ch < gap * k_tok      # at 2 bits the outlier channels' own error dominates both schemes
+        assert 0.9 < v_ch / v_tok < 1.1
