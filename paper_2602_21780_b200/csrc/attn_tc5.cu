@@ -881,6 +881,7 @@ __device__ __noinline__ void mma_loop(const Params& p, const Cta c) {
 // ------------------------------------------------------------------ the kernel
 template <typename T, int BITS>
 __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_constant__ Params p) {
+    xsv_dep_release();
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t smem_base = smem_u32(smem);
@@ -922,6 +923,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_cons
 
     const Cta cta{smem, smem_base, bar_base, tmem_base, abort_flag, b, u_first, u_last};
 
+    xsv_dep_sync();      // everything above is set-up that touches no global memory
     if (warp < 8) softmax_loop<T, BITS>(p, cta);
     else if (warp < 8 + NPROD) producer_loop<T, BITS>(p, cta);
     else mma_loop(p, cta);
@@ -939,6 +941,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_cons
 constexpr int MAX_PARTS = 256;         // a unit can be shared by as many CTAs as there are; the launcher keeps G <= MAX_PARTS
 template <typename T>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const Params p) {
+    xsv_dep_release();
     __shared__ int s_slot[MAX_PARTS];
     __shared__ int s_cand[MAX_PARTS];      // per candidate CTA: -1 nothing of this unit, -2 the whole unit, else its slot
     __shared__ int s_n, s_b0, s_nb;
@@ -976,6 +979,7 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const Params p) {
     __syncthreads();
     const int n = s_n;
     if (n == 0) return;
+    xsv_dep_sync();      // the part list is arithmetic on the parameters; the parts themselves come from the attention kernel
     const int h = u / p.npair, mp = u - h * p.npair;
     const int row = blockIdx.x * 16 + (threadIdx.x >> 4), c4 = threadIdx.x & 15;
     const int grow = mp * 2 * BM + row;
@@ -1030,8 +1034,8 @@ cudaError_t launch(const Params& p, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         attr_set = true;
     }
-    attn_tc5_kernel<T, BITS><<<p.G, NTHREADS, SMEM_BYTES, st>>>(p);
-    attn_combine_kernel<T><<<dim3(16, p.H * p.npair), 256, 0, st>>>(p);
+    xsv_launch_dep(attn_tc5_kernel<T, BITS>, dim3(p.G), dim3(NTHREADS), SMEM_BYTES, st, p);
+    xsv_launch_dep(attn_combine_kernel<T>, dim3(16, p.H * p.npair), dim3(256), 0, st, p);
     xsv_count_launch(2);
     return cudaGetLastError();
 }

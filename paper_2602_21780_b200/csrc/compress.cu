@@ -1,6 +1,8 @@
 // Bandwidth-bound kernels of the step: pooled-query reduction and importance
 // scores (Eq. 3-7), top-k selection (Eq. 8), quantise-and-pack of the new
 // cache order (Eq. 9-11).
+#include <cstdlib>
+
 #include "xsv_kernels.h"
 
 namespace {
@@ -14,6 +16,8 @@ namespace {
 template <typename T>
 __global__ void __launch_bounds__(256) qtilde_partial_kernel(const T* __restrict__ Q, int F, int n_special,
                                                              int g, float* __restrict__ qpart) {
+    xsv_dep_release();
+    xsv_dep_sync();
     const int h = blockIdx.y, chunk = blockIdx.x;
     const int per = (F + XSV_QCHUNKS - 1) / XSV_QCHUNKS;
     const int i0 = chunk * per, i1 = min(F, i0 + per);
@@ -71,6 +75,8 @@ __global__ void __launch_bounds__(256) qtilde_partial_kernel(const T* __restrict
 // Fixed-order sum of the n_part partial rows, written over the first row: qpart[0..64) = sum_h sum_i w_i Q[h,i,:].
 // 1024 threads: 16 per channel, each sums every 16th row (loads issued eight at a time), then a fixed-order sum of the 16.
 __global__ void __launch_bounds__(1024) qtilde_final_kernel(float* __restrict__ qpart, int n_part) {
+    xsv_dep_release();
+    xsv_dep_sync();
     __shared__ float red[16][64];
     const int c = threadIdx.x & 63, part = threadIdx.x >> 6;
     float s = 0.f;
@@ -110,6 +116,8 @@ template <int BITS>
 __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, int T_first, int T_c,
                                                           const float* __restrict__ qfinal, float qnorm,
                                                           float* __restrict__ scores) {
+    xsv_dep_release();
+    xsv_dep_sync();
     constexpr int ROWB = XSV_D * BITS / 8;
     constexpr int NV = ROWB / 16;              // 16-byte loads per row
     constexpr int SUB = (BITS == 8) ? 2 : (BITS == 4 ? 4 : 8);   // codes per 16-bit sub-word
@@ -221,6 +229,8 @@ template <typename T>
 __global__ void __launch_bounds__(SCORE_TPB) score_raw_kernel(LayerView lv, int H, int T_first, int T_c,
                                                               const float* __restrict__ qpart, float qnorm,
                                                               float* __restrict__ scores) {
+    xsv_dep_release();
+    xsv_dep_sync();
     __shared__ __align__(16) float qt[64];
     __shared__ float part[4][64];
     if (threadIdx.x < 64) qt[threadIdx.x] = qpart[threadIdx.x] * qnorm;
@@ -283,6 +293,8 @@ __device__ __forceinline__ uint32_t score_key(float s) {
 __global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ scores, int n, int k,
                                                       int T_first, int T_c, int* __restrict__ srcmap,
                                                       int* __restrict__ dscal) {
+    xsv_dep_release();
+    xsv_dep_sync();
     __shared__ int hist[256];
     __shared__ uint32_t s_prefix;
     __shared__ int s_remaining;
@@ -415,6 +427,8 @@ __device__ __forceinline__ int sel_block_scan(int v, int* ws, int* total) {
 template <int KPT>
 __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restrict__ scores, int n, int k, int T_first,
                                                           int T_c, int* __restrict__ srcmap, int* __restrict__ dscal) {
+    xsv_dep_release();
+    xsv_dep_sync();
     extern __shared__ __align__(16) int sel_sm[];     // [1024 * KPT]: undecided keys, later the kept positions
     __shared__ int cnt[36];
     __shared__ uint32_t s_lo, s_hi;
@@ -752,6 +766,8 @@ __global__ void __launch_bounds__(RQ_THREADS, 3) requant_k_kernel(LayerView src,
                                                                const int* __restrict__ fz_dev, int fz_host,
                                                                int g_base, int n_items, int n_vg, int n_vq,
                                                                long long origin0, int* __restrict__ status) {
+    xsv_dep_release();
+    xsv_dep_sync();
     using C = RqCfg<BITS>;
     constexpr int ROWB = C::ROWB, SUB = C::SUB, NSUB = C::NSUB;
     constexpr int NMAX = (1 << BITS) - 1;
@@ -1024,6 +1040,8 @@ __global__ void __launch_bounds__(RQ_THREADS, 3) requant_k_kernel(LayerView src,
 template <int ROWB>
 __global__ void __launch_bounds__(256) gather_v_kernel(LayerView src, LayerView dst, int H, int n_old_new,
                                                        int T_first, const int* __restrict__ srcmap) {
+    xsv_dep_release();
+    xsv_dep_sync();
     constexpr int PPR = ROWB / 16;
     const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
     const long long total = (long long)H * n_old_new * PPR;
@@ -1047,6 +1065,8 @@ __global__ void __launch_bounds__(256) gather_v_kernel(LayerView src, LayerView 
 // Same for raw 16-bit key rows (bits == 16).
 __global__ void __launch_bounds__(256) gather_kraw_kernel(LayerView src, LayerView dst, int H, int n_old_new,
                                                           int T_first, const int* __restrict__ srcmap) {
+    xsv_dep_release();
+    xsv_dep_sync();
     constexpr int PPR = 8;
     const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
     const long long total = (long long)H * n_old_new * PPR;
@@ -1064,6 +1084,8 @@ __global__ void __launch_bounds__(256) gather_kraw_kernel(LayerView src, LayerVi
 __global__ void __launch_bounds__(256) append_raw_kernel(LayerView dst, const uint4* __restrict__ Kf,
                                                          const uint4* __restrict__ Vf, int H, int F,
                                                          int n_old_new, long long origin0) {
+    xsv_dep_release();
+    xsv_dep_sync();
     const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
     const long long total = (long long)H * F * 8;
     if (idx >= total) return;
@@ -1079,6 +1101,11 @@ __global__ void __launch_bounds__(256) append_raw_kernel(LayerView dst, const ui
 }  // namespace
 
 // ------------------------------ launchers ----------------------------------
+bool xsv_dep_launch_enabled() {
+    static const bool on = (getenv("XSV_NO_DEP_LAUNCH") == nullptr);
+    return on;
+}
+
 int xsv_sm_count() {
     static int n = 0;
     if (n == 0) {
@@ -1093,9 +1120,9 @@ int xsv_sm_count() {
 cudaError_t xsv_launch_qtilde(const void* Q, int dtype, int H, int F, int n_special, int g, float* qpart,
                               cudaStream_t st) {
     dim3 grid(XSV_QCHUNKS, H);
-    if (dtype == 0) qtilde_partial_kernel<__half><<<grid, 256, 0, st>>>((const __half*)Q, F, n_special, g, qpart);
-    else qtilde_partial_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>((const __nv_bfloat16*)Q, F, n_special, g, qpart);
-    qtilde_final_kernel<<<1, 1024, 0, st>>>(qpart, H * XSV_QCHUNKS);
+    if (dtype == 0) xsv_launch_dep(qtilde_partial_kernel<__half>, grid, dim3(256), 0, st, (const __half*)Q, F, n_special, g, qpart);
+    else xsv_launch_dep(qtilde_partial_kernel<__nv_bfloat16>, grid, dim3(256), 0, st, (const __nv_bfloat16*)Q, F, n_special, g, qpart);
+    xsv_launch_dep(qtilde_final_kernel, dim3(1), dim3(1024), 0, st, qpart, H * XSV_QCHUNKS);
     xsv_count_launch(2);
     return cudaGetLastError();
 }
@@ -1115,7 +1142,7 @@ cudaError_t xsv_launch_score(const LayerView& lv, int H, int T_first, int T_c, c
             if (e != cudaSuccess) return e;                                                                \
             attr_set = true;                                                                               \
         }                                                                                                  \
-        score_kernel<B><<<grid, SCORE_TPB, smem, st>>>(lv, H, T_first, T_c, qpart, qnorm, scores);         \
+        xsv_launch_dep(score_kernel<B>, dim3(grid), dim3(SCORE_TPB), smem, st, lv, H, T_first, T_c, qpart, qnorm, scores); \
     }
     switch (lv.bits) {
         case 2: XSV_SCORE(2) break;
@@ -1133,8 +1160,8 @@ cudaError_t xsv_launch_score_raw(const LayerView& lv, int dtype, int H, int T_fi
     const int n = T_c - T_first;
     if (n <= 0) return cudaSuccess;
     const int grid = (n + 63) / 64;
-    if (dtype == 0) score_raw_kernel<__half><<<grid, SCORE_TPB, 0, st>>>(lv, H, T_first, T_c, qpart, qnorm, scores);
-    else score_raw_kernel<__nv_bfloat16><<<grid, SCORE_TPB, 0, st>>>(lv, H, T_first, T_c, qpart, qnorm, scores);
+    if (dtype == 0) xsv_launch_dep(score_raw_kernel<__half>, dim3(grid), dim3(SCORE_TPB), 0, st, lv, H, T_first, T_c, qpart, qnorm, scores);
+    else xsv_launch_dep(score_raw_kernel<__nv_bfloat16>, dim3(grid), dim3(SCORE_TPB), 0, st, lv, H, T_first, T_c, qpart, qnorm, scores);
     xsv_count_launch();
     return cudaGetLastError();
 }
@@ -1150,13 +1177,13 @@ cudaError_t xsv_launch_select(const float* scores, int n, int k, int T_first, in
             if (e != cudaSuccess) return e;                                                                      \
             attr_set = true;                                                                                     \
         }                                                                                                        \
-        select_reg_kernel<KPT><<<1, 1024, 1024 * KPT * 4, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);      \
+        xsv_launch_dep(select_reg_kernel<KPT>, dim3(1), dim3(1024), 1024 * KPT * 4, st, scores, n, k, T_first, T_c, srcmap, dscal); \
     }
     if (n <= 1024 * 8) XSV_SEL(8)
     else if (n <= 1024 * 16) XSV_SEL(16)
     else if (n <= 1024 * 24) XSV_SEL(24)
     else if (n <= 1024 * 32) XSV_SEL(32)
-    else select_kernel<<<1, 1024, 0, st>>>(scores, n, k, T_first, T_c, srcmap, dscal);
+    else xsv_launch_dep(select_kernel, dim3(1), dim3(1024), 0, st, scores, n, k, T_first, T_c, srcmap, dscal);
 #undef XSV_SEL
     xsv_count_launch();
     return cudaGetLastError();
@@ -1184,9 +1211,9 @@ cudaError_t xsv_launch_compress(const LayerView& src, const LayerView& dst, cons
                 per_sm = 2;                                                                                          \
         }                                                                                                            \
         const int grid = min((n_all + wpb - 1) / wpb, xsv_sm_count() * per_sm);                                      \
-        requant_k_kernel<TT, B><<<grid, RQ_THREADS, smem, st>>>(src, dst, (const TT*)Kf, (const TT*)Vf, H, F,        \
-                                                                n_old_new, T_new, T_first, srcmap, fz_dev, fz_host,  \
-                                                                g0, n_items, n_vg, n_vq, origin0, status);           \
+        xsv_launch_dep(requant_k_kernel<TT, B>, dim3(grid), dim3(RQ_THREADS), smem, st, src, dst, (const TT*)Kf,     \
+                       (const TT*)Vf, H, F, n_old_new, T_new, T_first, srcmap, fz_dev, fz_host, g0, n_items, n_vg,   \
+                       n_vq, origin0, status);                                                                       \
     }
     if (dtype == 0) {
         switch (src.bits) {
@@ -1214,12 +1241,12 @@ cudaError_t xsv_launch_raw_update(const LayerView& src, const LayerView& dst, co
     if (src.kcodes != dst.kcodes && n_old_new > 0) {
         const long long total = (long long)H * n_old_new * 8;
         const int grid = (int)((total + 255) / 256);
-        gather_kraw_kernel<<<grid, 256, 0, st>>>(src, dst, H, n_old_new, T_first, srcmap);
-        gather_v_kernel<128><<<grid, 256, 0, st>>>(src, dst, H, n_old_new, T_first, srcmap);
+        xsv_launch_dep(gather_kraw_kernel, dim3(grid), dim3(256), 0, st, src, dst, H, n_old_new, T_first, srcmap);
+        xsv_launch_dep(gather_v_kernel<128>, dim3(grid), dim3(256), 0, st, src, dst, H, n_old_new, T_first, srcmap);
         xsv_count_launch(2);
     }
     const long long total = (long long)H * F * 8;
-    append_raw_kernel<<<(int)((total + 255) / 256), 256, 0, st>>>(dst, (const uint4*)Kf, (const uint4*)Vf, H, F,
+    xsv_launch_dep(append_raw_kernel, dim3((int)((total + 255) / 256)), dim3(256), 0, st, dst, (const uint4*)Kf, (const uint4*)Vf, H, F,
                                                                   n_old_new, origin0);
     xsv_count_launch();
     return cudaGetLastError();

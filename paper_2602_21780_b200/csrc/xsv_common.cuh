@@ -101,5 +101,32 @@ __device__ __forceinline__ int xsv_quant_code(float x, float s, float inv_s, int
     return (int)(v < 0 ? 0 : (v > n ? n : v));
 }
 
+// Programmatic dependent launch.  A kernel launched with xsv_launch_dep may be scheduled while the kernel before
+// it in the stream is still running (once all of that kernel's blocks have called xsv_dep_release or exited); it must
+// call xsv_dep_sync() before it touches anything the earlier kernel reads or writes: the call returns when that kernel
+// has completed and its writes are visible.  Every kernel of the step calls xsv_dep_release() first, so that its own
+// successor is scheduled early too; what is saved is the launch latency between dependent kernels.  Without the
+// launch attribute both calls do nothing.
+__device__ __forceinline__ void xsv_dep_release() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void xsv_dep_sync() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+bool xsv_dep_launch_enabled();   // false when the environment variable XSV_NO_DEP_LAUNCH is set (host side)
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t xsv_launch_dep(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                  Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = xsv_dep_launch_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // Launch counter (host side), bumped by every kernel launch of the library.
 void xsv_count_launch(int n = 1);
