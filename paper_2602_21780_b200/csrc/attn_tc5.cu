@@ -37,8 +37,10 @@ constexpr int NSTAGE = 5;          // kv stages in shared memory
 constexpr int NPROD = 7;              // producer warps
 constexpr int NTHREADS = (8 + NPROD + 1) * 32;   // 8 softmax warps, the producers, the MMA issuer
 constexpr uint32_t TILE_BYTES = 128u * 128u;   // 128 rows x 64 fp16
-constexpr int COST_PAIR = 8, COST_SINGLE = 7;  // relative cost of a kv step with two / one active query tile (measured: the
-                                               // hand-over latencies, not the arithmetic, set the pace of a step)
+// Cost model of the work split, in ticks (fitted to per-CTA durations measured with %globaltimer): a kv step with two
+// active query tiles, with one (the hand-over latencies, not the arithmetic, set the pace of a step), and the fixed
+// cost of entering a unit (query tiles loaded, the first tile's rescale, the epilogue).
+constexpr int COST_PAIR = 16, COST_SINGLE = 13, COST_UNIT = 72;
 constexpr float RESCALE_THRESHOLD = 8.f;       // log2 units; below it the stale row maximum is kept
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
@@ -75,15 +77,20 @@ constexpr int PART_STRIDE = 256 * 66;   // floats per (CTA, slot)
 // ------------------------------------------------------------------ work split
 struct Span { int kv0, kv1; };
 
+// A unit's ticks: COST_UNIT, then its kv steps.  Inside a head the units with two active query tiles come first.
+__host__ __device__ inline long long unit_len(const Params& p, bool pair) {
+    return (long long)(pair ? COST_PAIR : COST_SINGLE) * p.nkv + COST_UNIT;
+}
 __host__ __device__ inline void unit_base_cost(const Params& p, int u, long long& base, int& cost) {
     const int h = u / p.npair, mp = u - h * p.npair;
     cost = mp < p.n_full ? COST_PAIR : COST_SINGLE;
-    base = h * p.ticks_head + (long long)(mp < p.n_full ? mp : p.n_full) * COST_PAIR * p.nkv;
+    base = h * p.ticks_head + (long long)(mp < p.n_full ? mp : p.n_full) * unit_len(p, true) +
+           (long long)(mp > p.n_full ? mp - p.n_full : 0) * unit_len(p, false);
 }
 __host__ __device__ inline int unit_of_tick(const Params& p, long long t) {
     const long long h = t / p.ticks_head, r = t - h * p.ticks_head;
-    long long mp = r / ((long long)COST_PAIR * p.nkv);
-    if (mp > p.n_full) mp = p.n_full;
+    long long mp = r / unit_len(p, true);
+    if (mp > p.n_full) mp = p.n_full + (r - p.n_full * unit_len(p, true)) / unit_len(p, false);
     if (mp >= p.npair) mp = p.npair - 1;
     return (int)(h * p.npair + mp);
 }
@@ -93,7 +100,7 @@ __host__ __device__ inline Span cta_span(const Params& p, int b, int u) {
     long long base;
     int cost;
     unit_base_cost(p, u, base, cost);
-    const long long t0 = cta_tick(p, b) - base, t1 = cta_tick(p, b + 1) - base;
+    const long long t0 = cta_tick(p, b) - base - COST_UNIT, t1 = cta_tick(p, b + 1) - base - COST_UNIT;   // kv step j starts at tick j * cost
     long long a = t0 <= 0 ? 0 : (t0 + cost - 1) / cost, e = t1 <= 0 ? 0 : (t1 + cost - 1) / cost;
     if (a > p.nkv) a = p.nkv;
     if (e > p.nkv) e = p.nkv;
@@ -881,7 +888,6 @@ __device__ __noinline__ void mma_loop(const Params& p, const Cta c) {
 // ------------------------------------------------------------------ the kernel
 template <typename T, int BITS>
 __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_constant__ Params p) {
-    xsv_dep_release();
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t smem_base = smem_u32(smem);
@@ -929,6 +935,9 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_cons
     else mma_loop(p, cta);
     tc_fence_before();
     __syncthreads();
+    // Only now may the next kernel be scheduled: released at the start, its blocks would sit through this whole kernel
+    // on whatever multiprocessor the grid leaves free (the one kept for the selection kernel of another stream).
+    xsv_dep_release();
     if (warp == 8 + NPROD) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
@@ -951,7 +960,7 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const Params p) {
         int cost;
         unit_base_cost(p, u, base, cost);
         // CTAs that may hold steps of this unit
-        int b0 = (int)(base * p.G / p.total), b1 = (int)((base + (long long)cost * (p.nkv - 1)) * p.G / p.total);
+        int b0 = (int)(base * p.G / p.total), b1 = (int)((base + COST_UNIT + (long long)cost * (p.nkv - 1)) * p.G / p.total);
         b0 = max(0, b0 - 1);
         b1 = min(p.G - 1, b1 + 1);
         s_b0 = b0;
@@ -1051,7 +1060,7 @@ cudaError_t xsv_launch_wait_selftest(int* status, cudaStream_t st) {
 size_t xsv_attn_tc5_workspace_bytes() { return (size_t)sm_count() * 2 * PART_STRIDE * sizeof(float); }
 
 cudaError_t xsv_launch_attn_tc5(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V, void* out,
-                                int dtype, int H, int F, float* workspace, int* status, cudaStream_t st) {
+                                int dtype, int H, int F, float* workspace, int* status, int spare_sms, cudaStream_t st) {
     if (!workspace) return cudaErrorNotSupported;
     Params p{};
     p.lv = lv; p.Q = Q; p.K = K; p.V = V; p.out = out; p.part = workspace; p.status = status;
@@ -1060,10 +1069,11 @@ cudaError_t xsv_launch_attn_tc5(const LayerView& lv, int T_c, const void* Q, con
     p.nkv = p.n_ct + (F + BN - 1) / BN;
     p.npair = (F + 2 * BM - 1) / (2 * BM);
     p.n_full = ((p.npair - 1) * 2 * BM + BM < F) ? p.npair : p.npair - 1;
-    p.ticks_head = (long long)p.nkv * (COST_PAIR * p.n_full + COST_SINGLE * (p.npair - p.n_full));
+    p.ticks_head = p.n_full * unit_len(p, true) + (p.npair - p.n_full) * unit_len(p, false);
     p.total = p.ticks_head * H;
     const long long steps = (long long)H * p.npair * p.nkv;
-    p.G = (int)(steps < sm_count() ? steps : sm_count());
+    const int sms = sm_count() - spare_sms > 0 ? sm_count() - spare_sms : 1;   // multiprocessors left to another kernel
+    p.G = (int)(steps < sms ? steps : sms);
     if (p.G > MAX_PARTS) p.G = MAX_PARTS;
 #define XSV_TC5(TT, B) return launch<TT, B>(p, st)
     if (dtype == 0) {

@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <cstdlib>
 #include <vector>
 
 #include "../../include/xsv.h"
@@ -69,6 +70,8 @@ struct xsv_cache {
     void* stage = nullptr;
     size_t stage_bytes = 0;
     cudaStream_t cs_in = nullptr, cs_out = nullptr;
+    cudaStream_t cs_sel = nullptr;                          // the selection kernel runs here, beside the attention kernel
+    cudaEvent_t ev_scored = nullptr, ev_selected = nullptr;
     cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
     bool slot_used[2] = {false, false}, out_pending[2] = {false, false};
     bool defer_output = false;
@@ -167,6 +170,12 @@ cudaEvent_t get_event(xsv_cache* c) {
     cudaEvent_t e = nullptr;
     cudaEventCreate(&e);
     return e;
+}
+
+// The selection kernel is one block; XSV_NO_SIDE_SELECT keeps it on the caller's stream (for comparisons).
+bool side_select_enabled() {
+    static const bool on = (getenv("XSV_NO_SIDE_SELECT") == nullptr);
+    return on;
 }
 
 struct PhaseTimer {
@@ -294,28 +303,18 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
     const LayerView& lv = c->bufs[cur].view;
     cudaError_t e;
 
-    // ---- Eq. 2 / Eq. 12: attention over [cache ; frame]
-    {
-        PhaseTimer pt(c, st, XSV_PHASE_ATTN);
-        e = cudaErrorNotSupported;
-        if (c->attn_impl != XSV_ATTN_MMA)
-            e = xsv_launch_attn_tc5(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, c->attn_ws, c->status, st);
-        if (e == cudaErrorNotSupported) {
-            if (c->attn_impl == XSV_ATTN_TC5) return XSV_ERR_ARG;
-            e = xsv_launch_attn_mma(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, st);
-        }
-        if (e != cudaSuccess) return cuda_fail(e);
-    }
-
     const long long origin0 = (t - 1) * (long long)F;
+    const int T_first = F;   // constant frame size: the first frame holds F tokens
+    const int n_mid = (int)(T_c - T_first);
+    const long long kk = c->L_max - T_first - F;
+    const int k = (int)(kk > 0 ? kk : 0);
+    // The scores (Eq. 3-7) need the frame's queries and the cached keys only, so they come first; the selection
+    // (Eq. 8), one block that is bound by latency, then runs on a stream of its own: it takes the first multiprocessor
+    // that an attention CTA leaves (the CTAs' finishing times are spread over some tens of microseconds) and so
+    // overlaps the tail of the attention kernel and the merge kernel.  Leaving it a multiprocessor of its own for the
+    // whole attention kernel measured slightly slower.
+    const bool side_select = prune && side_select_enabled() && c->attn_impl != XSV_ATTN_MMA && c->attn_ws != nullptr;
     if (prune) {
-        const int T_first = F;   // constant frame size: the first frame holds F tokens
-        const int n_mid = (int)(T_c - T_first);
-        const long long kk = c->L_max - T_first - F;
-        const int k = (int)(kk > 0 ? kk : 0);
-        const int n_old_new = T_first + k;
-        const int T_new = n_old_new + F;
-        const LayerView& dv = c->bufs[c->spare].view;
         {   // ---- Eq. 3-7
             PhaseTimer pt(c, st, XSV_PHASE_SCORE);
             e = xsv_launch_qtilde(Q, (int)dtype, H, F, c->n_special, c->g, c->qpart, st);
@@ -326,11 +325,44 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
             else e = xsv_launch_score(lv, H, T_first, (int)T_c, c->qpart, qnorm, c->scores, st);
             if (e != cudaSuccess) return cuda_fail(e);
         }
+        cudaStream_t sel_st = st;
+        if (side_select) {
+            if (!c->cs_sel) {
+                if ((e = cudaStreamCreateWithFlags(&c->cs_sel, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+                if ((e = cudaEventCreateWithFlags(&c->ev_scored, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+                if ((e = cudaEventCreateWithFlags(&c->ev_selected, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+            }
+            if ((e = cudaEventRecord(c->ev_scored, st)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaStreamWaitEvent(c->cs_sel, c->ev_scored, 0)) != cudaSuccess) return cuda_fail(e);
+            sel_st = c->cs_sel;
+        }
         {   // ---- Eq. 8
-            PhaseTimer pt(c, st, XSV_PHASE_SELECT);
-            e = xsv_launch_select(c->scores, n_mid, k, T_first, (int)T_c, c->srcmap, c->dscal, st);
+            PhaseTimer pt(c, sel_st, XSV_PHASE_SELECT);
+            e = xsv_launch_select(c->scores, n_mid, k, T_first, (int)T_c, c->srcmap, c->dscal, sel_st);
             if (e != cudaSuccess) return cuda_fail(e);
         }
+        if (side_select && (e = cudaEventRecord(c->ev_selected, c->cs_sel)) != cudaSuccess) return cuda_fail(e);
+    }
+
+    // ---- Eq. 2 / Eq. 12: attention over [cache ; frame]
+    {
+        PhaseTimer pt(c, st, XSV_PHASE_ATTN);
+        e = cudaErrorNotSupported;
+        if (c->attn_impl != XSV_ATTN_MMA)
+            e = xsv_launch_attn_tc5(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, c->attn_ws, c->status,
+                                    0, st);
+        if (e == cudaErrorNotSupported) {
+            if (c->attn_impl == XSV_ATTN_TC5) return XSV_ERR_ARG;
+            e = xsv_launch_attn_mma(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, st);
+        }
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (side_select && (e = cudaStreamWaitEvent(st, c->ev_selected, 0)) != cudaSuccess) return cuda_fail(e);
+
+    if (prune) {
+        const int n_old_new = T_first + k;
+        const int T_new = n_old_new + F;
+        const LayerView& dv = c->bufs[c->spare].view;
         {   // ---- Eq. 9-11 on the new order [first ; kept ; current], written to the spare buffer
             PhaseTimer pt(c, st, XSV_PHASE_QUANT);
             if (c->bits == 16) {
@@ -496,6 +528,9 @@ void xsv_cache_destroy(xsv_cache* c) {
         if (c->ev_done[i]) cudaEventDestroy(c->ev_done[i]);
         if (c->ev_out[i]) cudaEventDestroy(c->ev_out[i]);
     }
+    if (c->cs_sel) cudaStreamDestroy(c->cs_sel);
+    if (c->ev_scored) cudaEventDestroy(c->ev_scored);
+    if (c->ev_selected) cudaEventDestroy(c->ev_selected);
     if (c->cs_in) cudaStreamDestroy(c->cs_in);
     if (c->cs_out) cudaStreamDestroy(c->cs_out);
     for (auto& p : c->pending) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
