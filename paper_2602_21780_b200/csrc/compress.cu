@@ -759,6 +759,16 @@ __device__ __forceinline__ void rq_quant_v_item(const LayerView& dst, const T* _
     }
 }
 
+// The frame's value rows alone (used when the values are handled on another stream than the keys).
+template <typename T, int BITS>
+__global__ void __launch_bounds__(256) quant_v_kernel(LayerView dst, const T* __restrict__ Vf, int H, int F, int n_old_new,
+                                                      long long origin0, int n_vq, int* __restrict__ status) {
+    xsv_dep_release();
+    xsv_dep_sync();
+    const int item = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (item < n_vq) rq_quant_v_item<T, BITS>(dst, Vf, H, F, n_old_new, origin0, status, item, threadIdx.x & 31);
+}
+
 template <typename T, int BITS>
 __global__ void __launch_bounds__(RQ_THREADS, 3) requant_k_kernel(LayerView src, LayerView dst, const T* __restrict__ Kf,
                                                                const T* __restrict__ Vf, int H, int F, int n_old_new,
@@ -1191,13 +1201,14 @@ cudaError_t xsv_launch_select(const float* scores, int n, int k, int T_first, in
 
 cudaError_t xsv_launch_compress(const LayerView& src, const LayerView& dst, const void* Kf, const void* Vf, int dtype,
                                 int H, int F, int n_old_new, int T_new, int T_first, const int* srcmap,
-                                const int* fz_dev, int fz_host, long long origin0, int* status, cudaStream_t st) {
+                                const int* fz_dev, int fz_host, long long origin0, bool with_values, int* status,
+                                cudaStream_t st) {
     const int ngroups = (T_new + XSV_G - 1) / XSV_G;
     const bool same = src.kcodes == dst.kcodes;
     const int g0 = (fz_dev == nullptr && same) ? fz_host : 0;   // in place: skip the frozen prefix
     const int n_items = max(0, ngroups - g0) * H, wpb = RQ_THREADS / 32;
-    const int n_vg = same ? 0 : ((n_old_new + 63) / 64) * H;     // value rows that move
-    const int n_vq = ((F + RQ_VROWS - 1) / RQ_VROWS) * H;        // value rows of the frame
+    const int n_vg = (same || !with_values) ? 0 : ((n_old_new + 63) / 64) * H;     // value rows that move
+    const int n_vq = with_values ? ((F + RQ_VROWS - 1) / RQ_VROWS) * H : 0;        // value rows of the frame
     const int n_all = n_items + n_vg + n_vq;
     if (n_all <= 0) return cudaSuccess;
 #define XSV_RQ(TT, B)                                                                                                \
@@ -1231,6 +1242,43 @@ cudaError_t xsv_launch_compress(const LayerView& src, const LayerView& dst, cons
         }
     }
 #undef XSV_RQ
+    xsv_count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t xsv_launch_values(const LayerView& src, const LayerView& dst, const void* Vf, int dtype, int H, int F,
+                              int n_old_new, int T_first, const int* srcmap, long long origin0, int* status,
+                              cudaStream_t st) {
+    if (src.vcodes != dst.vcodes && n_old_new > 0) {
+        const long long total = (long long)H * n_old_new * (src.rowb / 16);
+        const int grid = (int)((total + 255) / 256);
+        switch (src.rowb) {
+            case 16: xsv_launch_dep(gather_v_kernel<16>, dim3(grid), dim3(256), 0, st, src, dst, H, n_old_new, T_first, srcmap); break;
+            case 32: xsv_launch_dep(gather_v_kernel<32>, dim3(grid), dim3(256), 0, st, src, dst, H, n_old_new, T_first, srcmap); break;
+            case 64: xsv_launch_dep(gather_v_kernel<64>, dim3(grid), dim3(256), 0, st, src, dst, H, n_old_new, T_first, srcmap); break;
+            default: return cudaErrorInvalidValue;
+        }
+        xsv_count_launch();
+    }
+    const int n_vq = ((F + RQ_VROWS - 1) / RQ_VROWS) * H;
+    const int grid = (n_vq + 7) / 8;
+#define XSV_QV(TT, B) xsv_launch_dep(quant_v_kernel<TT, B>, dim3(grid), dim3(256), 0, st, dst, (const TT*)Vf, H, F, n_old_new, origin0, n_vq, status)
+    if (dtype == 0) {
+        switch (dst.bits) {
+            case 2: XSV_QV(__half, 2); break;
+            case 4: XSV_QV(__half, 4); break;
+            case 8: XSV_QV(__half, 8); break;
+            default: return cudaErrorInvalidValue;
+        }
+    } else {
+        switch (dst.bits) {
+            case 2: XSV_QV(__nv_bfloat16, 2); break;
+            case 4: XSV_QV(__nv_bfloat16, 4); break;
+            case 8: XSV_QV(__nv_bfloat16, 8); break;
+            default: return cudaErrorInvalidValue;
+        }
+    }
+#undef XSV_QV
     xsv_count_launch();
     return cudaGetLastError();
 }

@@ -341,7 +341,17 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
             e = xsv_launch_select(c->scores, n_mid, k, T_first, (int)T_c, c->srcmap, c->dscal, sel_st);
             if (e != cudaSuccess) return cuda_fail(e);
         }
-        if (side_select && (e = cudaEventRecord(c->ev_selected, c->cs_sel)) != cudaSuccess) return cuda_fail(e);
+        if (side_select) {
+            // the values need the selection only (kept rows move verbatim, the frame's rows are quantised): they follow
+            // it on its stream, into the spare buffer, and are out of the way when the keys' turn comes
+            if (c->bits < 16) {
+                PhaseTimer pt(c, sel_st, XSV_PHASE_QUANT);
+                e = xsv_launch_values(lv, c->bufs[c->spare].view, V, (int)dtype, H, F, T_first + k, T_first, c->srcmap,
+                                      origin0, c->status, sel_st);
+                if (e != cudaSuccess) return cuda_fail(e);
+            }
+            if ((e = cudaEventRecord(c->ev_selected, c->cs_sel)) != cudaSuccess) return cuda_fail(e);
+        }
     }
 
     // ---- Eq. 2 / Eq. 12: attention over [cache ; frame]
@@ -369,7 +379,7 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
                 e = xsv_launch_raw_update(lv, dv, K, V, H, F, n_old_new, T_first, c->srcmap, origin0, st);
             } else {
                 e = xsv_launch_compress(lv, dv, K, V, (int)dtype, H, F, n_old_new, T_new, T_first, c->srcmap, c->dscal, 0,
-                                        origin0, c->status, st);
+                                        origin0, !side_select, c->status, st);
             }
             if (e != cudaSuccess) return cuda_fail(e);
         }
@@ -385,7 +395,7 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
             e = xsv_launch_raw_update(lv, lv, K, V, H, F, (int)T_c, F, nullptr, origin0, st);
         } else {
             e = xsv_launch_compress(lv, lv, K, V, (int)dtype, H, F, (int)T_c, (int)T, F, nullptr, nullptr,
-                                    (int)(T_c / XSV_G), origin0, c->status, st);
+                                    (int)(T_c / XSV_G), origin0, true, c->status, st);
         }
         if (e != cudaSuccess) return cuda_fail(e);
         c->len[layer] = T;

@@ -35,10 +35,16 @@ cudaError_t xsv_launch_select(const float* scores, int n, int k, int T_first, in
 // Values: kept rows move verbatim (codes, scale, zero-point, origin) to new positions [0, n_old_new) when
 //   dst != src; the frame's rows are quantised per token into [n_old_new, n_old_new + F), with their origins
 //   origin0 + token index.
+//   with_values == false leaves the values to xsv_launch_values.
 cudaError_t xsv_launch_compress(const LayerView& src, const LayerView& dst, const void* Kf, const void* Vf,
                                 int dtype, int H, int F, int n_old_new, int T_new, int T_first,
                                 const int* srcmap, const int* fz_dev, int fz_host, long long origin0,
-                                int* status, cudaStream_t st);
+                                bool with_values, int* status, cudaStream_t st);
+
+// The value part of the above as launches of its own (two small kernels), for a stream other than the keys'.
+cudaError_t xsv_launch_values(const LayerView& src, const LayerView& dst, const void* Vf, int dtype, int H, int F,
+                              int n_old_new, int T_first, const int* srcmap, long long origin0, int* status,
+                              cudaStream_t st);
 
 // bits == 16: gather / append raw 16-bit rows of K and V (no quantisation).
 cudaError_t xsv_launch_raw_update(const LayerView& src, const LayerView& dst, const void* Kf,
