@@ -341,7 +341,10 @@ def main():
             phases[name] = {"avg_ms": per, "algorithmic_bytes": nbytes, "GB/s": nbytes / (per * 1e-3) / 1e9,
                             "frac_of_hbm": nbytes / (per * 1e-3) / 1e9 / peaks["hbm"], "launches_per_step": pn / steps_n}
     phases["attn"] = {"avg_ms": attn_ms / attn_n if attn_n else None}
-    phases["note"] = f"score/select/quant: events around every phase, {n_phase_frames} frames after the timed region"
+    phases["note"] = (f"score/select/quant: events around every phase, {n_phase_frames} frames after the timed region; "
+                      "select and quant run on the library's second stream under the tail of the attention kernel, so "
+                      "their spans start when the scores are ready and include the wait for free multiprocessors: the "
+                      "phases overlap and do not add up to the step")
     cache.destroy()
 
     # ---- end to end: same metric through the C ABI with HOST buffers (copies inside the timed region)

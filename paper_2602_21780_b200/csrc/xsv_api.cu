@@ -342,12 +342,17 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
             if (e != cudaSuccess) return cuda_fail(e);
         }
         if (side_select) {
-            // the values need the selection only (kept rows move verbatim, the frame's rows are quantised): they follow
-            // it on its stream, into the spare buffer, and are out of the way when the keys' turn comes
+            // Eq. 9-11 need the selection only, not the attention output: they follow it on its stream, into the spare
+            // buffer -- first the values (two short kernels: kept rows move verbatim, the frame's rows are quantised),
+            // then the keys -- on the multiprocessors that the attention CTAs leave one by one, and beside the merge
+            // kernel.  The caller's stream waits for them below, so the step ends when all of it has.
             if (c->bits < 16) {
                 PhaseTimer pt(c, sel_st, XSV_PHASE_QUANT);
-                e = xsv_launch_values(lv, c->bufs[c->spare].view, V, (int)dtype, H, F, T_first + k, T_first, c->srcmap,
-                                      origin0, c->status, sel_st);
+                const LayerView& dv = c->bufs[c->spare].view;
+                e = xsv_launch_values(lv, dv, V, (int)dtype, H, F, T_first + k, T_first, c->srcmap, origin0, c->status, sel_st);
+                if (e == cudaSuccess)
+                    e = xsv_launch_compress(lv, dv, K, V, (int)dtype, H, F, T_first + k, T_first + k + F, T_first, c->srcmap,
+                                            c->dscal, 0, origin0, false, c->status, sel_st);
                 if (e != cudaSuccess) return cuda_fail(e);
             }
             if ((e = cudaEventRecord(c->ev_selected, c->cs_sel)) != cudaSuccess) return cuda_fail(e);
@@ -378,8 +383,9 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
             if (c->bits == 16) {
                 e = xsv_launch_raw_update(lv, dv, K, V, H, F, n_old_new, T_first, c->srcmap, origin0, st);
             } else {
-                e = xsv_launch_compress(lv, dv, K, V, (int)dtype, H, F, n_old_new, T_new, T_first, c->srcmap, c->dscal, 0,
-                                        origin0, !side_select, c->status, st);
+                if (!side_select)
+                    e = xsv_launch_compress(lv, dv, K, V, (int)dtype, H, F, n_old_new, T_new, T_first, c->srcmap, c->dscal, 0,
+                                            origin0, true, c->status, st);
             }
             if (e != cudaSuccess) return cuda_fail(e);
         }
