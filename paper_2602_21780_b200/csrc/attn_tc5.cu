@@ -1036,7 +1036,12 @@ int sm_count() {
 }
 
 template <typename T, int BITS>
-cudaError_t launch(const Params& p, cudaStream_t st) {
+cudaError_t launch(const Params& p, bool merge_only, cudaStream_t st) {
+    if (merge_only) {
+        xsv_launch_dep(attn_combine_kernel<T>, dim3(16, p.H * p.npair), dim3(256), 0, st, p);
+        xsv_count_launch(1);
+        return cudaGetLastError();
+    }
     static bool attr_set = false;
     if (!attr_set) {
         cudaError_t e = cudaFuncSetAttribute(attn_tc5_kernel<T, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
@@ -1044,8 +1049,7 @@ cudaError_t launch(const Params& p, cudaStream_t st) {
         attr_set = true;
     }
     xsv_launch_dep(attn_tc5_kernel<T, BITS>, dim3(p.G), dim3(NTHREADS), SMEM_BYTES, st, p);
-    xsv_launch_dep(attn_combine_kernel<T>, dim3(16, p.H * p.npair), dim3(256), 0, st, p);
-    xsv_count_launch(2);
+    xsv_count_launch(1);
     return cudaGetLastError();
 }
 
@@ -1059,8 +1063,10 @@ cudaError_t xsv_launch_wait_selftest(int* status, cudaStream_t st) {
 
 size_t xsv_attn_tc5_workspace_bytes() { return (size_t)sm_count() * 2 * PART_STRIDE * sizeof(float); }
 
-cudaError_t xsv_launch_attn_tc5(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V, void* out,
-                                int dtype, int H, int F, float* workspace, int* status, int spare_sms, cudaStream_t st) {
+namespace {
+cudaError_t launch_tc5(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V, void* out,
+                       int dtype, int H, int F, float* workspace, int* status, int spare_sms, bool merge_only,
+                       cudaStream_t st) {
     if (!workspace) return cudaErrorNotSupported;
     Params p{};
     p.lv = lv; p.Q = Q; p.K = K; p.V = V; p.out = out; p.part = workspace; p.status = status;
@@ -1075,7 +1081,7 @@ cudaError_t xsv_launch_attn_tc5(const LayerView& lv, int T_c, const void* Q, con
     const int sms = sm_count() - spare_sms > 0 ? sm_count() - spare_sms : 1;   // multiprocessors left to another kernel
     p.G = (int)(steps < sms ? steps : sms);
     if (p.G > MAX_PARTS) p.G = MAX_PARTS;
-#define XSV_TC5(TT, B) return launch<TT, B>(p, st)
+#define XSV_TC5(TT, B) return launch<TT, B>(p, merge_only, st)
     if (dtype == 0) {
         switch (lv.bits) {
             case 2: XSV_TC5(__half, 2);
@@ -1093,4 +1099,16 @@ cudaError_t xsv_launch_attn_tc5(const LayerView& lv, int T_c, const void* Q, con
     }
 #undef XSV_TC5
     return cudaErrorInvalidValue;
+}
+}  // namespace
+
+cudaError_t xsv_launch_attn_tc5(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V, void* out,
+                                int dtype, int H, int F, float* workspace, int* status, int spare_sms, cudaStream_t st) {
+    return launch_tc5(lv, T_c, Q, K, V, out, dtype, H, F, workspace, status, spare_sms, false, st);
+}
+
+cudaError_t xsv_launch_attn_tc5_merge(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V,
+                                      void* out, int dtype, int H, int F, float* workspace, int* status,
+                                      int spare_sms, cudaStream_t st) {
+    return launch_tc5(lv, T_c, Q, K, V, out, dtype, H, F, workspace, status, spare_sms, true, st);
 }

@@ -360,16 +360,21 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
     }
 
     // ---- Eq. 2 / Eq. 12: attention over [cache ; frame]
+    bool tc5 = false;
     {
-        PhaseTimer pt(c, st, XSV_PHASE_ATTN);
+        PhaseTimer pt(c, st, XSV_PHASE_ATTN);      // the attention kernel proper; the merge of shared tiles follows
         e = cudaErrorNotSupported;
         if (c->attn_impl != XSV_ATTN_MMA)
-            e = xsv_launch_attn_tc5(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, c->attn_ws, c->status,
-                                    0, st);
+            e = xsv_launch_attn_tc5(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, c->attn_ws, c->status, 0, st);
+        tc5 = (e == cudaSuccess);
         if (e == cudaErrorNotSupported) {
             if (c->attn_impl == XSV_ATTN_TC5) return XSV_ERR_ARG;
             e = xsv_launch_attn_mma(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, st);
         }
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (tc5) {
+        e = xsv_launch_attn_tc5_merge(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, c->attn_ws, c->status, 0, st);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     if (side_select && (e = cudaStreamWaitEvent(st, c->ev_selected, 0)) != cudaSuccess) return cuda_fail(e);

@@ -55,9 +55,10 @@ cudaError_t xsv_launch_raw_update(const LayerView& src, const LayerView& dst, co
 cudaError_t xsv_launch_attn_mma(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V,
                                 void* out, int dtype, int H, int F, cudaStream_t st);
 
-// Same contract; tcgen05 + TMEM kernel (followed by a small kernel that merges
-// the parts of query tiles shared by several CTAs).  `workspace` holds those
-// parts: xsv_attn_tc5_workspace_bytes() bytes of device memory; nullptr returns
+// Same contract; tcgen05 + TMEM kernel, to be followed by xsv_launch_attn_tc5_merge
+// with the same arguments: a small kernel that merges the parts of query tiles
+// shared by several CTAs.  `workspace` holds those parts:
+// xsv_attn_tc5_workspace_bytes() bytes of device memory; nullptr returns
 // cudaErrorNotSupported.  A bounded wait that runs out sets XSV_DEV_TIMEOUT in
 // *status.  spare_sms multiprocessors are left without a CTA (for a kernel that
 // runs beside this one on another stream).
@@ -65,6 +66,9 @@ size_t xsv_attn_tc5_workspace_bytes();
 cudaError_t xsv_launch_attn_tc5(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V,
                                 void* out, int dtype, int H, int F, float* workspace, int* status,
                                 int spare_sms, cudaStream_t st);
+cudaError_t xsv_launch_attn_tc5_merge(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V,
+                                      void* out, int dtype, int H, int F, float* workspace, int* status,
+                                      int spare_sms, cudaStream_t st);
 
 // One small kernel whose only wait can never be satisfied: it must come back after the
 // attention kernel's wait limit with XSV_DEV_TIMEOUT set in *status (device int).
