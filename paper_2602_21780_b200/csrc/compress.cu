@@ -714,9 +714,9 @@ __device__ __forceinline__ void rq_gather_v_item(const LayerView& src, const Lay
     }
 }
 
-// Eq. 9-11 for the frame's values: one warp per (16 tokens, head); a row of 64 channels at a time, two channels per
+// Eq. 9-11 for the frame's values: one warp per (4 tokens, head); a row of 64 channels at a time, two channels per
 // lane, shuffle reductions for min / max.
-constexpr int RQ_VROWS = 16;
+constexpr int RQ_VROWS = 4;
 template <typename T, int BITS>
 __device__ __forceinline__ void rq_quant_v_item(const LayerView& dst, const T* __restrict__ Vf, int H, int F,
                                                 int n_old_new, long long origin0, int* __restrict__ status, int item,
