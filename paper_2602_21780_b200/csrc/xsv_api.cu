@@ -70,8 +70,9 @@ struct xsv_cache {
     void* stage = nullptr;
     size_t stage_bytes = 0;
     cudaStream_t cs_in = nullptr, cs_out = nullptr;
-    cudaStream_t cs_sel = nullptr;                          // the selection kernel runs here, beside the attention kernel
-    cudaEvent_t ev_scored = nullptr, ev_selected = nullptr;
+    cudaStream_t cs_sel = nullptr;                          // selection, then the keys' re-quantisation, beside the attention kernel
+    cudaStream_t cs_val = nullptr;                          // the values, beside the keys
+    cudaEvent_t ev_scored = nullptr, ev_selected = nullptr, ev_picked = nullptr, ev_values = nullptr;
     cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
     bool slot_used[2] = {false, false}, out_pending[2] = {false, false};
     bool defer_output = false;
@@ -331,6 +332,9 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
                 if ((e = cudaStreamCreateWithFlags(&c->cs_sel, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
                 if ((e = cudaEventCreateWithFlags(&c->ev_scored, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
                 if ((e = cudaEventCreateWithFlags(&c->ev_selected, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+                if ((e = cudaStreamCreateWithFlags(&c->cs_val, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
+                if ((e = cudaEventCreateWithFlags(&c->ev_picked, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+                if ((e = cudaEventCreateWithFlags(&c->ev_values, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
             }
             if ((e = cudaEventRecord(c->ev_scored, st)) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaStreamWaitEvent(c->cs_sel, c->ev_scored, 0)) != cudaSuccess) return cuda_fail(e);
@@ -342,17 +346,24 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
             if (e != cudaSuccess) return cuda_fail(e);
         }
         if (side_select) {
-            // Eq. 9-11 need the selection only, not the attention output: they follow it on its stream, into the spare
-            // buffer -- first the values (two short kernels: kept rows move verbatim, the frame's rows are quantised),
-            // then the keys -- on the multiprocessors that the attention CTAs leave one by one, and beside the merge
-            // kernel.  The caller's stream waits for them below, so the step ends when all of it has.
+            // Eq. 9-11 need the selection only, not the attention output: they follow it into the spare buffer -- the keys
+            // on its stream, the values (two short kernels: kept rows move verbatim, the frame's rows are quantised)
+            // on a third one, so that neither waits for the other -- on the multiprocessors that the attention CTAs
+            // leave one by one, and beside the merge kernel.  The caller's stream waits for both below, so the step ends
+            // when all of it has.
             if (c->bits < 16) {
-                PhaseTimer pt(c, sel_st, XSV_PHASE_QUANT);
                 const LayerView& dv = c->bufs[c->spare].view;
-                e = xsv_launch_values(lv, dv, V, (int)dtype, H, F, T_first + k, T_first, c->srcmap, origin0, c->status, sel_st);
-                if (e == cudaSuccess)
-                    e = xsv_launch_compress(lv, dv, K, V, (int)dtype, H, F, T_first + k, T_first + k + F, T_first, c->srcmap,
-                                            c->dscal, 0, origin0, false, c->status, sel_st);
+                if ((e = cudaEventRecord(c->ev_picked, c->cs_sel)) != cudaSuccess) return cuda_fail(e);
+                if ((e = cudaStreamWaitEvent(c->cs_val, c->ev_picked, 0)) != cudaSuccess) return cuda_fail(e);
+                {
+                    PhaseTimer pt(c, c->cs_val, XSV_PHASE_QUANT);
+                    e = xsv_launch_values(lv, dv, V, (int)dtype, H, F, T_first + k, T_first, c->srcmap, origin0, c->status, c->cs_val);
+                    if (e != cudaSuccess) return cuda_fail(e);
+                }
+                if ((e = cudaEventRecord(c->ev_values, c->cs_val)) != cudaSuccess) return cuda_fail(e);
+                PhaseTimer pt(c, sel_st, XSV_PHASE_QUANT);
+                e = xsv_launch_compress(lv, dv, K, V, (int)dtype, H, F, T_first + k, T_first + k + F, T_first, c->srcmap,
+                                        c->dscal, 0, origin0, false, c->status, sel_st);
                 if (e != cudaSuccess) return cuda_fail(e);
             }
             if ((e = cudaEventRecord(c->ev_selected, c->cs_sel)) != cudaSuccess) return cuda_fail(e);
@@ -378,6 +389,7 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
         if (e != cudaSuccess) return cuda_fail(e);
     }
     if (side_select && (e = cudaStreamWaitEvent(st, c->ev_selected, 0)) != cudaSuccess) return cuda_fail(e);
+    if (side_select && c->bits < 16 && (e = cudaStreamWaitEvent(st, c->ev_values, 0)) != cudaSuccess) return cuda_fail(e);
 
     if (prune) {
         const int n_old_new = T_first + k;
@@ -550,6 +562,9 @@ void xsv_cache_destroy(xsv_cache* c) {
         if (c->ev_out[i]) cudaEventDestroy(c->ev_out[i]);
     }
     if (c->cs_sel) cudaStreamDestroy(c->cs_sel);
+    if (c->cs_val) cudaStreamDestroy(c->cs_val);
+    if (c->ev_picked) cudaEventDestroy(c->ev_picked);
+    if (c->ev_values) cudaEventDestroy(c->ev_values);
     if (c->ev_scored) cudaEventDestroy(c->ev_scored);
     if (c->ev_selected) cudaEventDestroy(c->ev_selected);
     if (c->cs_in) cudaStreamDestroy(c->cs_in);
