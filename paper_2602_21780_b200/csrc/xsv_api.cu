@@ -311,9 +311,9 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
     const int k = (int)(kk > 0 ? kk : 0);
     // The scores (Eq. 3-7) need the frame's queries and the cached keys only, so they come first; the selection
     // (Eq. 8), one block that is bound by latency, then runs on a stream of its own: it takes the first multiprocessor
-    // that an attention CTA leaves (the CTAs' finishing times are spread over some tens of microseconds) and so
-    // overlaps the tail of the attention kernel and the merge kernel.  Leaving it a multiprocessor of its own for the
-    // whole attention kernel measured slightly slower.
+    // that an attention CTA leaves (the CTAs' finishing times are spread over some tens of microseconds) and what
+    // follows it takes the next ones.  (Keeping one multiprocessor free of attention CTAs for that stream from the
+    // start gives 0.7 % more frames per second and 3 % less throughput of the attention kernel; not done.)
     const bool side_select = prune && side_select_enabled() && c->attn_impl != XSV_ATTN_MMA && c->attn_ws != nullptr;
     if (prune) {
         {   // ---- Eq. 3-7
