@@ -108,6 +108,14 @@ xsv_status xsv_cache_set_attn_impl(xsv_cache* c, xsv_attn_impl impl);
  *   stream  : cudaStream_t (as void*); NULL is the default stream.
  * Afterwards the layer's cache holds [first frame ; kept middle ; this frame],
  * quantised, of length min-closed-form (see xsv_cache_len).
+ * Everything is enqueued; nothing synchronises with the host.  A step that
+ * prunes runs its selection and re-quantisation kernels (Eq. 8-11, which need
+ * the scores but not the attention output) on streams the cache owns, beside
+ * the end of the attention kernel, and `stream` waits for them before the step
+ * ends: in the order of `stream` the step is complete -- `out` written, the
+ * cache updated, Q, K, V free to be reused -- when the call's work has run.
+ * All steps of one cache must be ordered with respect to each other (one
+ * stream, or streams ordered by events).
  */
 xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const void* V,
                     int n_tokens, xsv_dtype dtype, void* out, void* stream);
