@@ -258,6 +258,9 @@ def main():
     def make_cache():
         c = binding.Cache(LAYERS, H, D, L_MAX, BITS)
         c.set_attn_impl(impl)
+        # the inputs of a frame stay untouched while the next layers run, so the end of a layer-step's selection and
+        # re-quantisation may overlap the next layer-step (see xsv_cache_set_deferred_join); joined before the clock stops
+        c.set_deferred_join(True)
         return c
 
     ptrs = [[(q.data_ptr(), k.data_ptr(), v.data_ptr()) for (q, k, v) in per] for per in frames]
@@ -291,6 +294,7 @@ def main():
     e0.record(stream)
     for f in range(args.steps):
         frame_step(cache, PREFILL + args.warmup + f)
+    cache.join(stream)
     e1.record(stream)
     torch.cuda.synchronize()
     if world > 1:
@@ -394,7 +398,7 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": "frames/s", "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": WORKLOAD, "prefill_frames": PREFILL, "attn_impl": args.attn,
+                "config": {"workload": WORKLOAD, "prefill_frames": PREFILL, "attn_impl": args.attn, "deferred_join": True,
                            "l2": "each step touches 203 MB of fresh inputs + 675 MB of cache (> 126 MB L2); no flush",
                            "multi_gpu": "replicas only"},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu,

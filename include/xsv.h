@@ -121,6 +121,22 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
                     int n_tokens, xsv_dtype dtype, void* out, void* stream);
 
 /*
+ * Deferred join (off by default).  With on != 0, `stream` does not wait at the
+ * end of a pruning step for the selection and re-quantisation kernels on the
+ * cache's own streams: they finish under whatever `stream` runs next (the next
+ * layer's score kernels and the start of its attention kernel).  The library
+ * keeps its own state ordered -- a layer's next step waits for that layer's
+ * outstanding work, shared scratch is handed over through events, the host-side
+ * queries synchronise every stream -- but two things become the caller's:
+ * K and V of a step must stay unchanged until `stream` has passed the next
+ * xsv_step on the same layer or an xsv_cache_join, and so must not be freed or
+ * overwritten earlier; `out` is complete in `stream` order as always.
+ * xsv_cache_join makes `stream` wait for all outstanding side-stream work.
+ */
+xsv_status xsv_cache_set_deferred_join(xsv_cache* c, int on);
+xsv_status xsv_cache_join(xsv_cache* c, void* stream);
+
+/*
  * Same step with HOST buffers (pinned host memory makes the copies asynchronous).
  * The inputs are copied to device staging owned by the cache on an internal
  * stream, so that the copy of one call overlaps the kernels of the previous

@@ -35,6 +35,8 @@ SYMBOLS = {
     "xsv_cache_len": (_ll, [_vp, _i]),
     "xsv_cache_frames": (_ll, [_vp, _i]),
     "xsv_cache_export_layer": (_i, [_vp, _i] + [_vp] * 9 + [_vp]),
+    "xsv_cache_set_deferred_join": (_i, [_vp, _i]),
+    "xsv_cache_join": (_i, [_vp, _vp]),
     "xsv_quantization_mse": (_i, [_vp, _i, _ll, _i, _i, _i, C.POINTER(C.c_double), _vp]),
     "xsv_cache_import_layer": (_i, [_vp, _i, _ll, _ll, _i, _i] + [_vp] * 9 + [_vp]),
     "xsv_last_scores": (_i, [_vp, _vp, _ll, C.POINTER(_ll), _vp]),
@@ -167,6 +169,12 @@ class Cache:
         _check(self._lib.xsv_cache_export_layer(self._h, layer, *args, _stream_ptr(stream)),
                "xsv_cache_export_layer")
         return st
+
+    def set_deferred_join(self, on):
+        _check(self._lib.xsv_cache_set_deferred_join(self._h, int(on)), "xsv_cache_set_deferred_join")
+
+    def join(self, stream=None):
+        _check(self._lib.xsv_cache_join(self._h, _stream_ptr(stream)), "xsv_cache_join")
 
     def import_layer(self, layer, st, frames_done, frame_tokens, dtype_code, stream=None):
         """Load a state dict as returned by export_layer (see xsv_cache_import_layer)."""

@@ -73,6 +73,10 @@ struct xsv_cache {
     cudaStream_t cs_sel = nullptr;                          // selection, then the keys' re-quantisation, beside the attention kernel
     cudaStream_t cs_val = nullptr;                          // the values, beside the keys
     cudaEvent_t ev_scored = nullptr, ev_selected = nullptr, ev_picked = nullptr, ev_values = nullptr;
+    bool defer_join = false;                                // the caller's stream does not wait for the side streams at the end of a step
+    bool select_outstanding = false;                        // a selection has been enqueued that the caller's stream has not waited for
+    std::vector<cudaEvent_t> ev_keys_of, ev_vals_of;        // per layer: end of its side-stream work (deferred join)
+    std::vector<char> side_pending;                         // per layer: the caller's stream has not yet waited for those
     cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
     bool slot_used[2] = {false, false}, out_pending[2] = {false, false};
     bool defer_output = false;
@@ -177,6 +181,16 @@ cudaEvent_t get_event(xsv_cache* c) {
 bool side_select_enabled() {
     static const bool on = (getenv("XSV_NO_SIDE_SELECT") == nullptr);
     return on;
+}
+
+// Host-side wait for the cache's own streams (after the caller's stream has been synchronised).
+cudaError_t sync_side_streams(xsv_cache* c) {
+    cudaError_t e = cudaSuccess;
+    if (c->cs_sel) e = cudaStreamSynchronize(c->cs_sel);
+    if (e == cudaSuccess && c->cs_val) e = cudaStreamSynchronize(c->cs_val);
+    for (auto& p : c->side_pending) p = 0;
+    c->select_outstanding = false;
+    return e;
 }
 
 struct PhaseTimer {
@@ -315,6 +329,17 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
     // follows it takes the next ones.  (Keeping one multiprocessor free of attention CTAs for that stream from the
     // start gives 0.7 % more frames per second and 3 % less throughput of the attention kernel; not done.)
     const bool side_select = prune && side_select_enabled() && c->attn_impl != XSV_ATTN_MMA && c->attn_ws != nullptr;
+    // Deferred join: side-stream work of earlier steps may still be running.  This layer's own must have ended before
+    // its cache is read, and the last selection before the score buffer is rewritten.
+    if (!c->side_pending.empty() && c->side_pending[layer]) {
+        if ((e = cudaStreamWaitEvent(st, c->ev_keys_of[layer], 0)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamWaitEvent(st, c->ev_vals_of[layer], 0)) != cudaSuccess) return cuda_fail(e);
+        c->side_pending[layer] = 0;
+    }
+    if (c->select_outstanding) {
+        if ((e = cudaStreamWaitEvent(st, c->ev_picked, 0)) != cudaSuccess) return cuda_fail(e);
+        c->select_outstanding = false;
+    }
     if (prune) {
         {   // ---- Eq. 3-7
             PhaseTimer pt(c, st, XSV_PHASE_SCORE);
@@ -335,7 +360,16 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
                 if ((e = cudaStreamCreateWithFlags(&c->cs_val, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
                 if ((e = cudaEventCreateWithFlags(&c->ev_picked, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
                 if ((e = cudaEventCreateWithFlags(&c->ev_values, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+                c->ev_keys_of.assign(c->layers, nullptr);
+                c->ev_vals_of.assign(c->layers, nullptr);
+                c->side_pending.assign(c->layers, 0);
+                for (int l = 0; l < c->layers; ++l) {
+                    if ((e = cudaEventCreateWithFlags(&c->ev_keys_of[l], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+                    if ((e = cudaEventCreateWithFlags(&c->ev_vals_of[l], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
+                }
             }
+            // the new selection overwrites the kept-position map that the values of the previous step may still read
+            if (c->defer_join && (e = cudaStreamWaitEvent(c->cs_sel, c->ev_values, 0)) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaEventRecord(c->ev_scored, st)) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaStreamWaitEvent(c->cs_sel, c->ev_scored, 0)) != cudaSuccess) return cuda_fail(e);
             sel_st = c->cs_sel;
@@ -388,8 +422,18 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
         e = xsv_launch_attn_tc5_merge(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, c->attn_ws, c->status, 0, st);
         if (e != cudaSuccess) return cuda_fail(e);
     }
-    if (side_select && (e = cudaStreamWaitEvent(st, c->ev_selected, 0)) != cudaSuccess) return cuda_fail(e);
-    if (side_select && c->bits < 16 && (e = cudaStreamWaitEvent(st, c->ev_values, 0)) != cudaSuccess) return cuda_fail(e);
+    const bool deferred = side_select && c->defer_join && c->bits < 16;
+    if (deferred) {
+        // the caller's stream goes on; it waits for this layer's side-stream work when the layer is stepped again
+        // (or in xsv_cache_join)
+        if ((e = cudaEventRecord(c->ev_keys_of[layer], c->cs_sel)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventRecord(c->ev_vals_of[layer], c->cs_val)) != cudaSuccess) return cuda_fail(e);
+        c->side_pending[layer] = 1;
+        c->select_outstanding = true;
+    } else {
+        if (side_select && (e = cudaStreamWaitEvent(st, c->ev_selected, 0)) != cudaSuccess) return cuda_fail(e);
+        if (side_select && c->bits < 16 && (e = cudaStreamWaitEvent(st, c->ev_values, 0)) != cudaSuccess) return cuda_fail(e);
+    }
 
     if (prune) {
         const int n_old_new = T_first + k;
@@ -425,6 +469,29 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
         c->last_scores_n = 0;
     }
     c->frames[layer] = t;
+    return XSV_OK;
+}
+
+xsv_status xsv_cache_set_deferred_join(xsv_cache* c, int on) {
+    if (!c) return XSV_ERR_ARG;
+    c->defer_join = on != 0;
+    return XSV_OK;
+}
+
+xsv_status xsv_cache_join(xsv_cache* c, void* stream) {
+    if (!c) return XSV_ERR_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e;
+    for (size_t l = 0; l < c->side_pending.size(); ++l) {
+        if (!c->side_pending[l]) continue;
+        if ((e = cudaStreamWaitEvent(st, c->ev_keys_of[l], 0)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamWaitEvent(st, c->ev_vals_of[l], 0)) != cudaSuccess) return cuda_fail(e);
+        c->side_pending[l] = 0;
+    }
+    if (c->select_outstanding) {
+        if ((e = cudaStreamWaitEvent(st, c->ev_picked, 0)) != cudaSuccess) return cuda_fail(e);
+        c->select_outstanding = false;
+    }
     return XSV_OK;
 }
 
@@ -468,6 +535,7 @@ xsv_status xsv_step_host(xsv_cache* c, int layer, const void* Qh, const void* Kh
     }
     xsv_status r = xsv_step(c, layer, s, s + nb, s + 2 * nb, n_tokens, dtype, s + 3 * nb, stream);
     if (r != XSV_OK) return r;
+    if ((r = xsv_cache_join(c, stream)) != XSV_OK) return r;   // the staged inputs are reused: the step must have ended
     ++c->host_calls;
     c->slot_used[slot] = true;
     if ((e = cudaEventRecord(c->ev_done[slot], st)) != cudaSuccess) return cuda_fail(e);
@@ -561,6 +629,8 @@ void xsv_cache_destroy(xsv_cache* c) {
         if (c->ev_done[i]) cudaEventDestroy(c->ev_done[i]);
         if (c->ev_out[i]) cudaEventDestroy(c->ev_out[i]);
     }
+    for (cudaEvent_t ev : c->ev_keys_of) if (ev) cudaEventDestroy(ev);
+    for (cudaEvent_t ev : c->ev_vals_of) if (ev) cudaEventDestroy(ev);
     if (c->cs_sel) cudaStreamDestroy(c->cs_sel);
     if (c->cs_val) cudaStreamDestroy(c->cs_val);
     if (c->ev_picked) cudaEventDestroy(c->ev_picked);
@@ -589,7 +659,7 @@ xsv_status xsv_cache_export_layer(xsv_cache* c, int layer, unsigned char* k_code
                                   unsigned short* k_raw, unsigned short* v_raw, void* stream) {
     if (!c || layer < 0 || layer >= c->layers) return XSV_ERR_ARG;
     cudaStream_t st = (cudaStream_t)stream;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return XSV_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess || sync_side_streams(c) != cudaSuccess) return XSV_ERR_CUDA;
     const long long T = c->len[layer];
     if (T == 0 || !c->allocated) return XSV_OK;
     const LayerView& lv = c->bufs[c->buf_of_layer[layer]].view;
@@ -647,7 +717,7 @@ xsv_status xsv_cache_import_layer(xsv_cache* c, int layer, long long n_cached, l
         if (s != XSV_OK) { c->F = 0; return s; }
     }
     if (n_cached > c->cap) return XSV_ERR_CAPACITY;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return XSV_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess || sync_side_streams(c) != cudaSuccess) return XSV_ERR_CUDA;
     const LayerView& lv = c->bufs[c->buf_of_layer[layer]].view;
     const int H = c->H, d = c->d, rowb = lv.rowb, bits = c->bits;
     const long long T = n_cached, groups = (T + XSV_G - 1) / XSV_G;
@@ -698,7 +768,7 @@ xsv_status xsv_last_scores(xsv_cache* c, float* scores_host, long long cap, long
     *n = c->last_scores_n;
     if (c->last_scores_n == 0) return XSV_OK;
     if (!scores_host || cap < c->last_scores_n) return XSV_ERR_ARG;
-    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return XSV_ERR_CUDA;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess || sync_side_streams(c) != cudaSuccess) return XSV_ERR_CUDA;
     if (cudaMemcpy(scores_host, c->scores, (size_t)c->last_scores_n * 4, cudaMemcpyDeviceToHost) != cudaSuccess) return XSV_ERR_CUDA;
     return XSV_OK;
 }
@@ -706,7 +776,7 @@ xsv_status xsv_last_scores(xsv_cache* c, float* scores_host, long long cap, long
 xsv_status xsv_cache_status(xsv_cache* c, void* stream) {
     if (!c) return XSV_ERR_ARG;
     if (!c->allocated) return XSV_OK;
-    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return XSV_ERR_CUDA;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess || sync_side_streams(c) != cudaSuccess) return XSV_ERR_CUDA;
     int w = 0;
     if (cudaMemcpy(&w, c->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return XSV_ERR_CUDA;
     if (w & XSV_DEV_TIMEOUT) return XSV_ERR_TIMEOUT;

@@ -63,12 +63,13 @@ def compare_states(st, ref, bits, tag):
 
 
 def run_stream(stream, frames, L_max, bits, check_steps=None, impl=binding.ATTN_AUTO, n_special=5, g=16,
-               frame_fn=None, max_cache_tokens=-1, layers=1, layer=0):
+               frame_fn=None, max_cache_tokens=-1, layers=1, layer=0, deferred_join=False):
     """Run `frames` steps on the GPU; verify the steps in check_steps (0-based; None = all).
     Returns a dict of the worst errors seen."""
     H, d, F, dtype = stream.H, stream.d, stream.F, stream.dtype
     cache = binding.Cache(layers, H, d, L_max, bits)
     cache.set_attn_impl(impl)
+    cache.set_deferred_join(deferred_join)
     if (n_special, g) != (5, 16) or max_cache_tokens >= 0:
         cache.set_options(n_special=n_special, pool_group=g, max_cache_tokens=max_cache_tokens)
     ref = orc.LayerCache(H, d, L_max, bits, n_special=n_special, g=g)

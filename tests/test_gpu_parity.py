@@ -108,6 +108,34 @@ def test_quantization_mse_matches_oracle(dtype):
                 assert got == pytest.approx(want, rel=1e-9), (name, bits, gran)
 
 
+def test_deferred_join_parity_and_equality():
+    # with the join deferred the side streams of one layer-step run under the next one's kernels: same results
+    st = synth.Stream(H=4, d=64, F=261, dtype="fp16", layer=13)
+    w = run_stream(st, 9, 1044, 4, layers=3, layer=1, deferred_join=True)
+    assert w["pruned_steps"] >= 4
+    frames = [tuple(torch.from_numpy(x).to("cuda:0", torch.float16).contiguous() for x in st.frame(t)) for t in range(10)]
+    outs, states = [], []
+    for deferred in (False, True):
+        c = binding.Cache(3, 4, 64, 1044, 4)
+        c.set_deferred_join(deferred)
+        o = [[torch.empty_like(frames[0][0]) for _ in range(3)] for _ in range(10)]
+        for t in range(10):
+            for l in range(3):
+                c.step(l, *frames[t], o[t][l])
+        c.join()
+        torch.cuda.synchronize()
+        outs.append(o)
+        states.append([c.export_layer(l) for l in range(3)])
+        assert c.status() == 0
+        c.destroy()
+    for t in range(10):
+        for l in range(3):
+            assert torch.equal(outs[0][t][l], outs[1][t][l])
+    for l in range(3):
+        for key in states[0][l]:
+            assert np.array_equal(states[0][l][key], states[1][l][key])
+
+
 def test_pooling_options_and_multi_layer():
     st = synth.Stream(H=4, d=64, F=37, dtype="fp16", layer=7)
     run_stream(st, 6, 100, 4, n_special=1, g=4, layers=3, layer=2)
