@@ -79,6 +79,7 @@ struct xsv_cache {
     std::vector<char> side_pending;                         // per layer: the caller's stream has not yet waited for those
     cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
     bool slot_used[2] = {false, false}, out_pending[2] = {false, false};
+    int slot_layer[2] = {0, 0};                             // the layer whose step last read the slot
     bool defer_output = false;
     unsigned long long host_calls = 0;
 
@@ -524,6 +525,11 @@ xsv_status xsv_step_host(xsv_cache* c, int layer, const void* Qh, const void* Kh
     const int slot = (int)(c->host_calls & 1ull);
     uint8_t* s = (uint8_t*)c->stage + (size_t)slot * 4 * nb;
     if (c->slot_used[slot] && (e = cudaStreamWaitEvent(c->cs_in, c->ev_done[slot], 0)) != cudaSuccess) return cuda_fail(e);
+    if (c->slot_used[slot] && !c->side_pending.empty() && c->side_pending[c->slot_layer[slot]]) {
+        // deferred join: that step's side-stream kernels may still be reading the staged K and V
+        if ((e = cudaStreamWaitEvent(c->cs_in, c->ev_keys_of[c->slot_layer[slot]], 0)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamWaitEvent(c->cs_in, c->ev_vals_of[c->slot_layer[slot]], 0)) != cudaSuccess) return cuda_fail(e);
+    }
     if ((e = cudaMemcpyAsync(s, Qh, nb, cudaMemcpyHostToDevice, c->cs_in)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaMemcpyAsync(s + nb, Kh, nb, cudaMemcpyHostToDevice, c->cs_in)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaMemcpyAsync(s + 2 * nb, Vh, nb, cudaMemcpyHostToDevice, c->cs_in)) != cudaSuccess) return cuda_fail(e);
@@ -535,9 +541,9 @@ xsv_status xsv_step_host(xsv_cache* c, int layer, const void* Qh, const void* Kh
     }
     xsv_status r = xsv_step(c, layer, s, s + nb, s + 2 * nb, n_tokens, dtype, s + 3 * nb, stream);
     if (r != XSV_OK) return r;
-    if ((r = xsv_cache_join(c, stream)) != XSV_OK) return r;   // the staged inputs are reused: the step must have ended
     ++c->host_calls;
     c->slot_used[slot] = true;
+    c->slot_layer[slot] = layer;
     if ((e = cudaEventRecord(c->ev_done[slot], st)) != cudaSuccess) return cuda_fail(e);
     if (!c->defer_output) {
         if ((e = cudaMemcpyAsync(out_h, s + 3 * nb, nb, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);

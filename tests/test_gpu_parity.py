@@ -218,12 +218,13 @@ def test_api_errors_and_bytes_constant():
     c.destroy()
 
 
-@pytest.mark.parametrize("defer", [False, True])
-def test_host_step_matches_device_step(defer):
+@pytest.mark.parametrize("defer,deferred_join", [(False, False), (True, False), (True, True)])
+def test_host_step_matches_device_step(defer, deferred_join):
     st = synth.Stream(H=4, d=64, F=90, dtype="bf16", layer=8)
     a = binding.Cache(1, 4, 64, 300, 4)
     b = binding.Cache(1, 4, 64, 300, 4)
     a.set_host_pipelining(defer)
+    a.set_deferred_join(deferred_join)
     hosts, devs = [], []
     for t in range(7):
         q, k, v = (torch.from_numpy(x).to(torch.bfloat16) for x in st.frame(t))
