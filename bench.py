@@ -3,7 +3,7 @@
 
 A "step" is one frame through the whole hot path for all 24 layers: fused
 dequant + attention, importance scores, top-k prune, quantise + pack
-(BASELINE config 2: 16 heads x 64, 1374 tokens/frame, budget 21984 tokens per
+(configuration 2: 16 heads x 64, 1374 tokens/frame, budget 21984 tokens per
 layer, 4-bit KV, bf16), in steady state (the cache is filled to its budget by
 untimed prefill frames first).  Prints ONE JSON line.
 

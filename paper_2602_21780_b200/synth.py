@@ -109,7 +109,7 @@ class Stream:
                 round_to_dtype(v, self.dtype))
 
 
-# The five BASELINE configurations (shapes, budgets, bit widths).
+# The five workload configurations (shapes, budgets, bit widths).
 CONFIGS = {
     0: dict(H=16, d=64, F=261, dtype="fp16", frames=8, L_max=1044, bits=4, layers=1),
     1: dict(H=16, d=64, F=1374, dtype="bf16", frames=64, L_max=21984, bits=4, layers=1),
