@@ -994,17 +994,43 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const Params p) {
     const int grow = mp * 2 * BM + row;
     if (grow >= p.F) return;
     float M = -INFINITY;
-    for (int i = 0; i < n; ++i)
-        M = fmaxf(M, reinterpret_cast<const float2*>(p.part + (size_t)s_slot[i] * PART_STRIDE + 256 * 64)[row].x);
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     float L = 0.f;
-    for (int i = 0; i < n; ++i) {
-        const float* part = p.part + (size_t)s_slot[i] * PART_STRIDE;
-        const float2 ml = reinterpret_cast<const float2*>(part + 256 * 64)[row];
-        const float w = exp2f(ml.x - M);
-        L += ml.y * w;
-        const float4 v = reinterpret_cast<const float4*>(part + (size_t)row * 64)[c4];
-        acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+    if (n <= 4) {
+        // the usual case: every load of every part is issued before the first use (one round trip to memory)
+        float2 ml[4];
+        float4 v[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            ml[i] = make_float2(-INFINITY, 0.f);
+            v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (i < n) {
+                const float* part = p.part + (size_t)s_slot[i] * PART_STRIDE;
+                ml[i] = reinterpret_cast<const float2*>(part + 256 * 64)[row];
+                v[i] = reinterpret_cast<const float4*>(part + (size_t)row * 64)[c4];
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) M = fmaxf(M, ml[i].x);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (i < n) {
+                const float w = exp2f(ml[i].x - M);
+                L += ml[i].y * w;
+                acc.x += v[i].x * w; acc.y += v[i].y * w; acc.z += v[i].z * w; acc.w += v[i].w * w;
+            }
+        }
+    } else {
+        for (int i = 0; i < n; ++i)
+            M = fmaxf(M, reinterpret_cast<const float2*>(p.part + (size_t)s_slot[i] * PART_STRIDE + 256 * 64)[row].x);
+        for (int i = 0; i < n; ++i) {
+            const float* part = p.part + (size_t)s_slot[i] * PART_STRIDE;
+            const float2 ml = reinterpret_cast<const float2*>(part + 256 * 64)[row];
+            const float w = exp2f(ml.x - M);
+            L += ml.y * w;
+            const float4 v = reinterpret_cast<const float4*>(part + (size_t)row * 64)[c4];
+            acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+        }
     }
     const float inv = 1.f / L;
     uint2* dst = reinterpret_cast<uint2*>(reinterpret_cast<T*>(p.out) + ((size_t)h * p.F + grow) * XSV_D) + c4;
