@@ -282,7 +282,9 @@ def main():
     assert cache.len(0) == L_MAX
     bytes_before = cache.bytes()
 
-    cache.set_profiling(2)                 # events around the attention kernel only: its live duration for the roofline
+    # events around every seventh attention kernel (a sample that walks through the layers): its live duration for the
+    # roofline; a pair of events costs the stream a few microseconds, around every launch they took 3-5 % off the step
+    cache.set_profiling(3)
     cache.profile_read(reset=True)
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -321,7 +323,7 @@ def main():
     # ---- roofline of the dominant kernel (attention), live CUDA-event durations
     peaks = measured_peaks()
     attn_ms, attn_launches = prof["attn"]
-    attn_n = args.steps * LAYERS                      # attention launches its main kernel once per layer-step
+    attn_n = attn_launches                            # the timed sample: one attention kernel per timed phase
     T_all = L_MAX + F
     flops = 4.0 * F * T_all * D * H
     achieved = flops / (attn_ms / attn_n * 1e-3) / 1e12 if attn_n else None
@@ -329,6 +331,7 @@ def main():
                 "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"] if achieved else None,
                 "traffic": None if sweep else attn_traffic_bytes(), "peak_source": peaks["source"],
                 "flops_per_launch": flops, "avg_launch_ms": attn_ms / attn_n if attn_n else None,
+                "launches_timed": attn_n, "launches_total": args.steps * LAYERS,
                 "kernels_per_launch": attn_launches / attn_n if attn_n else None}
     # the bandwidth-bound phases: algorithmic bytes per layer-step / live duration
     k_keep = L_MAX - 2 * F

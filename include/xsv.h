@@ -281,7 +281,9 @@ xsv_status xsv_cache_status(xsv_cache* c, void* stream);
 /* Per-phase CUDA-event timing.  on = 1: every step records events around each
  * phase on the step's stream; on = 2: around the attention phase only (each
  * pair of events costs the stream a few microseconds, which matters when the
- * whole step is being timed as well); on = 0: none.  xsv_cache_profile_read
+ * whole step is being timed as well); on = 3: around every seventh attention
+ * phase (a sample that walks through the layers of a 24-layer stack); on = 0:
+ * none.  xsv_cache_profile_read
  * synchronises the recorded events, adds their durations to per-phase totals,
  * and returns the totals (milliseconds) and launch counts accumulated since
  * the last reset. */

@@ -85,7 +85,8 @@ struct xsv_cache {
 
     size_t bytes = 0;
 
-    int profiling = 0;          // 0 off, 1 events around every phase, 2 around the attention phase only
+    int profiling = 0;          // 0 off, 1 events around every phase, 2 around the attention phase only, 3 around every 7th one
+    unsigned long long attn_calls = 0;
     std::vector<PendingEvent> pending;
     std::vector<cudaEvent_t> free_events;
     double prof_ms[XSV_PHASE_COUNT] = {0, 0, 0, 0};
@@ -203,7 +204,8 @@ struct PhaseTimer {
     bool on;
     PhaseTimer(xsv_cache* c_, cudaStream_t st_, int phase_) : c(c_), st(st_), phase(phase_) {
         launches0 = g_launches.load(std::memory_order_relaxed);
-        on = c->profiling == 1 || (c->profiling == 2 && phase == XSV_PHASE_ATTN);
+        on = c->profiling == 1 || (c->profiling == 2 && phase == XSV_PHASE_ATTN) ||
+             (c->profiling == 3 && phase == XSV_PHASE_ATTN && (c->attn_calls++ % 7ull) == 0ull);
         if (on) {
             a = get_event(c);
             b = get_event(c);
@@ -792,7 +794,7 @@ xsv_status xsv_cache_status(xsv_cache* c, void* stream) {
 
 xsv_status xsv_cache_set_profiling(xsv_cache* c, int on) {
     if (!c) return XSV_ERR_ARG;
-    if (on < 0 || on > 2) return XSV_ERR_ARG;
+    if (on < 0 || on > 3) return XSV_ERR_ARG;
     c->profiling = on;
     return XSV_OK;
 }
