@@ -278,6 +278,14 @@ xsv_status xsv_last_scores(xsv_cache* c, float* scores_host, long long cap, long
  * XSV_OK, XSV_ERR_TIMEOUT or XSV_ERR_RANGE. */
 xsv_status xsv_cache_status(xsv_cache* c, void* stream);
 
+/* The raw status word behind xsv_cache_status (diagnostic; the paper has no
+ * counterpart): bit 0 a bounded wait ran out, bit 1 a value left the supported
+ * range, bits 8-14 which wait of the attention kernel gave up (0x100 a
+ * producer waiting for a free stage, 0x200 / 0x400 a softmax warp waiting for
+ * S / for the completion of P V, 0x800 / 0x1000 / 0x4000 the issuing warp
+ * waiting for the query tiles / a filled stage / a sub-tile's probabilities).  Synchronises `stream`; -1 on error. */
+int xsv_cache_status_word(xsv_cache* c, void* stream);
+
 /* Per-phase CUDA-event timing.  on = 1: every step records events around each
  * phase on the step's stream; on = 2: around the attention phase only (each
  * pair of events costs the stream a few microseconds, which matters when the

@@ -41,6 +41,7 @@ SYMBOLS = {
     "xsv_cache_import_layer": (_i, [_vp, _i, _ll, _ll, _i, _i] + [_vp] * 9 + [_vp]),
     "xsv_last_scores": (_i, [_vp, _vp, _ll, C.POINTER(_ll), _vp]),
     "xsv_cache_status": (_i, [_vp, _vp]),
+    "xsv_cache_status_word": (_i, [_vp, _vp]),
     "xsv_cache_set_profiling": (_i, [_vp, _i]),
     "xsv_cache_profile_read": (_i, [_vp, C.POINTER(C.c_double), C.POINTER(_ll), _i]),
     "xsv_selftest_bounded_wait": (_i, [_vp]),
@@ -200,6 +201,9 @@ class Cache:
 
     def status(self, stream=None):
         return int(self._lib.xsv_cache_status(self._h, _stream_ptr(stream)))
+
+    def status_word(self, stream=None):
+        return int(self._lib.xsv_cache_status_word(self._h, _stream_ptr(stream)))
 
     def set_profiling(self, on):
         _check(self._lib.xsv_cache_set_profiling(self._h, int(on)), "xsv_cache_set_profiling")

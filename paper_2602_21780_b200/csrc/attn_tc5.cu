@@ -23,7 +23,9 @@
 // sets XSV_DEV_TIMEOUT in the status word, after which all waits fall through
 // and the kernel runs to its end (tensor memory is always released).
 //
-// Operands are fp16 for both input types (bf16 converts exactly, saturating).
+// Operands are fp16 for both input types: bf16 inputs convert without rounding for magnitudes in [2^-14, 65504];
+// smaller magnitudes are held as fp16 subnormals (absolute error at most 2^-25), larger ones saturate to +-65504
+// and set XSV_DEV_RANGE in the status word.
 // The channel order inside shared memory is permuted (the order in which the
 // codes fall out of a packed 32-bit word); Q and fresh K rows are permuted the
 // same way, and the output columns are un-permuted in the epilogue.
@@ -33,9 +35,11 @@ namespace {
 
 constexpr int BM = 128;            // query rows per tile
 constexpr int BN = 128;            // keys per kv tile
+constexpr int SUB = 64;            // keys per S sub-tile: a kv tile is consumed as two halves
+constexpr int NBUF = 3;            // S sub-tile buffers per query tile in tensor memory
 constexpr int NSTAGE = 5;          // kv stages in shared memory
-constexpr int NPROD = 7;              // producer warps
-constexpr int NTHREADS = (8 + NPROD + 1) * 32;   // 8 softmax warps, the producers, the MMA issuer
+constexpr int NPROD = 6;              // producer warps
+constexpr int NTHREADS = (8 + NPROD + 2) * 32;   // 8 softmax warps, the producers, one MMA issuer per query tile
 constexpr uint32_t TILE_BYTES = 128u * 128u;   // 128 rows x 64 fp16
 // Cost model of the work split, in ticks (fitted to per-CTA durations measured with %globaltimer): a kv step with two
 // active query tiles, with one (the hand-over latencies, not the arithmetic, set the pace of a step), and the fixed
@@ -49,12 +53,18 @@ constexpr uint32_t OFF_Q = 0;                                  // 2 tiles
 constexpr uint32_t OFF_KV = 2 * TILE_BYTES;                    // NSTAGE x (K tile, V tile)
 constexpr uint32_t OFF_META = OFF_KV + NSTAGE * 2 * TILE_BYTES;   // key parameters as halves: [producer warp][offset | scale | bias][64]
 constexpr uint32_t OFF_BAR = OFF_META + 3072;
-constexpr uint32_t SMEM_BYTES = OFF_BAR + 256 + 1024;          // + alignment slack
+constexpr uint32_t BAR_BYTES = 512;
+constexpr uint32_t SMEM_BYTES = OFF_BAR + BAR_BYTES + 1024;    // + alignment slack
 
 // barrier slots (8 bytes each) inside the barrier block
-enum { B_KFULL = 0, B_VFULL = NSTAGE, B_EMPTY = 2 * NSTAGE, B_SFULL = 3 * NSTAGE, B_SFREE = B_SFULL + 2,
-       B_PREADY = B_SFREE + 2, B_PVDONE = B_PREADY + 2, B_QFULL = B_PVDONE + 2, B_COUNT = B_QFULL + 2 };
-static_assert(B_COUNT * 8 + 16 <= 256, "barrier block");
+enum { B_KFULL = 0, B_VFULL = NSTAGE, B_EMPTY = 2 * NSTAGE, B_SFULL = 3 * NSTAGE, B_PREADY = B_SFULL + 2 * NBUF,
+       B_PVDONE = B_PREADY + 2 * NBUF, B_QFULL = B_PVDONE + 2 * NBUF, B_COUNT = B_QFULL + 2 };
+static_assert(B_COUNT * 8 + 16 <= BAR_BYTES, "barrier block");
+// tensor-memory columns: S sub-tile buffer b of query tile x (its P, as fp16 pairs, overwrites the first half of
+// the S it was computed from), then the two output accumulators
+__host__ __device__ constexpr uint32_t TM_S(int x, int b) { return (uint32_t)((x * NBUF + b) * SUB); }
+constexpr uint32_t TM_O0 = 2 * NBUF * SUB;
+static_assert(TM_O0 + 2 * XSV_D <= 512, "tensor memory columns");
 static_assert(NPROD * 3 * 64 * 2 <= 3072, "staging area of the key parameters");
 
 struct Params {
@@ -131,21 +141,10 @@ __device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok;
 }
-// non-blocking test of a phase
-__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
 // Bounded wait.  On expiry (or once another thread gave up) it raises the abort
 // flag, records XSV_DEV_TIMEOUT and returns, so the kernel always terminates.
-__device__ __noinline__ void mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
+// `site` (one of the XSV_DEV_SITE_* bits) is recorded beside the flag: which kind of wait gave up.
+__device__ __noinline__ void mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int site) {
     const unsigned long long t0 = globaltimer();
     for (uint32_t i = 0;; ++i) {
         if (mbar_try(bar, parity)) return;
@@ -153,16 +152,16 @@ __device__ __noinline__ void mbar_wait_slow(uint32_t bar, uint32_t parity, volat
             if (*abort_flag) return;
             if (globaltimer() - t0 > WAIT_LIMIT_NS) {
                 *abort_flag = 1;
-                atomicOr(status, XSV_DEV_TIMEOUT);
+                atomicOr(status, XSV_DEV_TIMEOUT | site);
                 return;
             }
         }
     }
 }
-__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status) {
-    if (*abort_flag) return;
+__device__ __forceinline__ void mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int site) {
     if (mbar_try(bar, parity)) return;
-    mbar_wait_slow(bar, parity, abort_flag, status);
+    if (*abort_flag) return;
+    mbar_wait_slow(bar, parity, abort_flag, status, site);
 }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -220,11 +219,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
         : "r"(taddr)
         : "memory");
 }
-__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&v)[8]) {
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
-                 ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
-                 : "memory");
-}
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -257,7 +251,7 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
            (2ull << 61) /* 128-byte swizzle */;
 }
 // kind::f16, fp16 x fp16 -> fp32, M = 128
-constexpr uint32_t IDESC_QK = (1u << 4) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);                  // A, B K-major, N = 128
+constexpr uint32_t IDESC_QK = (1u << 4) | ((uint32_t)(SUB >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);                 // A, B K-major, N = 64
 constexpr uint32_t IDESC_PV = (1u << 4) | (1u << 16) | ((uint32_t)(XSV_D >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);   // B MN-major, N = 64
 
 // Channel held at shared-memory position p: the codes of one packed 32-bit word
@@ -276,10 +270,20 @@ template <> __device__ __forceinline__ uint32_t to_h2<__nv_bfloat16>(uint32_t w)
     return pack_h2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
 }
 
+// Nonzero iff one of the two bf16 halves of w has magnitude 2^16 or more (exponent field >= 143; Inf and NaN too),
+// i.e. converts to fp16 by saturation.  Carry-free: each masked half is at most 0x7F80.
+template <typename T> __device__ __forceinline__ uint32_t beyond_h2(uint32_t w);
+template <> __device__ __forceinline__ uint32_t beyond_h2<__half>(uint32_t) { return 0u; }
+template <> __device__ __forceinline__ uint32_t beyond_h2<__nv_bfloat16>(uint32_t w) {
+    return ((w & 0x7F807F80u) + 0x38803880u) & 0x80008000u;
+}
+
 // One row of 64 16-bit values (global) -> fp16, permuted, one swizzled 128-byte
-// row of a shared-memory tile.  grow == nullptr writes zeros.
+// row of a shared-memory tile.  grow == nullptr writes zeros.  Returns nonzero if a
+// value lay beyond the fp16 range (bf16 inputs only).
 template <typename T, int W>
-__device__ __forceinline__ void row16_to_tile(const T* grow, uint8_t* tile, int row) {
+__device__ __forceinline__ uint32_t row16_to_tile(const T* grow, uint8_t* tile, int row) {
+    uint32_t beyond = 0u;
 #pragma unroll
     for (int blk = 0; blk < 4; ++blk) {   // 16 channels = 8 input words = two 16-byte chunks
         uint32_t in[8];
@@ -290,6 +294,8 @@ __device__ __forceinline__ void row16_to_tile(const T* grow, uint8_t* tile, int 
 #pragma unroll
             for (int i = 0; i < 8; ++i) in[i] = 0u;
         }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) beyond |= beyond_h2<T>(in[i]);
         uint32_t o[8];
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
@@ -302,6 +308,7 @@ __device__ __forceinline__ void row16_to_tile(const T* grow, uint8_t* tile, int 
         *reinterpret_cast<uint4*>(tile + swz(row, 2 * blk)) = make_uint4(o[0], o[1], o[2], o[3]);
         *reinterpret_cast<uint4*>(tile + swz(row, 2 * blk + 1)) = make_uint4(o[4], o[5], o[6], o[7]);
     }
+    return beyond;
 }
 
 // In-register unpack.  The codes of one packed 32-bit word come out as pairs
@@ -341,11 +348,6 @@ __device__ __forceinline__ uint16_t f2h_sat(float x) {
     asm("cvt.rn.satfinite.f16.f32 %0, %1;" : "=h"(h) : "f"(x));
     return h;
 }
-__device__ __forceinline__ float h2f(uint16_t h) {
-    float f;
-    asm("cvt.f32.f16 %0, %1;" : "=f"(f) : "h"(h));
-    return f;
-}
 // the fp16 parameters (a, s, b) of dq_pair for scale s, zero-point z and offset off
 __device__ __forceinline__ void dq_params(float s, int z, int off, uint16_t& ah, uint16_t& sh, uint16_t& bh) {
     const int zo = z > 0x70000000 ? z : z + off;   // no overflow; such a z takes the far branch anyway
@@ -355,7 +357,7 @@ __device__ __forceinline__ void dq_params(float s, int z, int off, uint16_t& ah,
         bh = 0;
     } else {
         ah = 0;
-        bh = f2h_sat(-(float)zo * h2f(sh));
+        bh = f2h_sat(-(float)zo * s);   // from the float32 scale: the rounding error of sh times a large zero-point would be of the order of the values
     }
 }
 
@@ -365,18 +367,34 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     return d;
 }
 
-// 32 logits of one row -> 32 probabilities 2^(s * sc - m) packed as fp16 pairs;
-// accumulates their sum and the running maximum of the raw logits.
-template <bool WITH_MAX>
-__device__ __forceinline__ void softmax32(const uint32_t (&v)[32], float sc, float nm, float& mx, float& ls, uint32_t (&pk)[16]) {
+// 32 logits of one row -> 32 probabilities 2^(s * sc - m) packed as fp16 pairs; accumulates their sum.
+// Columns at or beyond `valid` (a ragged last tile) give probability 0.
+template <bool MASK>
+__device__ __forceinline__ void softmax32(const uint32_t (&v)[32], float sc, float nm, int valid, float& ls, uint32_t (&pk)[16]) {
 #pragma unroll
     for (int i = 0; i < 32; i += 2) {
-        const float s0 = __uint_as_float(v[i]), s1 = __uint_as_float(v[i + 1]);
-        if (WITH_MAX) mx = fmax3(mx, s0, s1);
-        const float p0 = ex2(fmaf(s0, sc, nm)), p1 = ex2(fmaf(s1, sc, nm));
+        float p0 = ex2(fmaf(__uint_as_float(v[i]), sc, nm)), p1 = ex2(fmaf(__uint_as_float(v[i + 1]), sc, nm));
+        if (MASK) {
+            if (i >= valid) p0 = 0.f;
+            if (i + 1 >= valid) p1 = 0.f;
+        }
         ls += p0 + p1;
         pk[i >> 1] = pack_h2(p0, p1);
     }
+}
+// running maximum of 32 raw logits (the first `valid` of them)
+template <bool MASK>
+__device__ __forceinline__ float max32(const uint32_t (&v)[32], int valid, float mx) {
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        float s0 = __uint_as_float(v[i]), s1 = __uint_as_float(v[i + 1]);
+        if (MASK) {
+            if (i >= valid) s0 = -INFINITY;
+            if (i + 1 >= valid) s1 = -INFINITY;
+        }
+        mx = fmax3(mx, s0, s1);
+    }
+    return mx;
 }
 
 // What every role needs to know about its CTA.
@@ -480,6 +498,7 @@ __device__ __noinline__ void producer_loop(const Params& p, const Cta c) {
         }
     };
 
+    uint32_t beyond = 0u;                           // a raw 16-bit input outside the fp16 range was seen
     TileIter cur{c.u_first, 0, 0, 0, false}, nxt;
     tile_iter_settle(p, b, u_last, cur);
     uint32_t it = 0;                                // kv tile of `cur`
@@ -505,7 +524,7 @@ __device__ __noinline__ void producer_loop(const Params& p, const Cta c) {
         const uint32_t st = it % NSTAGE;
         uint8_t* tile = smem + OFF_KV + st * 2 * TILE_BYTES + (sl < 4 ? 0u : TILE_BYTES);
         const int row = (sl & 3) * 32 + lane;
-        if (it >= NSTAGE) mbar_wait(BAR(B_EMPTY + st), ((it / NSTAGE) - 1u) & 1u, abort_flag, status);
+        if (it >= NSTAGE) mbar_wait(BAR(B_EMPTY + st), ((it / NSTAGE) - 1u) & 1u, abort_flag, status, XSV_DEV_SITE_STAGE);
         const bool cached = cur.kv < n_ct;
         if (BITS < 16 && cached) {
             if (sl < 4) {
@@ -569,7 +588,7 @@ __device__ __noinline__ void producer_loop(const Params& p, const Cta c) {
                 const int tok = (cur.kv - n_ct) * BN + row;
                 if (tok < F) src = (sl < 4 ? Kg : Vg) + ((size_t)cur.h * F + tok) * XSV_D;
             }
-            row16_to_tile<T, W>(src, tile, row);
+            beyond |= row16_to_tile<T, W>(src, tile, row);
         }
         fence_async_smem();
         __syncwarp();
@@ -579,6 +598,7 @@ __device__ __noinline__ void producer_loop(const Params& p, const Cta c) {
         it = itn;
         g = gn;
     }
+    if (beyond) atomicOr(status, XSV_DEV_RANGE);
 }
 
 // Softmax warpgroups (warps 0-3: query tile A, warps 4-7: tile B) and the epilogue.
@@ -600,12 +620,18 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
         const int X = warp >> 2;                       // query tile of this warpgroup
         const int row = tid & 127;
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem_base + lane_base + (uint32_t)(X * 128);
-        const uint32_t tP = tmem_base + lane_base + 256u + (uint32_t)(X * 64);
-        const uint32_t tO = tmem_base + lane_base + 384u + (uint32_t)(X * 64);
+        const uint32_t tS = tmem_base + lane_base + TM_S(X, 0);
+        const uint32_t tO = tmem_base + lane_base + TM_O0 + (uint32_t)(X * XSV_D);
         uint8_t* sQ = smem + OFF_Q + X * TILE_BYTES;
         const float SC = 0.125f * 1.4426950408889634f;   // 1/sqrt(64) * log2(e)
-        uint32_t cX = 0, uX = 0;
+        uint32_t cX = 0;                               // sub-tiles of this query tile so far (all units of the CTA)
+        // Completion of the P V of sub-tile j (and of every MMA issued before it).  One barrier per S buffer: a parity
+        // wait is only meaningful while the barrier is at most one phase ahead, and the barrier of buffer j % NBUF
+        // cannot complete again before this warp has handed over the P of sub-tile j + NBUF; its previous phase
+        // (sub-tile j - NBUF) is known complete once S of sub-tile j' >= j has been received.
+        auto wait_pv = [&](uint32_t j) {
+            mbar_wait(BAR(B_PVDONE + X * NBUF + (int)(j % NBUF)), (j / NBUF) & 1u, abort_flag, status, XSV_DEV_SITE_PV);
+        };
         for (int u = u_first; u <= u_last; ++u) {
             const Span sp = cta_span(p, b, u);
             if (sp.kv0 >= sp.kv1) continue;
@@ -615,80 +641,42 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
             const int grow = q0 + row;
             // ---- this unit's queries -> shared memory (all MMAs reading the previous unit's tile are complete:
             //      the last S of that unit has been received)
-            row16_to_tile<T, W>(grow < F ? Qg + ((size_t)h * F + grow) * XSV_D : nullptr, sQ, row);
+            if (row16_to_tile<T, W>(grow < F ? Qg + ((size_t)h * F + grow) * XSV_D : nullptr, sQ, row)) atomicOr(status, XSV_DEV_RANGE);
             fence_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(BAR(B_QFULL + X));
-            ++uX;
 
+            // Online softmax over sub-tiles of 64 keys.  S arrives in one of NBUF buffers (the QK^T of the next
+            // sub-tiles are already in flight or done while this one is worked on); the probabilities, as fp16
+            // pairs, overwrite the first half of the buffer they were computed from.  The row maximum in use is
+            // updated lazily: it stays while the true maximum is at most RESCALE_THRESHOLD (log2 units) above
+            // it, so the accumulator is rarely rescaled (always on a span's first sub-tile).
             float m_used = -INFINITY, l = 0.f;
+            bool first = true;
             for (int kv = sp.kv0; kv < sp.kv1; ++kv) {
                 const int cnt = kv < n_ct ? min(BN, T_c - kv * BN) : min(BN, F - (kv - n_ct) * BN);
-                const bool tail = cnt < BN;
-                const bool first = kv == sp.kv0;
-                mbar_wait(BAR(B_SFULL + X), cX & 1u, abort_flag, status);
-                tc_fence_after();
-                float nm = -m_used, ls = 0.f, mx = -INFINITY;
-                bool done = false;
-                if (!tail) {
-                    // ---- whole tile, one pass with the row maximum in use (stale by at most the threshold).  The
-                    //      first two 32-column chunks are turned into probabilities (kept in registers) while the
-                    //      other two are fetched; then all of S has been read, its maximum is known, and if the
-                    //      maximum in use may stay, S is released: the next QK^T and its hand-over latency
-                    //      overlap the second half of the tile.  The wait for the previous PV (P is single-buffered)
-                    //      comes only then, half a tile after that PV was triggered.
-                    uint32_t va[32], vb[32], pa[16], pb[16];
-                    tmem_ld32(tS, va);
+                for (int sub = 0; sub * SUB < cnt; ++sub) {
+                    const int valid = cnt - sub * SUB;             // >= SUB: a whole sub-tile
+                    const uint32_t buf = cX % NBUF;
+                    const uint32_t tSb = tS + buf * SUB;
+                    mbar_wait(BAR(B_SFULL + X * NBUF + (int)buf), (cX / NBUF) & 1u, abort_flag, status, XSV_DEV_SITE_S);
+                    tc_fence_after();
+                    uint32_t va[32], vb[32], pk[16];
+                    tmem_ld32(tSb, va);
+                    tmem_ld32(tSb + 32u, vb);
                     tc_wait_ld();
-                    tmem_ld32(tS + 32u, vb);
-                    softmax32<true>(va, SC, nm, mx, ls, pa);
-                    tc_wait_ld();
-                    tmem_ld32(tS + 64u, va);
-                    softmax32<true>(vb, SC, nm, mx, ls, pb);
-                    tc_wait_ld();
-                    tmem_ld32(tS + 96u, vb);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        mx = fmax3(mx, __uint_as_float(va[i]), __uint_as_float(va[i + 1]));
-                        mx = fmax3(mx, __uint_as_float(vb[i]), __uint_as_float(vb[i + 1]));
-                    }
-                    if (!__any_sync(0xFFFFFFFFu, mx * SC > m_used + RESCALE_THRESHOLD)) {
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(BAR(B_SFREE + X));
-                        mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, status);
-                        tc_fence_after();
-                        tmem_st16(tP, pa);
-                        tmem_st16(tP + 16u, pb);
-                        softmax32<false>(va, SC, nm, mx, ls, pa);
-                        tmem_st16(tP + 32u, pa);
-                        softmax32<false>(vb, SC, nm, mx, ls, pb);
-                        tmem_st16(tP + 48u, pb);
-                        done = true;
-                    }
-                } else {
-                    // ---- ragged tile: masked maximum (compact loop)
-#pragma unroll 1
-                    for (int c = 0; c < 8; ++c) {
-                        uint32_t v[16];
-                        tmem_ld16(tS + 16u * c, v);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            if (16 * c + i < cnt) mx = fmaxf(mx, __uint_as_float(v[i]));
-                    }
-                }
-                if (!done) {
-                    // ---- rare (always on the span's first tile): the maximum moved by more than the threshold, or
-                    //      the tile is ragged
-                    if (!first) {   // PV of the previous tile must be complete before P is overwritten or O rescaled
-                        mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, status);
-                        tc_fence_after();
-                    }
+                    float mx;
+                    if (valid >= SUB) mx = max32<false>(vb, 32, max32<false>(va, 32, -INFINITY));
+                    else mx = max32<true>(vb, valid - 32, max32<true>(va, valid, -INFINITY));
                     const float m_new = mx * SC;
                     const bool need = m_new > m_used + RESCALE_THRESHOLD;
-                    if (__any_sync(0xFFFFFFFFu, need)) {   // rescale the accumulator and the row sum
+                    if (__any_sync(0xFFFFFFFFu, need)) {
+                        // the maximum moved by more than the threshold: rescale the accumulator and the row sum
+                        // (the previous sub-tile's P V must have completed first)
+                        if (!first) {
+                            wait_pv(cX - 1u);
+                            tc_fence_after();
+                        }
                         const float alpha = need ? ex2(m_used - m_new) : 1.f;
                         if (need) m_used = m_new;
                         l *= alpha;
@@ -704,39 +692,30 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
                             }
                         }
                     }
-                    // this tile's probabilities with the maximum now in use, masking a ragged tail
-                    nm = -m_used;
-                    ls = 0.f;
-#pragma unroll 1
-                    for (int c = 0; c < 8; ++c) {
-                        uint32_t v[16], pk[8];
-                        tmem_ld16(tS + 16u * c, v);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int i = 0; i < 16; i += 2) {
-                            float s0 = __uint_as_float(v[i]), s1 = __uint_as_float(v[i + 1]);
-                            if (16 * c + i >= cnt) s0 = -INFINITY;
-                            if (16 * c + i + 1 >= cnt) s1 = -INFINITY;
-                            const float p0 = ex2(fmaf(s0, SC, nm)), p1 = ex2(fmaf(s1, SC, nm));
-                            ls += p0 + p1;
-                            pk[i >> 1] = pack_h2(p0, p1);
-                        }
-                        tmem_st8(tP + 8u * c, pk);
+                    const float nm = -m_used;
+                    float ls = 0.f;
+                    if (valid >= SUB) {
+                        softmax32<false>(va, SC, nm, 32, ls, pk);
+                        tmem_st16(tSb, pk);
+                        softmax32<false>(vb, SC, nm, 32, ls, pk);
+                        tmem_st16(tSb + 16u, pk);
+                    } else {
+                        softmax32<true>(va, SC, nm, valid, ls, pk);
+                        tmem_st16(tSb, pk);
+                        softmax32<true>(vb, SC, nm, valid - 32, ls, pk);
+                        tmem_st16(tSb + 16u, pk);
                     }
-                    // S has been read for good: the next QK^T may overwrite it
+                    l += ls;
+                    tc_wait_st();
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(BAR(B_SFREE + X));
+                    if (lane == 0) mbar_arrive(BAR(B_PREADY + X * NBUF + (int)buf));
+                    ++cX;
+                    first = false;
                 }
-                l += ls;
-                tc_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(BAR(B_PREADY + X));
-                ++cX;
             }
             // ---- epilogue of the span
-            mbar_wait(BAR(B_PVDONE + X), (cX - 1u) & 1u, abort_flag, status);
+            wait_pv(cX - 1u);
             tc_fence_after();
             const bool full = sp.kv0 == 0 && sp.kv1 == nkv;
             const float inv = 1.f / l;
@@ -786,102 +765,108 @@ __device__ __forceinline__ bool elect_one() {
     return p != 0;
 }
 
-// MMA issuer: one warp running converged; the tensor-core instructions and their
-// commits are issued by its elected lane (a single thread issuing from a diverged
-// warp measured about twice as slow per instruction).
-__device__ __noinline__ void mma_loop(const Params& p, const Cta c) {
+// MMA issuers: one warp per query tile, each running converged; the tensor-core instructions and their commits
+// are issued by its elected lane.
+//
+// Tile x consumes the span's kv tiles as sub-tiles of 64 keys: S_j = Q K_j^T into buffer j % NBUF, then (once the
+// softmax warps have turned S_j into P_j in place) O += P_j V_j.  The tensor pipe executes the MMAs of one thread
+// in issue order, so QK(j + NBUF) is issued right behind PV(j) into the buffer that PV(j) reads: no barrier is
+// needed for the reuse, and NBUF QK^T run ahead of the softmax.
+//
+// The order of issue is fixed -- PV(j), QK(j + NBUF), j = 0, 1, ... -- and every counter is a loop variable that
+// depends on the kernel parameters and the block index only, never on the outcome of a barrier test; that keeps
+// the operands of the tcgen05 instructions (descriptors, tensor-memory addresses, barrier addresses) uniform.
+// What sets the pace of this loop is the chain of waits, fences and elections around each group of four MMAs,
+// not the MMAs themselves (which execute in 35-52 clocks each), hence one such loop per query tile.
+__device__ __noinline__ void mma_loop(const Params& p, const Cta c, const int x) {
     const uint32_t smem_base = c.smem_base, tmem_base = c.tmem_base;
     volatile int* const abort_flag = c.abort_flag;
     const int b = c.b, u_first = c.u_first, u_last = c.u_last;
     auto BAR = [&](int i) { return c.bar_base + 8u * (uint32_t)i; };
-    const int F = p.F;
+    const int F = p.F, n_ct = p.n_ct, T_c = p.T_c;
     int* const status = p.status;
-    // Each query tile has its own strictly ordered sequence QK(0), QK(1), PV(0), QK(2), PV(1), ... in which
-    // every operation is gated by one barrier phase; the two sequences are merged by readiness, so that a
-    // tile never waits for the other tile's softmax.  Every lane takes the same decisions: a barrier test is
-    // broadcast from lane 0.
-    const uint32_t tS0 = tmem_base, tP0 = tmem_base + 256u, tO0 = tmem_base + 384u;
-    uint32_t it0 = 0, cT[2] = {0, 0}, uT[2] = {0, 0};
+    const uint32_t tS = tmem_base + TM_S(0, 0) + (uint32_t)x * (NBUF * SUB), tO = tmem_base + TM_O0 + (uint32_t)(x * XSV_D);
+    const uint64_t qd = smem_desc(smem_base + OFF_Q + (uint32_t)x * TILE_BYTES);
+    auto nsub_of = [&](int kv) {   // sub-tiles of kv tile `kv`: 1 when at most 64 of its keys exist
+        const int cnt = kv < n_ct ? min(BN, T_c - kv * BN) : min(BN, F - (kv - n_ct) * BN);
+        return cnt > SUB ? 2 : 1;
+    };
+    // S = Q K^T of sub-tile (kv tile number `it` of the CTA, half `half`) into buffer `buf`
+    auto issue_qk = [&](uint32_t it, int half, uint32_t buf) {
+        const uint32_t st = it % NSTAGE;
+        if (half == 0) mbar_wait(BAR(B_KFULL + (int)st), (it / NSTAGE) & 1u, abort_flag, status, XSV_DEV_SITE_K);
+        tc_fence_after();
+        const uint64_t kd = smem_desc(smem_base + OFF_KV + st * 2 * TILE_BYTES + (uint32_t)half * (SUB * 128u));
+        if (elect_one()) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k)            // 16 channels = 32 bytes inside the swizzled row
+                mma_ss(tS + buf * SUB, qd + 2u * k, kd + 2u * k, IDESC_QK, k > 0);
+            tc_commit(BAR(B_SFULL + x * NBUF + (int)buf));
+        }
+        __syncwarp();
+    };
+    uint32_t it0 = 0;            // kv tiles of the CTA before this unit
+    uint32_t cT = 0, uT = 0;     // sub-tiles and units of this query tile before this unit
     for (int u = u_first; u <= u_last; ++u) {
         const Span sp = cta_span(p, b, u);
         if (sp.kv0 >= sp.kv1) continue;
         const int mp = u % p.npair;
         const int ntile = (mp * 2 * BM + BM < F) ? 2 : 1;
         const int n = sp.kv1 - sp.kv0;
-        for (int x = 0; x < ntile; ++x) mbar_wait(BAR(B_QFULL + x), uT[x] & 1u, abort_flag, status);
+        if (x >= ntile) {
+            // This unit has no second query tile: tile 0's warp releases the stages for both.  This warp still
+            // consumes the stages' barrier phases one by one, so that it never runs more than one phase ahead
+            // of a barrier (a parity wait means nothing beyond that).
+            for (int i = 0; i < n; ++i) {
+                const uint32_t it = it0 + (uint32_t)i, st = it % NSTAGE;
+                mbar_wait(BAR(B_KFULL + (int)st), (it / NSTAGE) & 1u, abort_flag, status, XSV_DEV_SITE_K);
+                mbar_wait(BAR(B_VFULL + (int)st), (it / NSTAGE) & 1u, abort_flag, status, XSV_DEV_SITE_K);
+            }
+            it0 += (uint32_t)n;
+            continue;
+        }
+        mbar_wait(BAR(B_QFULL + x), uT & 1u, abort_flag, status, XSV_DEV_SITE_Q);
         tc_fence_after();
-        int qk_next[2] = {0, 0}, pv_next[2] = {0, 0};
-        if (ntile == 1) { qk_next[1] = n; pv_next[1] = n; }
-        unsigned long long t_idle = 0;
-        uint32_t idle = 0;
-        while (pv_next[0] < n || pv_next[1] < n) {
-            bool progress = false;
-            // Test the gates of the next QK and the next PV of both tiles at once: the eight barrier reads are
-            // independent, so their latencies overlap (one after the other they cost far more than the issue).
-            uint32_t itq[2], sq[2], cq[2], itp[2], sv[2], bits = 0;
+        // ---- the first NBUF QK^T of the unit
+        int qi = 0, qs = 0, qj = 0;                      // next QK: kv tile of the span, half, sub-tile of the unit
+        for (; qj < NBUF && qi < n; ++qj) {
+            issue_qk(it0 + (uint32_t)qi, qs, (cT + (uint32_t)qj) % NBUF);
+            if (qs + 1 >= nsub_of(sp.kv0 + qi)) { ++qi; qs = 0; } else ++qs;
+        }
+        // ---- PV(j), then QK(j + NBUF)
+        int pj = 0;
+        for (int i = 0; i < n; ++i) {
+            const uint32_t it = it0 + (uint32_t)i, st = it % NSTAGE;
+            const int ns = nsub_of(sp.kv0 + i);
+            mbar_wait(BAR(B_VFULL + (int)st), (it / NSTAGE) & 1u, abort_flag, status, XSV_DEV_SITE_K);
+            for (int half = 0; half < ns; ++half, ++pj) {
+                const uint32_t cp = cT + (uint32_t)pj, buf = cp % NBUF;
+                mbar_wait(BAR(B_PREADY + x * NBUF + (int)buf), (cp / NBUF) & 1u, abort_flag, status, XSV_DEV_SITE_P);
+                tc_fence_after();
+                const uint64_t vd = smem_desc(smem_base + OFF_KV + st * 2 * TILE_BYTES + TILE_BYTES + (uint32_t)half * (SUB * 128u));
+                const uint32_t acc0 = pj > 0 ? 1u : 0u;
+                const bool release = half + 1 == ns;          // this tile is through with the stage
+                if (elect_one()) {
 #pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                const uint32_t jq = (uint32_t)min(qk_next[x], n - 1), jp = (uint32_t)min(pv_next[x], n - 1);
-                itq[x] = it0 + jq; sq[x] = itq[x] % NSTAGE; cq[x] = cT[x] + jq;   // cq: number of this tile's S among all of the CTA's
-                itp[x] = it0 + jp; sv[x] = itp[x] % NSTAGE;
-                bits |= mbar_test(BAR(B_KFULL + sq[x]), (itq[x] / NSTAGE) & 1u) << (4 * x);
-                bits |= (cq[x] == 0 ? 1u : mbar_test(BAR(B_SFREE + x), (cq[x] - 1u) & 1u)) << (4 * x + 1);
-                bits |= mbar_test(BAR(B_VFULL + sv[x]), (itp[x] / NSTAGE) & 1u) << (4 * x + 2);
-                bits |= mbar_test(BAR(B_PREADY + x), (cT[x] + jp) & 1u) << (4 * x + 3);
-            }
-            bits = __shfl_sync(0xFFFFFFFFu, bits, 0);      // every lane takes lane 0's view
-#pragma unroll
-            for (int x = 0; x < 2; ++x) {
-                if (qk_next[x] < n && ((bits >> (4 * x)) & 3u) == 3u) {
-                    tc_fence_after();
-                    const uint64_t qd = smem_desc(smem_base + OFF_Q + x * TILE_BYTES);
-                    const uint64_t kd = smem_desc(smem_base + OFF_KV + sq[x] * 2 * TILE_BYTES);
-                    if (elect_one()) {
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)        // 16 channels = 32 bytes inside the swizzled row
-                            mma_ss(tS0 + (uint32_t)(x * 128), qd + 2u * k, kd + 2u * k, IDESC_QK, k > 0);
-                        tc_commit(BAR(B_SFULL + x));
+                    for (int k = 0; k < SUB / 16; ++k)     // 16 tokens: 8 columns of P, 2048 bytes of V
+                        mma_ts(tO, tS + buf * SUB + 8u * k, vd + 128u * k, IDESC_PV, k > 0 ? 1u : acc0);
+                    tc_commit(BAR(B_PVDONE + x * NBUF + (int)buf));
+                    if (release) {
+                        tc_commit(BAR(B_EMPTY + (int)st));
+                        if (ntile == 1) tc_commit(BAR(B_EMPTY + (int)st));   // the other tile's share
                     }
-                    __syncwarp();
-                    ++qk_next[x];
-                    progress = true;
-                } else if (pv_next[x] < n && pv_next[x] < qk_next[x] && ((bits >> (4 * x + 2)) & 3u) == 3u) {
-                    const int j = pv_next[x];
-                    tc_fence_after();
-                    const uint64_t vd = smem_desc(smem_base + OFF_KV + sv[x] * 2 * TILE_BYTES + TILE_BYTES);
-                    const bool release = pv_next[x ^ 1] > j;   // both tiles are through with this stage
-                    if (elect_one()) {
-                        if (j > 0) {
-#pragma unroll
-                            for (int k = 0; k < 8; ++k)    // 16 tokens: 8 columns of P, 2048 bytes of V
-                                mma_ts(tO0 + (uint32_t)(x * 64), tP0 + (uint32_t)(x * 64) + 8u * k, vd + 128u * k, IDESC_PV, 1u);
-                        } else {
-#pragma unroll
-                            for (int k = 0; k < 8; ++k)
-                                mma_ts(tO0 + (uint32_t)(x * 64), tP0 + (uint32_t)(x * 64) + 8u * k, vd + 128u * k, IDESC_PV, k > 0);
-                        }
-                        tc_commit(BAR(B_PVDONE + x));
-                        if (release) tc_commit(BAR(B_EMPTY + sv[x]));
-                    }
-                    __syncwarp();
-                    ++pv_next[x];
-                    progress = true;
                 }
-            }
-            if (progress) {
-                idle = 0;
-            } else {
-                if (*abort_flag) break;
-                if (++idle == 64u) t_idle = globaltimer();
-                if (idle > 64u && (idle & 255u) == 0u && globaltimer() - t_idle > WAIT_LIMIT_NS) {
-                    *abort_flag = 1;
-                    atomicOr(status, XSV_DEV_TIMEOUT);
-                    break;
+                __syncwarp();
+                if (qi < n) {
+                    issue_qk(it0 + (uint32_t)qi, qs, (cT + (uint32_t)qj) % NBUF);
+                    ++qj;
+                    if (qs + 1 >= nsub_of(sp.kv0 + qi)) { ++qi; qs = 0; } else ++qs;
                 }
             }
         }
         it0 += (uint32_t)n;
-        for (int x = 0; x < ntile; ++x) { cT[x] += (uint32_t)n; ++uT[x]; }
+        cT += (uint32_t)pj;
+        ++uT;
     }
 }
 
@@ -899,26 +884,30 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_cons
     const int tid = threadIdx.x, warp = tid >> 5;
     const int b = blockIdx.x;
     const long long tick0 = cta_tick(p, b), tick1 = cta_tick(p, b + 1);
-    if (tick0 >= tick1) return;                       // uniform: nothing to do, nothing allocated
+    if (tick0 >= tick1) {                             // uniform: nothing to do, nothing allocated
+        xsv_dep_sync();                               // every block waits for the kernel before it, so that the order of the chain holds
+        return;
+    }
     const int u_first = unit_of_tick(p, tick0), u_last = unit_of_tick(p, tick1 - 1);
 
     if (tid == 0) {
         for (int i = 0; i < NSTAGE; ++i) {
             mbar_init(BAR(B_KFULL + i), 4);     // one arrival per producer warp
             mbar_init(BAR(B_VFULL + i), 4);
-            mbar_init(BAR(B_EMPTY + i), 1);
+            mbar_init(BAR(B_EMPTY + i), 2);     // one commit per query tile
         }
         for (int x = 0; x < 2; ++x) {
-            mbar_init(BAR(B_SFULL + x), 1);
-            mbar_init(BAR(B_SFREE + x), 4);     // one arrival per softmax warp
-            mbar_init(BAR(B_PREADY + x), 4);
-            mbar_init(BAR(B_PVDONE + x), 1);
+            for (int i = 0; i < NBUF; ++i) {
+                mbar_init(BAR(B_SFULL + x * NBUF + i), 1);
+                mbar_init(BAR(B_PREADY + x * NBUF + i), 4);     // one arrival per softmax warp
+                mbar_init(BAR(B_PVDONE + x * NBUF + i), 1);
+            }
             mbar_init(BAR(B_QFULL + x), 4);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 8 + NPROD) {
+    if (warp == 8 + NPROD + 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32((const void*)tmem_slot)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -932,13 +921,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_cons
     xsv_dep_sync();      // everything above is set-up that touches no global memory
     if (warp < 8) softmax_loop<T, BITS>(p, cta);
     else if (warp < 8 + NPROD) producer_loop<T, BITS>(p, cta);
-    else mma_loop(p, cta);
+    else mma_loop(p, cta, warp - (8 + NPROD));
     tc_fence_before();
     __syncthreads();
     // Only now may the next kernel be scheduled: released at the start, its blocks would sit through this whole kernel
     // on whatever multiprocessor the grid leaves free (the one kept for the selection kernel of another stream).
     xsv_dep_release();
-    if (warp == 8 + NPROD) {
+    if (warp == 8 + NPROD + 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     }
@@ -987,8 +976,8 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const Params p) {
     }
     __syncthreads();
     const int n = s_n;
-    if (n == 0) return;
     xsv_dep_sync();      // the part list is arithmetic on the parameters; the parts themselves come from the attention kernel
+    if (n == 0) return;  // (after the wait: every block of every kernel of the chain waits for its predecessor)
     const int h = u / p.npair, mp = u - h * p.npair;
     const int row = blockIdx.x * 16 + (threadIdx.x >> 4), c4 = threadIdx.x & 15;
     const int grow = mp * 2 * BM + row;
@@ -1048,7 +1037,7 @@ __global__ void wait_selftest_kernel(int* status) {
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    mbar_wait(smem_u32(&bar), 0u, &abort_flag, status);
+    mbar_wait(smem_u32(&bar), 0u, &abort_flag, status, XSV_DEV_SITE_SELFTEST);
 }
 
 int sm_count() {

@@ -792,6 +792,15 @@ xsv_status xsv_cache_status(xsv_cache* c, void* stream) {
     return XSV_OK;
 }
 
+int xsv_cache_status_word(xsv_cache* c, void* stream) {
+    if (!c) return -1;
+    if (!c->allocated) return 0;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess || sync_side_streams(c) != cudaSuccess) return -1;
+    int w = 0;
+    if (cudaMemcpy(&w, c->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+    return w;
+}
+
 xsv_status xsv_cache_set_profiling(xsv_cache* c, int on) {
     if (!c) return XSV_ERR_ARG;
     if (on < 0 || on > 3) return XSV_ERR_ARG;

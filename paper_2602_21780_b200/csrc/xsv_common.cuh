@@ -13,6 +13,14 @@
 // Bits of the sticky device status word.
 #define XSV_DEV_TIMEOUT 1
 #define XSV_DEV_RANGE 2
+// Beside XSV_DEV_TIMEOUT: which wait of the attention kernel ran out (diagnostic only).
+#define XSV_DEV_SITE_STAGE 0x100     // a producer waiting for a free kv stage
+#define XSV_DEV_SITE_S 0x200         // a softmax warp waiting for S
+#define XSV_DEV_SITE_PV 0x400        // a softmax warp waiting for the completion of P V
+#define XSV_DEV_SITE_Q 0x800         // the MMA warp waiting for a unit's query tiles
+#define XSV_DEV_SITE_K 0x1000        // the MMA warp waiting for a kv stage to be filled
+#define XSV_DEV_SITE_P 0x4000        // the MMA warp waiting for a sub-tile's probabilities
+#define XSV_DEV_SITE_SELFTEST 0x2000
 
 // One layer's cache as the kernels see it.  All arrays live in one slab.
 //   kcodes/vcodes [H][cap][rowb] : packed codes of one (head, token) row, code c
