@@ -45,7 +45,7 @@ constexpr uint32_t TILE_BYTES = 128u * 128u;   // 128 rows x 64 fp16
 // active query tiles, with one (the hand-over latencies, not the arithmetic, set the pace of a step), and the fixed
 // cost of entering a unit (query tiles loaded, the first tile's rescale, the epilogue).
 constexpr int COST_PAIR = 16, COST_SINGLE = 13, COST_UNIT = 72;
-constexpr float RESCALE_THRESHOLD = 8.f;       // log2 units; below it the stale row maximum is kept
+constexpr float SUM_LIMIT = 256.f;             // a sub-tile's row sum that reaches 2^8 (a logit 8 log2 units above the maximum in use does) triggers the careful path
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 // shared-memory map (from a 1024-byte aligned base)
@@ -367,8 +367,38 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     return d;
 }
 
-// 32 logits of one row -> 32 probabilities 2^(s * sc - m) packed as fp16 pairs; accumulates their sum.
-// Columns at or beyond `valid` (a ragged last tile) give probability 0.
+// packed pairs of float32 (one 64-bit register): two lanes of fma / add per instruction
+__device__ __forceinline__ unsigned long long f2_pack(float a, float b) {
+    unsigned long long r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(unsigned long long v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ unsigned long long f2_fma(unsigned long long a, unsigned long long b, unsigned long long c) {
+    unsigned long long d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ unsigned long long f2_add(unsigned long long a, unsigned long long b) {
+    unsigned long long d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// 32 logits of one row -> 32 probabilities 2^(s * sc - m) packed as fp16 pairs; their sum is added to the two
+// lanes of ls2.  Whole sub-tiles only.  The scaling and the sum run as packed float32 pairs (half the issue slots).
+__device__ __forceinline__ void softmax32_fast(const uint32_t (&v)[32], unsigned long long sc2, unsigned long long nm2,
+                                               unsigned long long& ls2, uint32_t (&pk)[16]) {
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        float x0, x1;
+        f2_unpack(f2_fma(f2_pack(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), sc2, nm2), x0, x1);
+        const float p0 = ex2(x0), p1 = ex2(x1);
+        ls2 = f2_add(ls2, f2_pack(p0, p1));
+        pk[i >> 1] = pack_h2(p0, p1);
+    }
+}
+// The same with a mask: columns at or beyond `valid` (a ragged last tile) give probability 0.
 template <bool MASK>
 __device__ __forceinline__ void softmax32(const uint32_t (&v)[32], float sc, float nm, int valid, float& ls, uint32_t (&pk)[16]) {
 #pragma unroll
@@ -648,9 +678,14 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
 
             // Online softmax over sub-tiles of 64 keys.  S arrives in one of NBUF buffers (the QK^T of the next
             // sub-tiles are already in flight or done while this one is worked on); the probabilities, as fp16
-            // pairs, overwrite the first half of the buffer they were computed from.  The row maximum in use is
-            // updated lazily: it stays while the true maximum is at most RESCALE_THRESHOLD (log2 units) above
-            // it, so the accumulator is rarely rescaled (always on a span's first sub-tile).
+            // pairs, overwrite the first half of the buffer they were computed from.
+            //
+            // The row maximum in use, m_used, is updated lazily.  The usual path does not look for the maximum at
+            // all: it exponentiates with m_used and watches the row sum of the sub-tile.  A logit more than
+            // 8 (log2 units) above m_used makes that sum reach SUM_LIMIT = 2^8; then (and on
+            // a span's first sub-tile, and on ragged ones) the careful path below finds the true maximum, rescales
+            // the accumulator and the running sum if it lies above m_used, and redoes the sub-tile from the
+            // logits, which are still in registers.  A sum that large without such a logit only costs the redo.
             float m_used = -INFINITY, l = 0.f;
             bool first = true;
             for (int kv = sp.kv0; kv < sp.kv1; ++kv) {
@@ -665,45 +700,60 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
                     tmem_ld32(tSb, va);
                     tmem_ld32(tSb + 32u, vb);
                     tc_wait_ld();
-                    float mx;
-                    if (valid >= SUB) mx = max32<false>(vb, 32, max32<false>(va, 32, -INFINITY));
-                    else mx = max32<true>(vb, valid - 32, max32<true>(va, valid, -INFINITY));
-                    const float m_new = mx * SC;
-                    const bool need = m_new > m_used + RESCALE_THRESHOLD;
-                    if (__any_sync(0xFFFFFFFFu, need)) {
-                        // the maximum moved by more than the threshold: rescale the accumulator and the row sum
-                        // (the previous sub-tile's P V must have completed first)
-                        if (!first) {
-                            wait_pv(cX - 1u);
-                            tc_fence_after();
-                        }
-                        const float alpha = need ? ex2(m_used - m_new) : 1.f;
-                        if (need) m_used = m_new;
-                        l *= alpha;
-                        if (!first) {
+                    float ls = 0.f;
+                    bool careful = first || valid < SUB;           // uniform
+                    if (!careful) {
+                        const unsigned long long sc2 = f2_pack(SC, SC), nm2 = f2_pack(-m_used, -m_used);
+                        unsigned long long ls2 = f2_pack(0.f, 0.f);
+                        softmax32_fast(va, sc2, nm2, ls2, pk);
+                        tmem_st16(tSb, pk);
+                        softmax32_fast(vb, sc2, nm2, ls2, pk);
+                        tmem_st16(tSb + 16u, pk);
+                        float l0, l1;
+                        f2_unpack(ls2, l0, l1);
+                        ls = l0 + l1;
+                        careful = __any_sync(0xFFFFFFFFu, !(ls < SUM_LIMIT));
+                    }
+                    if (careful) {
+                        float mx;
+                        if (valid >= SUB) mx = max32<false>(vb, 32, max32<false>(va, 32, -INFINITY));
+                        else mx = max32<true>(vb, valid - 32, max32<true>(va, valid, -INFINITY));
+                        const float m_new = mx * SC;
+                        const bool need = m_new > m_used;
+                        if (__any_sync(0xFFFFFFFFu, need)) {
+                            // rescale the accumulator and the row sum (the previous sub-tile's P V must have completed)
+                            if (!first) {
+                                wait_pv(cX - 1u);
+                                tc_fence_after();
+                            }
+                            const float alpha = need ? ex2(m_used - m_new) : 1.f;
+                            if (need) m_used = m_new;
+                            l *= alpha;
+                            if (!first) {
 #pragma unroll 1
-                            for (int c = 0; c < 4; ++c) {
-                                uint32_t o[16];
-                                tmem_ld16(tO + 16u * c, o);
-                                tc_wait_ld();
+                                for (int c = 0; c < 4; ++c) {
+                                    uint32_t o[16];
+                                    tmem_ld16(tO + 16u * c, o);
+                                    tc_wait_ld();
 #pragma unroll
-                                for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-                                tmem_st16(tO + 16u * c, o);
+                                    for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                                    tmem_st16(tO + 16u * c, o);
+                                }
                             }
                         }
-                    }
-                    const float nm = -m_used;
-                    float ls = 0.f;
-                    if (valid >= SUB) {
-                        softmax32<false>(va, SC, nm, 32, ls, pk);
-                        tmem_st16(tSb, pk);
-                        softmax32<false>(vb, SC, nm, 32, ls, pk);
-                        tmem_st16(tSb + 16u, pk);
-                    } else {
-                        softmax32<true>(va, SC, nm, valid, ls, pk);
-                        tmem_st16(tSb, pk);
-                        softmax32<true>(vb, SC, nm, valid - 32, ls, pk);
-                        tmem_st16(tSb + 16u, pk);
+                        const float nm = -m_used;
+                        ls = 0.f;
+                        if (valid >= SUB) {
+                            softmax32<false>(va, SC, nm, 32, ls, pk);
+                            tmem_st16(tSb, pk);
+                            softmax32<false>(vb, SC, nm, 32, ls, pk);
+                            tmem_st16(tSb + 16u, pk);
+                        } else {
+                            softmax32<true>(va, SC, nm, valid, ls, pk);
+                            tmem_st16(tSb, pk);
+                            softmax32<true>(vb, SC, nm, valid - 32, ls, pk);
+                            tmem_st16(tSb + 16u, pk);
+                        }
                     }
                     l += ls;
                     tc_wait_st();
