@@ -23,14 +23,25 @@
  *  - Q, K, V, out: [heads][n_tokens][head_dim], contiguous, 16-bit elements
  *    (fp16 or bf16 as given by `dtype`), 16-byte aligned.  `out` must not
  *    alias an input.
- *  - xsv_step only enqueues work on `stream`; it does not synchronise and
- *    does not allocate (all device memory is allocated by
- *    xsv_cache_create / xsv_cache_set_options / the first step).
+ *  - Input range: finite values of magnitude at most 65504.  The attention
+ *    kernels hold their tensor-core operands as fp16; bf16 inputs convert
+ *    without rounding for magnitudes in [2^-14, 65504], smaller ones are
+ *    held with an absolute error of at most 2^-25, and a bf16 magnitude of
+ *    2^16 or more saturates and sets XSV_ERR_RANGE in the status word (the
+ *    default attention kernel reports it; see xsv_cache_status).
+ *  - xsv_step only enqueues work on `stream`; it does not synchronise and,
+ *    after the call that allocates, creates nothing: all device memory, the
+ *    cache's own streams and its events come from xsv_cache_set_options with
+ *    max_frame_tokens > 0, else from the first step (or the first import).
+ *    Exceptions, each made once and outside the frame loop if wanted so: the
+ *    first xsv_step_host call allocates the staging slots and two copy
+ *    streams; profiling (off by default) creates events as it needs them.
  *  - All steps of one cache share scratch buffers: issue them on one stream
  *    (or order them yourself).  Each layer is stepped once per frame, frames
  *    in order; layers may be stepped in any order.
- *  - Lengths never need a device read-back: the cache length after a step is
- *    a closed-form function of the step count, n_tokens and the budget.
+ *  - Lengths never need a device read-back: the cache length after a step
+ *    follows on the host from the length before it, the sizes of the first
+ *    and of the current frame, and the budget (see xsv_cache_len).
  */
 #ifndef XSV_H
 #define XSV_H
@@ -46,12 +57,12 @@ typedef struct xsv_cache xsv_cache; /* opaque, library-owned */
 typedef enum {
     XSV_OK = 0,
     XSV_ERR_ARG = 1,     /* null pointer, value out of range                          */
-    XSV_ERR_SHAPE = 2,   /* n_tokens / dtype differ from the first step, bad alignment */
+    XSV_ERR_SHAPE = 2,   /* n_tokens beyond max_frame_tokens, dtype differs, bad alignment */
     XSV_ERR_ORDER = 3,   /* options changed after the first step, layer stepped twice  */
     XSV_ERR_OOM = 4,     /* device or host allocation failed                          */
     XSV_ERR_CUDA = 5,    /* a CUDA runtime call failed                                */
     XSV_ERR_TIMEOUT = 6, /* a bounded device-side wait ran out (status word)          */
-    XSV_ERR_RANGE = 7,   /* a zero-point left the int32 range (status word)           */
+    XSV_ERR_RANGE = 7,   /* a zero-point left int32, or an input the fp16 range (status word) */
     XSV_ERR_CAPACITY = 8,/* unbounded cache grew past max_cache_tokens                */
     XSV_ERR_LIMIT = 9    /* size beyond the fixed maximum of a no-allocation entry point */
 } xsv_status;
@@ -88,8 +99,10 @@ xsv_status xsv_cache_create(xsv_cache** out, int layers, int heads, int head_dim
  *                      kept un-pooled by the query pooling (Eq. 3).  Default 5.
  *   pool_group       : g, patch tokens averaged per pooled query (Eq. 3).  Default 16.
  *   quant_group      : G, quantisation group size (section 4.1).  Must be 64.
- *   max_frame_tokens : tokens per frame F if known (allocates now); 0: learnt
- *                      from the first step.
+ *   max_frame_tokens : the most tokens any frame will hold (frames may differ
+ *                      in size: inputs resized to a maximum edge, section 4.1);
+ *                      allocates now.  0: the first frame's size, i.e. no
+ *                      later frame may be larger than the first.
  *   max_cache_tokens : capacity in tokens for an unbounded cache
  *                      (budget_tokens <= 0); ignored otherwise.  Default 16 frames.
  * A negative value leaves a setting unchanged.
@@ -97,17 +110,20 @@ xsv_status xsv_cache_create(xsv_cache** out, int layers, int heads, int head_dim
 xsv_status xsv_cache_set_options(xsv_cache* c, int n_special, int pool_group, int quant_group,
                                  int max_frame_tokens, long long max_cache_tokens);
 
-/* Select the attention kernel (default XSV_ATTN_AUTO). */
+/* Select the attention kernel (default XSV_ATTN_AUTO); both compute Eq. 2 with Eq. 12 fused. */
 xsv_status xsv_cache_set_attn_impl(xsv_cache* c, xsv_attn_impl impl);
 
 /*
  * One streaming step of layer `layer` (Fig. 2; Eq. 2-12).
  *   Q, K, V : device, the new frame's queries / keys / values.
- *   n_tokens: F; must equal the first step's.
+ *   n_tokens: tokens of this frame (T_current of Eq. 8); at most
+ *             max_frame_tokens, XSV_ERR_SHAPE beyond.  The first frame's size
+ *             is T_first; Eq. 8 keeps k = max(0, L_max - T_first - T_current)
+ *             tokens of the middle segment.
  *   out     : device, receives softmax(Q [K~cache ; K]^T / sqrt(head_dim)) [V~cache ; V].
  *   stream  : cudaStream_t (as void*); NULL is the default stream.
  * Afterwards the layer's cache holds [first frame ; kept middle ; this frame],
- * quantised, of length min-closed-form (see xsv_cache_len).
+ * quantised (see xsv_cache_len for its length).
  * Everything is enqueued; nothing synchronises with the host.  A step that
  * prunes runs its selection and re-quantisation kernels (Eq. 8-11, which need
  * the scores but not the attention output) on streams the cache owns, beside
@@ -132,6 +148,7 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
  * xsv_step on the same layer or an xsv_cache_join, and so must not be freed or
  * overwritten earlier; `out` is complete in `stream` order as always.
  * xsv_cache_join makes `stream` wait for all outstanding side-stream work.
+ * (How the launches are ordered is the library's; the paper has no counterpart.)
  */
 xsv_status xsv_cache_set_deferred_join(xsv_cache* c, int on);
 xsv_status xsv_cache_join(xsv_cache* c, void* stream);
@@ -149,16 +166,20 @@ xsv_status xsv_cache_join(xsv_cache* c, void* stream);
  *   second internal stream and the next step does not wait for it: `out_host`
  *   is complete once `stream` has passed a later xsv_cache_host_flush(c, stream)
  *   (at most two results are in flight; a third call waits for the first).
+ * The first call allocates the staging slots (sized for max_frame_tokens) and
+ * creates the copy streams; later calls allocate nothing.  (Host staging is
+ * the library's; the paper has no counterpart.)
  */
 xsv_status xsv_step_host(xsv_cache* c, int layer, const void* Q_host, const void* K_host,
                          const void* V_host, int n_tokens, xsv_dtype dtype, void* out_host,
                          void* stream);
 
 /* Deferred copy-back of xsv_step_host results (see there); off by default.
- * XSV_ERR_ORDER while results are in flight (flush first). */
+ * XSV_ERR_ORDER while results are in flight (flush first).  (No counterpart in the paper.) */
 xsv_status xsv_cache_set_host_pipelining(xsv_cache* c, int defer_output);
 
-/* Makes `stream` wait for every result of xsv_step_host still on its way to the host. */
+/* Makes `stream` wait for every result of xsv_step_host still on its way to the host.
+ * (No counterpart in the paper.) */
 xsv_status xsv_cache_host_flush(xsv_cache* c, void* stream);
 
 /*
@@ -227,10 +248,14 @@ size_t xsv_cache_layer_kv_bytes(const xsv_cache* c, int layer);
 
 void xsv_cache_destroy(xsv_cache* c);
 
-/* Tokens currently cached in `layer` (host-side closed form; no device read). */
+/* Tokens currently cached in `layer`, kept on the host without a device read
+ * (section 3.2's trigger rule and Eq. 8): after a step on a cache of T_c tokens
+ * with a frame of F tokens it is T_c + F if this was the layer's first step,
+ * the cache is unbounded or T_c + F <= L_max; else
+ * T_first + max(0, L_max - T_first - F) + F = max(L_max, T_first + F). */
 long long xsv_cache_len(const xsv_cache* c, int layer);
 
-/* Frames stepped so far in `layer`. */
+/* Frames stepped so far in `layer` (bookkeeping; the paper has no counterpart). */
 long long xsv_cache_frames(const xsv_cache* c, int layer);
 
 /*
@@ -239,7 +264,8 @@ long long xsv_cache_frames(const xsv_cache* c, int layer);
  *   k_codes, v_codes : unsigned char [H][T][d], one code per byte (bits < 16);
  *   k_scale / k_zero : float / int [H][ceil(T/64)][d]  (Eq. 10, per channel per 64-token group);
  *   v_scale / v_zero : float / int [H][T]              (per token);
- *   origin           : long long [T], frame_index * F + token_index of each slot;
+ *   origin           : long long [T], the running index in the stream of the token in each slot
+ *                      (tokens of all earlier frames + its index in its frame);
  *   k_raw, v_raw     : unsigned short [H][T][d], the 16-bit cache when bits == 16.
  */
 xsv_status xsv_cache_export_layer(xsv_cache* c, int layer, unsigned char* k_codes, float* k_scale,
@@ -250,15 +276,18 @@ xsv_status xsv_cache_export_layer(xsv_cache* c, int layer, unsigned char* k_code
 /*
  * The inverse of xsv_cache_export_layer: load one layer's logical state from
  * HOST arrays (checkpoint restore; also the way to continue a stream on another
- * cache object).  Synchronises `stream`.
+ * cache object; the paper has no counterpart).  Synchronises `stream`.
  *   n_cached     : T, tokens in the arrays; at most the cache's capacity
- *                  (max(budget, 2 * frame_tokens), or max_cache_tokens when unbounded).
+ *                  (max(budget, 2 * max_frame_tokens), or max_cache_tokens when unbounded).
  *   frames_done  : frames this layer has been stepped with (the next step is
  *                  frame frames_done + 1; all layers must agree before stepping on).
- *   frame_tokens, dtype : F and the element type of the stream (fixed per cache).
+ *   frame_tokens : T_first, the tokens of the layer's first frame (they head the arrays);
+ *                  also max_frame_tokens if that was not set before.
+ *   dtype        : the element type of the stream (fixed per cache).
  *   arrays       : as in xsv_cache_export_layer (codes one per byte, < 2^bits;
  *                  k_raw / v_raw instead when bits == 16); `origin` is required.
- * Errors leave the cache unchanged, except XSV_ERR_CUDA.
+ * Every array is validated before anything is written: errors leave the cache
+ * unchanged, except XSV_ERR_CUDA.
  */
 xsv_status xsv_cache_import_layer(xsv_cache* c, int layer, long long n_cached, long long frames_done,
                                   int frame_tokens, xsv_dtype dtype, const unsigned char* k_codes,
@@ -294,7 +323,9 @@ int xsv_cache_status_word(xsv_cache* c, void* stream);
  * none.  xsv_cache_profile_read
  * synchronises the recorded events, adds their durations to per-phase totals,
  * and returns the totals (milliseconds) and launch counts accumulated since
- * the last reset. */
+ * the last reset.  Events are created when profiling is switched on and, if
+ * more phases are recorded between two reads than that pool holds, on demand.
+ * (Measurement support; the paper has no counterpart.) */
 xsv_status xsv_cache_set_profiling(xsv_cache* c, int on);
 xsv_status xsv_cache_profile_read(xsv_cache* c, double ms[XSV_PHASE_COUNT], long long launches[XSV_PHASE_COUNT], int reset);
 
@@ -308,14 +339,24 @@ xsv_status xsv_cache_profile_read(xsv_cache* c, double ms[XSV_PHASE_COUNT], long
  */
 xsv_status xsv_selftest_bounded_wait(void* stream);
 
-/* Kernels launched by this library in the calling process since load. */
+/*
+ * Host-only self-test of the table in which the library keeps what it has
+ * configured per CUDA device (opt-in shared memory of a kernel, occupancy,
+ * multiprocessor count): slots of different devices are independent, and
+ * device indices beyond the table are never cached.  Needs no GPU; returns 0
+ * when the table behaves.  (The paper has no counterpart.)
+ */
+int xsv_selftest_device_table(void);
+
+/* Kernels launched by this library in the calling process since load (the paper has no counterpart). */
 long long xsv_kernel_launches(void);
 
+/* Text for a status code (the paper has no counterpart). */
 const char* xsv_strerror(xsv_status s);
 
 /* Text of the CUDA runtime error behind the calling thread's most recent
  * XSV_ERR_CUDA from xsv_step / xsv_step_host / xsv_importance_scores
- * ("no error" if there was none).  The pointer is to static storage. */
+ * ("no error" if there was none).  The pointer is to static storage.  (No counterpart in the paper.) */
 const char* xsv_last_cuda_error(void);
 
 #ifdef __cplusplus

@@ -201,7 +201,9 @@ class LayerCache:
     [H, ceil(T/G), d] (per channel, groups of G consecutive tokens, Eq. 11);
     Vs float32 / Vz int32 [H, T, d/G] (per token, groups of G channels).
     bits == 16: quantisation off, Kc/Vc hold the 16-bit inputs as float32.
-    origin[T] = frame_index * F + token_index of the token in each slot.
+    origin[T] = running index of the token in the stream (tokens of all earlier frames + its index in its
+    frame; frame_index * F + token_index when every frame holds F tokens) -- a label by which kept sets
+    are compared, not part of the method's arithmetic.
     L_max <= 0 means unbounded (no pruning)."""
 
     def __init__(self, H, d, L_max, bits, n_special=5, g=16, G=64):
@@ -211,6 +213,7 @@ class LayerCache:
         self.n_special, self.g, self.G = n_special, g, G
         self.t = 0
         self.F_first = 0
+        self.tokens_seen = 0
         self.T = 0
         cdt = F32 if bits == 16 else np.uint8
         self.Kc = np.zeros((H, 0, d), cdt)
@@ -282,7 +285,8 @@ class LayerCache:
         T_new = keep.shape[0]
         assert np.all(keep[n_old:] == np.arange(T_c, T))
         origin_new = np.concatenate(
-            [self.origin[from_cache], (self.t - 1) * Fc + np.arange(Fc, dtype=np.int64)])
+            [self.origin[from_cache], self.tokens_seen + np.arange(Fc, dtype=np.int64)])
+        self.tokens_seen += Fc
 
         if self.bits == 16:
             self.Kc = np.concatenate([self.Kc[:, from_cache], K], axis=1)
@@ -335,6 +339,7 @@ class LayerCache:
         self.Ks, self.Kz = np.asarray(Ks, F32), np.asarray(Kz, np.int32)
         self.Vs, self.Vz = np.asarray(Vs, F32), np.asarray(Vz, np.int32)
         self.origin = np.asarray(origin, np.int64)
+        self.tokens_seen = int(self.origin[-1]) + 1 if self.T else 0     # the last frame's last token is always kept
 
     def kv_bytes_packed(self):
         """Bytes of the packed representation: b-bit codes + float32 scale +
@@ -353,3 +358,12 @@ def expected_cache_len(t, F, L_max):
     if t == 1 or L_max <= 0 or T <= L_max:
         return T
     return max(L_max, 2 * F)
+
+
+def next_cache_len(t, T_c, F_first, F_t, L_max):
+    """Cache length after step t (1-based) that appends a frame of F_t tokens to a cache of T_c tokens whose
+    first frame holds F_first: the trigger rule of section 3.2 and the size of Eq. 8's keep set."""
+    T = T_c + F_t
+    if t == 1 or L_max <= 0 or T <= L_max:
+        return T
+    return F_first + max(0, L_max - F_first - F_t) + F_t

@@ -45,6 +45,7 @@ SYMBOLS = {
     "xsv_cache_set_profiling": (_i, [_vp, _i]),
     "xsv_cache_profile_read": (_i, [_vp, C.POINTER(C.c_double), C.POINTER(_ll), _i]),
     "xsv_selftest_bounded_wait": (_i, [_vp]),
+    "xsv_selftest_device_table": (_i, []),
     "xsv_kernel_launches": (_ll, []),
     "xsv_strerror": (C.c_char_p, [_i]),
     "xsv_last_cuda_error": (C.c_char_p, []),

@@ -1090,16 +1090,6 @@ __global__ void wait_selftest_kernel(int* status) {
     mbar_wait(smem_u32(&bar), 0u, &abort_flag, status, XSV_DEV_SITE_SELFTEST);
 }
 
-int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-            n = 148;
-    }
-    return n;
-}
-
 template <typename T, int BITS>
 cudaError_t launch(const Params& p, bool merge_only, cudaStream_t st) {
     if (merge_only) {
@@ -1107,11 +1097,12 @@ cudaError_t launch(const Params& p, bool merge_only, cudaStream_t st) {
         xsv_count_launch(1);
         return cudaGetLastError();
     }
-    static bool attr_set = false;
-    if (!attr_set) {
+    static XsvPerDeviceInt attr_set;      // the opt-in to large dynamic shared memory holds per device
+    const int dev = xsv_current_device();
+    if (!attr_set.get(dev)) {
         cudaError_t e = cudaFuncSetAttribute(attn_tc5_kernel<T, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        attr_set.set(dev, 1);
     }
     xsv_launch_dep(attn_tc5_kernel<T, BITS>, dim3(p.G), dim3(NTHREADS), SMEM_BYTES, st, p);
     xsv_count_launch(1);
@@ -1126,7 +1117,7 @@ cudaError_t xsv_launch_wait_selftest(int* status, cudaStream_t st) {
     return cudaGetLastError();
 }
 
-size_t xsv_attn_tc5_workspace_bytes() { return (size_t)sm_count() * 2 * PART_STRIDE * sizeof(float); }
+size_t xsv_attn_tc5_workspace_bytes() { return (size_t)xsv_sm_count() * 2 * PART_STRIDE * sizeof(float); }
 
 namespace {
 cudaError_t launch_tc5(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V, void* out,
@@ -1143,7 +1134,7 @@ cudaError_t launch_tc5(const LayerView& lv, int T_c, const void* Q, const void* 
     p.ticks_head = p.n_full * unit_len(p, true) + (p.npair - p.n_full) * unit_len(p, false);
     p.total = p.ticks_head * H;
     const long long steps = (long long)H * p.npair * p.nkv;
-    const int sms = sm_count() - spare_sms > 0 ? sm_count() - spare_sms : 1;   // multiprocessors left to another kernel
+    const int sms = xsv_sm_count() - spare_sms > 0 ? xsv_sm_count() - spare_sms : 1;   // multiprocessors left to another kernel
     p.G = (int)(steps < sms ? steps : sms);
     if (p.G > MAX_PARTS) p.G = MAX_PARTS;
 #define XSV_TC5(TT, B) return launch<TT, B>(p, merge_only, st)

@@ -1116,13 +1116,22 @@ bool xsv_dep_launch_enabled() {
     return on;
 }
 
+int xsv_current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return -1;
+    }
+    return dev;
+}
+
 int xsv_sm_count() {
-    static int n = 0;
+    static XsvPerDeviceInt table;
+    const int dev = xsv_current_device();
+    int n = table.get(dev);
     if (n == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
-            n = 148;
+        if (dev < 0 || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        table.set(dev, n);
     }
     return n;
 }
@@ -1146,11 +1155,12 @@ cudaError_t xsv_launch_score(const LayerView& lv, int H, int T_first, int T_c, c
     cudaError_t e = cudaSuccess;
 #define XSV_SCORE(B)                                                                                       \
     {                                                                                                      \
-        static bool attr_set = false;                                                                      \
-        if (!attr_set && smem > 48 * 1024) {                                                               \
+        static XsvPerDeviceInt attr_set;   /* largest opt-in size configured per device */               \
+        const int dev = xsv_current_device();                                                              \
+        if (smem > 48 * 1024 && attr_set.get(dev) < (int)smem) {                                           \
             e = cudaFuncSetAttribute(score_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
             if (e != cudaSuccess) return e;                                                                \
-            attr_set = true;                                                                               \
+            attr_set.set(dev, (int)smem);                                                                  \
         }                                                                                                  \
         xsv_launch_dep(score_kernel<B>, dim3(grid), dim3(SCORE_TPB), smem, st, lv, H, T_first, T_c, qpart, qnorm, scores); \
     }
@@ -1180,12 +1190,13 @@ cudaError_t xsv_launch_select(const float* scores, int n, int k, int T_first, in
                               cudaStream_t st) {
 #define XSV_SEL(KPT)                                                                                             \
     {                                                                                                            \
-        static bool attr_set = false;                                                                            \
-        if (!attr_set) {                                                                                         \
+        static XsvPerDeviceInt attr_set;                                                                         \
+        const int dev = xsv_current_device();                                                                    \
+        if (!attr_set.get(dev)) {                                                                                \
             cudaError_t e = cudaFuncSetAttribute(select_reg_kernel<KPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
                                                  1024 * KPT * 4);                                                \
             if (e != cudaSuccess) return e;                                                                      \
-            attr_set = true;                                                                                     \
+            attr_set.set(dev, 1);                                                                                \
         }                                                                                                        \
         xsv_launch_dep(select_reg_kernel<KPT>, dim3(1), dim3(1024), 1024 * KPT * 4, st, scores, n, k, T_first, T_c, srcmap, dscal); \
     }
@@ -1214,12 +1225,15 @@ cudaError_t xsv_launch_compress(const LayerView& src, const LayerView& dst, cons
 #define XSV_RQ(TT, B)                                                                                                \
     {                                                                                                                \
         const size_t smem = (size_t)wpb * RqCfg<B>::WORDS * 4;                                                       \
-        static int per_sm = 0;   /* resident blocks per multiprocessor: the grid is one wave of them */              \
+        static XsvPerDeviceInt per_sm_of;   /* resident blocks per multiprocessor: the grid is one wave of them */   \
+        const int dev = xsv_current_device();                                                                        \
+        int per_sm = per_sm_of.get(dev);                                                                             \
         if (per_sm == 0) {                                                                                           \
             cudaFuncSetAttribute(requant_k_kernel<TT, B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);   \
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, requant_k_kernel<TT, B>, RQ_THREADS, smem) != \
                     cudaSuccess || per_sm <= 0)                                                                      \
                 per_sm = 2;                                                                                          \
+            per_sm_of.set(dev, per_sm);                                                                              \
         }                                                                                                            \
         const int grid = min((n_all + wpb - 1) / wpb, xsv_sm_count() * per_sm);                                      \
         xsv_launch_dep(requant_k_kernel<TT, B>, dim3(grid), dim3(RQ_THREADS), smem, st, src, dst, (const TT*)Kf,     \

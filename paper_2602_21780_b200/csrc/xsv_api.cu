@@ -43,7 +43,7 @@ struct xsv_cache {
     int layers = 0, H = 0, d = 0, bits = 0;
     long long L_max = 0;
     int n_special = 5, g = 16, G = 64;
-    int F = 0;               // tokens per frame (0 until known)
+    int F_max = 0;           // most tokens a frame may hold (0 until known: set_options, or the first frame's size)
     int dtype = -1;          // xsv_dtype of the first step
     long long max_cache_tokens = 0;
     long long cap = 0;       // capacity in tokens of each buffer set
@@ -55,6 +55,8 @@ struct xsv_cache {
     std::vector<int> buf_of_layer;
     int spare = 0;
     std::vector<long long> len, frames;
+    std::vector<long long> tokens_seen;   // per layer: tokens of all frames so far (the origin of the next frame's first token)
+    std::vector<int> F_first;             // per layer: tokens of its first frame (T_first of Eq. 8), 0 before the first step
 
     // scratch shared by all layers (steps are ordered on one stream)
     float* qpart = nullptr;
@@ -79,6 +81,7 @@ struct xsv_cache {
     std::vector<char> side_pending;                         // per layer: the caller's stream has not yet waited for those
     cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_done[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
     bool slot_used[2] = {false, false}, out_pending[2] = {false, false};
+    bool slot_deferred[2] = {false, false};                 // the step that last read the slot left side-stream work outstanding
     int slot_layer[2] = {0, 0};                             // the layer whose step last read the slot
     bool defer_output = false;
     unsigned long long host_calls = 0;
@@ -109,9 +112,36 @@ size_t bufset_bytes(const xsv_cache* c, long long cap, size_t off[7]) {
     return o;
 }
 
+void release_device_memory(xsv_cache* c) {
+    for (auto& b : c->bufs) if (b.slab) cudaFree(b.slab);
+    c->bufs.clear();
+    if (c->scratch_slab) cudaFree(c->scratch_slab);
+    c->scratch_slab = nullptr;
+}
+
+// Streams and events of the cache: created once, with the device memory, so that no later step creates any.
+cudaError_t create_streams_and_events(xsv_cache* c) {
+    cudaError_t e;
+    if ((e = cudaStreamCreateWithFlags(&c->cs_sel, cudaStreamNonBlocking)) != cudaSuccess) return e;
+    if ((e = cudaStreamCreateWithFlags(&c->cs_val, cudaStreamNonBlocking)) != cudaSuccess) return e;
+    cudaEvent_t* single[4] = {&c->ev_scored, &c->ev_selected, &c->ev_picked, &c->ev_values};
+    for (cudaEvent_t* ev : single)
+        if ((e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming)) != cudaSuccess) return e;
+    c->ev_keys_of.assign(c->layers, nullptr);
+    c->ev_vals_of.assign(c->layers, nullptr);
+    c->side_pending.assign(c->layers, 0);
+    for (int l = 0; l < c->layers; ++l) {
+        if ((e = cudaEventCreateWithFlags(&c->ev_keys_of[l], cudaEventDisableTiming)) != cudaSuccess) return e;
+        if ((e = cudaEventCreateWithFlags(&c->ev_vals_of[l], cudaEventDisableTiming)) != cudaSuccess) return e;
+    }
+    return cudaSuccess;
+}
+
+// All device memory of the cache (and its streams and events).  Capacity: a bounded cache never holds more than
+// max(L_max, first frame + current frame) tokens, and neither frame exceeds F_max.
 xsv_status allocate(xsv_cache* c) {
     if (c->allocated) return XSV_OK;
-    const long long F = c->F;
+    const long long F = c->F_max;
     long long cap;
     if (c->L_max > 0) cap = c->L_max > 2 * F ? c->L_max : 2 * F;
     else cap = c->max_cache_tokens > 0 ? c->max_cache_tokens : 16 * F;
@@ -121,14 +151,14 @@ xsv_status allocate(xsv_cache* c) {
     size_t off[7];
     const size_t per = bufset_bytes(c, cap, off);
     const int nb = c->layers + (c->L_max > 0 ? 1 : 0);
-    c->bufs.resize(nb);
+    c->bufs.assign(nb, BufSet{});
     size_t total = 0;
     for (int i = 0; i < nb; ++i) {
         void* p = nullptr;
-        if (cudaMalloc(&p, per) != cudaSuccess) { cudaGetLastError(); return XSV_ERR_OOM; }
-        if (cudaMemset(p, 0, per) != cudaSuccess) return XSV_ERR_CUDA;
+        if (cudaMalloc(&p, per) != cudaSuccess) { cudaGetLastError(); release_device_memory(c); return XSV_ERR_OOM; }
+        c->bufs[i].slab = p;
+        if (cudaMemset(p, 0, per) != cudaSuccess) { release_device_memory(c); return XSV_ERR_CUDA; }
         BufSet& b = c->bufs[i];
-        b.slab = p;
         uint8_t* base = (uint8_t*)p;
         b.view.kcodes = base + off[0];
         b.view.vcodes = base + off[1];
@@ -154,8 +184,8 @@ xsv_status allocate(xsv_cache* c) {
     const size_t o_d = so; so = align_up(so + 64, 256);
     const size_t o_t = so; so = align_up(so + 64, 256);
     const size_t o_w = so; so = align_up(so + xsv_attn_tc5_workspace_bytes(), 256);
-    if (cudaMalloc(&c->scratch_slab, so) != cudaSuccess) { cudaGetLastError(); return XSV_ERR_OOM; }
-    if (cudaMemset(c->scratch_slab, 0, so) != cudaSuccess) return XSV_ERR_CUDA;
+    if (cudaMalloc(&c->scratch_slab, so) != cudaSuccess) { cudaGetLastError(); release_device_memory(c); return XSV_ERR_OOM; }
+    if (cudaMemset(c->scratch_slab, 0, so) != cudaSuccess) { release_device_memory(c); return XSV_ERR_CUDA; }
     uint8_t* sb = (uint8_t*)c->scratch_slab;
     c->qpart = (float*)(sb + o_q);
     c->scores = (float*)(sb + o_s);
@@ -163,6 +193,10 @@ xsv_status allocate(xsv_cache* c) {
     c->dscal = (int*)(sb + o_d);
     c->status = (int*)(sb + o_t);
     c->attn_ws = (float*)(sb + o_w);
+    if (!c->cs_sel) {
+        const cudaError_t e = create_streams_and_events(c);
+        if (e != cudaSuccess) { release_device_memory(c); g_last_cuda = e; cudaGetLastError(); return XSV_ERR_CUDA; }
+    }
     c->bytes = total + so;
     c->allocated = true;
     return XSV_OK;
@@ -234,7 +268,7 @@ const char* xsv_strerror(xsv_status s) {
         case XSV_ERR_OOM: return "out of memory";
         case XSV_ERR_CUDA: return "CUDA runtime error";
         case XSV_ERR_TIMEOUT: return "bounded device-side wait ran out";
-        case XSV_ERR_RANGE: return "zero-point outside the int32 range";
+        case XSV_ERR_RANGE: return "value outside the supported range (zero-point beyond int32, or a 16-bit input beyond +-65504)";
         case XSV_ERR_CAPACITY: return "unbounded cache exceeded max_cache_tokens";
         case XSV_ERR_LIMIT: return "size exceeds the fixed maximum of this no-allocation entry point";
     }
@@ -259,6 +293,8 @@ xsv_status xsv_cache_create(xsv_cache** out, int layers, int heads, int head_dim
     c->L_max = budget_tokens > 0 ? budget_tokens : 0;
     c->len.assign(layers, 0);
     c->frames.assign(layers, 0);
+    c->tokens_seen.assign(layers, 0);
+    c->F_first.assign(layers, 0);
     *out = c;
     return XSV_OK;
 }
@@ -274,9 +310,11 @@ xsv_status xsv_cache_set_options(xsv_cache* c, int n_special, int pool_group, in
     if (max_cache_tokens >= 0) c->max_cache_tokens = max_cache_tokens;
     if (max_frame_tokens > 0) {
         if (c->n_special > max_frame_tokens) return XSV_ERR_ARG;
-        c->F = max_frame_tokens;
+        c->F_max = max_frame_tokens;
         cudaSetDevice(c->device);
-        return allocate(c);
+        const xsv_status st = allocate(c);
+        if (st != XSV_OK) c->F_max = 0;
+        return st;
     }
     return XSV_OK;
 }
@@ -294,7 +332,7 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
     if (dtype != XSV_F16 && dtype != XSV_BF16) return XSV_ERR_ARG;
     if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)out) & 15) return XSV_ERR_SHAPE;
     if (out == Q || out == K || out == V) return XSV_ERR_ARG;
-    if (c->F != 0 && n_tokens != c->F) return XSV_ERR_SHAPE;
+    if (c->F_max != 0 && n_tokens > c->F_max) return XSV_ERR_SHAPE;   // frames may differ in size up to max_frame_tokens
     if (c->dtype >= 0 && (int)dtype != c->dtype) return XSV_ERR_SHAPE;
     if (c->n_special > n_tokens) return XSV_ERR_ARG;
     long long min_frames = c->frames[0];
@@ -303,12 +341,12 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
 
     cudaStream_t st = (cudaStream_t)stream;
     if (!c->allocated) {
-        c->F = n_tokens;
+        c->F_max = n_tokens;          // not told otherwise: no later frame is larger than the first
         cudaSetDevice(c->device);
         xsv_status s = allocate(c);
-        if (s != XSV_OK) { c->F = 0; return s; }
+        if (s != XSV_OK) { c->F_max = 0; return s; }
     }
-    const int F = c->F, H = c->H;
+    const int F = n_tokens, H = c->H;
     const long long T_c = c->len[layer];
     const long long T = T_c + F;
     const long long t = c->frames[layer] + 1;
@@ -321,8 +359,10 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
     const LayerView& lv = c->bufs[cur].view;
     cudaError_t e;
 
-    const long long origin0 = (t - 1) * (long long)F;
-    const int T_first = F;   // constant frame size: the first frame holds F tokens
+    // Eq. 8 with the sizes of the first and of the current frame as separate quantities:
+    // k = max(0, L_max - T_first - T_current) of the middle segment's T_c - T_first tokens are kept.
+    const long long origin0 = c->tokens_seen[layer];
+    const int T_first = t == 1 ? F : c->F_first[layer];
     const int n_mid = (int)(T_c - T_first);
     const long long kk = c->L_max - T_first - F;
     const int k = (int)(kk > 0 ? kk : 0);
@@ -356,21 +396,6 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
         }
         cudaStream_t sel_st = st;
         if (side_select) {
-            if (!c->cs_sel) {
-                if ((e = cudaStreamCreateWithFlags(&c->cs_sel, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
-                if ((e = cudaEventCreateWithFlags(&c->ev_scored, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
-                if ((e = cudaEventCreateWithFlags(&c->ev_selected, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
-                if ((e = cudaStreamCreateWithFlags(&c->cs_val, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
-                if ((e = cudaEventCreateWithFlags(&c->ev_picked, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
-                if ((e = cudaEventCreateWithFlags(&c->ev_values, cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
-                c->ev_keys_of.assign(c->layers, nullptr);
-                c->ev_vals_of.assign(c->layers, nullptr);
-                c->side_pending.assign(c->layers, 0);
-                for (int l = 0; l < c->layers; ++l) {
-                    if ((e = cudaEventCreateWithFlags(&c->ev_keys_of[l], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
-                    if ((e = cudaEventCreateWithFlags(&c->ev_vals_of[l], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
-                }
-            }
             // the new selection overwrites the kept-position map that the values of the previous step may still read
             if (c->defer_join && (e = cudaStreamWaitEvent(c->cs_sel, c->ev_values, 0)) != cudaSuccess) return cuda_fail(e);
             if ((e = cudaEventRecord(c->ev_scored, st)) != cudaSuccess) return cuda_fail(e);
@@ -472,6 +497,8 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
         c->last_scores_n = 0;
     }
     c->frames[layer] = t;
+    c->tokens_seen[layer] = origin0 + F;
+    if (t == 1) c->F_first[layer] = F;
     return XSV_OK;
 }
 
@@ -501,19 +528,18 @@ xsv_status xsv_cache_join(xsv_cache* c, void* stream) {
 xsv_status xsv_step_host(xsv_cache* c, int layer, const void* Qh, const void* Kh, const void* Vh, int n_tokens,
                          xsv_dtype dtype, void* out_h, void* stream) {
     if (!c || !Qh || !Kh || !Vh || !out_h || n_tokens <= 0) return XSV_ERR_ARG;
-    if (c->F != 0 && n_tokens != c->F) return XSV_ERR_SHAPE;
+    if (c->F_max != 0 && n_tokens > c->F_max) return XSV_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
-    const size_t nb = (size_t)c->H * n_tokens * c->d * 2;
     cudaError_t e = cudaSuccess;
-    if (c->stage_bytes < 8 * nb) {
+    if (!c->stage) {
+        // First call: the staging slots (sized for the largest frame), two copy streams and their events.  This is the
+        // only call of the host path that allocates; make it before the frame loop.
+        const int F_stage = c->F_max != 0 ? c->F_max : n_tokens;
+        const size_t nb_max = (size_t)c->H * F_stage * c->d * 2;
         cudaSetDevice(c->device);
-        if (c->stage) { cudaDeviceSynchronize(); cudaFree(c->stage); c->bytes -= c->stage_bytes; c->stage = nullptr; c->stage_bytes = 0; }
-        if (cudaMalloc(&c->stage, 8 * nb) != cudaSuccess) { cudaGetLastError(); return XSV_ERR_OOM; }
-        c->stage_bytes = 8 * nb;
+        if (cudaMalloc(&c->stage, 8 * nb_max) != cudaSuccess) { cudaGetLastError(); c->stage = nullptr; return XSV_ERR_OOM; }
+        c->stage_bytes = 8 * nb_max;
         c->bytes += c->stage_bytes;
-        c->slot_used[0] = c->slot_used[1] = c->out_pending[0] = c->out_pending[1] = false;
-    }
-    if (!c->cs_in) {
         if ((e = cudaStreamCreateWithFlags(&c->cs_in, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
         if ((e = cudaStreamCreateWithFlags(&c->cs_out, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(e);
         for (int i = 0; i < 2; ++i) {
@@ -522,36 +548,42 @@ xsv_status xsv_step_host(xsv_cache* c, int layer, const void* Qh, const void* Kh
             if ((e = cudaEventCreateWithFlags(&c->ev_out[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(e);
         }
     }
+    const size_t nb = (size_t)c->H * n_tokens * c->d * 2;          // this frame's bytes per tensor
+    const size_t slot_bytes = c->stage_bytes / 2, part = slot_bytes / 4;
+    if (nb > part) return XSV_ERR_SHAPE;
     // Two staging slots alternate.  The inputs of this call are copied on a stream of their own, as soon as the
     // step that last used the slot has finished, so the copy overlaps the previous call's kernels.
     const int slot = (int)(c->host_calls & 1ull);
-    uint8_t* s = (uint8_t*)c->stage + (size_t)slot * 4 * nb;
+    uint8_t* s = (uint8_t*)c->stage + (size_t)slot * slot_bytes;
     if (c->slot_used[slot] && (e = cudaStreamWaitEvent(c->cs_in, c->ev_done[slot], 0)) != cudaSuccess) return cuda_fail(e);
-    if (c->slot_used[slot] && !c->side_pending.empty() && c->side_pending[c->slot_layer[slot]]) {
-        // deferred join: that step's side-stream kernels may still be reading the staged K and V
+    if (c->slot_used[slot] && c->slot_deferred[slot]) {
+        // Deferred join: the side-stream kernels of the step that read this slot may still be reading the staged K and
+        // V.  Their events are waited for whatever the caller's stream has joined since (a join makes only that stream
+        // wait, not this copy stream).
         if ((e = cudaStreamWaitEvent(c->cs_in, c->ev_keys_of[c->slot_layer[slot]], 0)) != cudaSuccess) return cuda_fail(e);
         if ((e = cudaStreamWaitEvent(c->cs_in, c->ev_vals_of[c->slot_layer[slot]], 0)) != cudaSuccess) return cuda_fail(e);
     }
     if ((e = cudaMemcpyAsync(s, Qh, nb, cudaMemcpyHostToDevice, c->cs_in)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaMemcpyAsync(s + nb, Kh, nb, cudaMemcpyHostToDevice, c->cs_in)) != cudaSuccess) return cuda_fail(e);
-    if ((e = cudaMemcpyAsync(s + 2 * nb, Vh, nb, cudaMemcpyHostToDevice, c->cs_in)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(s + part, Kh, nb, cudaMemcpyHostToDevice, c->cs_in)) != cudaSuccess) return cuda_fail(e);
+    if ((e = cudaMemcpyAsync(s + 2 * part, Vh, nb, cudaMemcpyHostToDevice, c->cs_in)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaEventRecord(c->ev_in[slot], c->cs_in)) != cudaSuccess) return cuda_fail(e);
     if ((e = cudaStreamWaitEvent(st, c->ev_in[slot], 0)) != cudaSuccess) return cuda_fail(e);
     if (c->out_pending[slot]) {   // the slot's previous result must have left before the step overwrites it
         if ((e = cudaStreamWaitEvent(st, c->ev_out[slot], 0)) != cudaSuccess) return cuda_fail(e);
         c->out_pending[slot] = false;
     }
-    xsv_status r = xsv_step(c, layer, s, s + nb, s + 2 * nb, n_tokens, dtype, s + 3 * nb, stream);
+    xsv_status r = xsv_step(c, layer, s, s + part, s + 2 * part, n_tokens, dtype, s + 3 * part, stream);
     if (r != XSV_OK) return r;
     ++c->host_calls;
     c->slot_used[slot] = true;
     c->slot_layer[slot] = layer;
+    c->slot_deferred[slot] = !c->side_pending.empty() && c->side_pending[layer] != 0;
     if ((e = cudaEventRecord(c->ev_done[slot], st)) != cudaSuccess) return cuda_fail(e);
     if (!c->defer_output) {
-        if ((e = cudaMemcpyAsync(out_h, s + 3 * nb, nb, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpyAsync(out_h, s + 3 * part, nb, cudaMemcpyDeviceToHost, st)) != cudaSuccess) return cuda_fail(e);
     } else {
         if ((e = cudaStreamWaitEvent(c->cs_out, c->ev_done[slot], 0)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaMemcpyAsync(out_h, s + 3 * nb, nb, cudaMemcpyDeviceToHost, c->cs_out)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaMemcpyAsync(out_h, s + 3 * part, nb, cudaMemcpyDeviceToHost, c->cs_out)) != cudaSuccess) return cuda_fail(e);
         if ((e = cudaEventRecord(c->ev_out[slot], c->cs_out)) != cudaSuccess) return cuda_fail(e);
         c->out_pending[slot] = true;
     }
@@ -599,6 +631,22 @@ xsv_status xsv_importance_scores(const void* Q, const void* keys, int heads, int
     if (e == cudaSuccess) e = xsv_launch_score_raw(lv, (int)dtype, heads, 0, (int)n_keys, qpart, qnorm, scores, st);
     cudaFreeAsync(qpart, st);
     return e == cudaSuccess ? XSV_OK : cuda_fail(e);
+}
+
+int xsv_selftest_device_table(void) {
+    // host-only: the per-device slots are independent, survive other slots' updates, and ignore devices
+    // beyond the table (which then are configured on every launch instead of once)
+    XsvPerDeviceInt t;
+    for (int d = 0; d < XSV_MAX_DEVICES; ++d) if (t.get(d) != 0) return 1;
+    t.set(0, 5);
+    if (t.get(0) != 5 || t.get(1) != 0) return 2;
+    t.set(1, 9);
+    t.set(XSV_MAX_DEVICES - 1, 7);
+    if (t.get(0) != 5 || t.get(1) != 9 || t.get(XSV_MAX_DEVICES - 1) != 7 || t.get(2) != 0) return 3;
+    t.set(XSV_MAX_DEVICES, 11);
+    t.set(-1, 13);
+    if (t.get(XSV_MAX_DEVICES) != 0 || t.get(-1) != 0 || t.get(0) != 5 || t.get(XSV_MAX_DEVICES - 1) != 7) return 4;
+    return 0;
 }
 
 xsv_status xsv_selftest_bounded_wait(void* stream) {
@@ -714,15 +762,23 @@ xsv_status xsv_cache_import_layer(xsv_cache* c, int layer, long long n_cached, l
     if (!c || layer < 0 || layer >= c->layers || n_cached < 0 || frames_done < 0 || frame_tokens <= 0 || !origin) return XSV_ERR_ARG;
     if (dtype != XSV_F16 && dtype != XSV_BF16) return XSV_ERR_ARG;
     if (c->bits == 16 ? (!k_raw || !v_raw) : (!k_codes || !k_scale || !k_zero || !v_codes || !v_scale || !v_zero)) return XSV_ERR_ARG;
-    if (c->F != 0 && frame_tokens != c->F) return XSV_ERR_SHAPE;
+    if (c->F_max != 0 && frame_tokens > c->F_max) return XSV_ERR_SHAPE;
     if (c->dtype >= 0 && (int)dtype != c->dtype) return XSV_ERR_SHAPE;
     if (c->n_special > frame_tokens) return XSV_ERR_ARG;
+    if (n_cached > 0 && n_cached < frame_tokens) return XSV_ERR_ARG;      // the first frame is always in the cache
+    if (c->bits < 16) {
+        // every code is checked before anything is written, so that an error leaves the cache unchanged
+        const unsigned mask = (1u << c->bits) - 1u;
+        const size_t n = (size_t)c->H * (size_t)n_cached * c->d;
+        for (size_t i = 0; i < n; ++i)
+            if (k_codes[i] > mask || v_codes[i] > mask) return XSV_ERR_ARG;
+    }
     cudaStream_t st = (cudaStream_t)stream;
     if (!c->allocated) {
-        c->F = frame_tokens;
+        c->F_max = frame_tokens;
         cudaSetDevice(c->device);
         const xsv_status s = allocate(c);
-        if (s != XSV_OK) { c->F = 0; return s; }
+        if (s != XSV_OK) { c->F_max = 0; return s; }
     }
     if (n_cached > c->cap) return XSV_ERR_CAPACITY;
     if (cudaStreamSynchronize(st) != cudaSuccess || sync_side_streams(c) != cudaSuccess) return XSV_ERR_CUDA;
@@ -744,8 +800,7 @@ xsv_status xsv_cache_import_layer(xsv_cache* c, int layer, long long n_cached, l
                     const unsigned mask = (1u << bits) - 1u;
                     for (long long p = 0; p < T; ++p)
                         for (int ch = 0; ch < d; ++ch) {
-                            const unsigned code = codes[((size_t)h * T + p) * d + ch];
-                            if (code > mask) return XSV_ERR_ARG;
+                            const unsigned code = codes[((size_t)h * T + p) * d + ch] & mask;   // validated above
                             const int bit = ch * bits;
                             tmp[(size_t)p * rowb + bit / 8] |= (uint8_t)(code << (bit % 8));
                         }
@@ -766,6 +821,8 @@ xsv_status xsv_cache_import_layer(xsv_cache* c, int layer, long long n_cached, l
     if (e != cudaSuccess) return cuda_fail(e);
     c->len[layer] = T;
     c->frames[layer] = frames_done;
+    c->F_first[layer] = frames_done > 0 ? frame_tokens : 0;
+    c->tokens_seen[layer] = T > 0 ? origin[T - 1] + 1 : 0;      // the last token of the last frame is always kept
     c->dtype = (int)dtype;
     c->stepped = true;
     return XSV_OK;
@@ -804,6 +861,15 @@ int xsv_cache_status_word(xsv_cache* c, void* stream) {
 xsv_status xsv_cache_set_profiling(xsv_cache* c, int on) {
     if (!c) return XSV_ERR_ARG;
     if (on < 0 || on > 3) return XSV_ERR_ARG;
+    if (on && c->free_events.empty() && c->pending.empty()) {
+        // a pool of timing events, so that the steps that follow create none
+        cudaSetDevice(c->device);
+        for (int i = 0; i < 64 + 16 * c->layers; ++i) {
+            cudaEvent_t e = nullptr;
+            if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); break; }
+            c->free_events.push_back(e);
+        }
+    }
     c->profiling = on;
     return XSV_OK;
 }

@@ -1,10 +1,11 @@
 // Host-side launchers of the xsv kernels (one per phase of the step).
 #pragma once
 #include "xsv_common.cuh"
+#include "xsv_device.h"
 
 // dtype: 0 = fp16, 1 = bf16 (xsv_dtype).
 
-// Multiprocessors of the current device (queried once).
+// Multiprocessors of the current device (queried once per device).
 int xsv_sm_count();
 
 // Eq. 3-4 folded by linearity: per-(head, chunk) partial sums of the pooling-weighted

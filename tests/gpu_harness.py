@@ -34,17 +34,28 @@ def load_oracle_state(ref, st, frames_done, F):
                        st["Vz"][..., None], st["origin"])
 
 
-def check_state_invariants(st, bits, F, frames_done, L_max):
+def check_state_invariants(st, bits, F_first, F_last, tokens_seen, T_expected):
+    """What must hold for any cache state, checked wherever a state is imported into the oracle: its length,
+    ascending origins, the first and the latest frame present in full, codes in range, positive scales."""
     T = st["T"]
-    assert T == orc.expected_cache_len(frames_done, F, L_max)
+    assert T == T_expected
     o = st["origin"]
     assert np.all(np.diff(o) > 0)
-    assert np.array_equal(o[:F], np.arange(F))
-    assert np.array_equal(o[-F:], (frames_done - 1) * F + np.arange(F))
+    assert np.array_equal(o[:F_first], np.arange(F_first))
+    assert np.array_equal(o[-F_last:], tokens_seen - F_last + np.arange(F_last))
     if bits < 16:
         n = (1 << bits) - 1
         assert st["Kc"].max() <= n and st["Vc"].max() <= n
         assert np.all(st["Ks"] > 0) and np.all(st["Vs"] > 0)
+        assert np.all(np.isfinite(st["Ks"])) and np.all(np.isfinite(st["Vs"]))
+        # every stored (s, z) reproduces its group's codes from the values they dequantise to (Eq. 9 after Eq. 12)
+        grp = np.arange(T) // 64
+        for codes, s, z in ((st["Kc"], st["Ks"][:, grp, :], st["Kz"][:, grp, :]),
+                            (st["Vc"], st["Vs"][..., None], st["Vz"][..., None])):
+            x = orc.dequantize(codes, s, z)
+            with np.errstate(over="ignore", invalid="ignore"):
+                back = np.clip(np.rint(x / s.astype(np.float32)).astype(np.int64) + z.astype(np.int64), 0, n)
+            assert np.array_equal(back, codes)
 
 
 def compare_states(st, ref, bits, tag):
@@ -63,32 +74,47 @@ def compare_states(st, ref, bits, tag):
 
 
 def run_stream(stream, frames, L_max, bits, check_steps=None, impl=binding.ATTN_AUTO, n_special=5, g=16,
-               frame_fn=None, max_cache_tokens=-1, layers=1, layer=0, deferred_join=False):
+               frame_fn=None, max_cache_tokens=-1, layers=1, layer=0, deferred_join=False, max_frame_tokens=0,
+               device_fn=None):
     """Run `frames` steps on the GPU; verify the steps in check_steps (0-based; None = all).
+    frame_fn(t) may return frames of different sizes (then max_frame_tokens names the largest).
+    device_fn(t), if given, supplies the inputs of the steps that are not checked as CUDA tensors (long streams:
+    the state a checked step starts from is imported from the GPU, so those inputs need no CPU twin).
     Returns a dict of the worst errors seen."""
-    H, d, F, dtype = stream.H, stream.d, stream.F, stream.dtype
+    H, d, dtype = stream.H, stream.d, stream.dtype
     cache = binding.Cache(layers, H, d, L_max, bits)
     cache.set_attn_impl(impl)
     cache.set_deferred_join(deferred_join)
-    if (n_special, g) != (5, 16) or max_cache_tokens >= 0:
-        cache.set_options(n_special=n_special, pool_group=g, max_cache_tokens=max_cache_tokens)
+    if (n_special, g) != (5, 16) or max_cache_tokens >= 0 or max_frame_tokens > 0:
+        cache.set_options(n_special=n_special, pool_group=g, max_cache_tokens=max_cache_tokens,
+                          max_frame_tokens=max_frame_tokens)
     ref = orc.LayerCache(H, d, L_max, bits, n_special=n_special, g=g)
     ref._dtype = dtype
     worst = dict(attn=0.0, score=0.0, pruned_steps=0, checked=0)
+    F_first, F_prev, tokens_seen, T_expected = 0, 0, 0, 0
     for t in range(frames):
-        q, k, v = frame_fn(t) if frame_fn else stream.frame(t)
-        Q, K, V = to_dev(q, dtype), to_dev(k, dtype), to_dev(v, dtype)
-        out = torch.empty_like(Q)
         checked = check_steps is None or t in check_steps
+        if checked or device_fn is None:
+            q, k, v = frame_fn(t) if frame_fn else stream.frame(t)
+            Q, K, V = to_dev(q, dtype), to_dev(k, dtype), to_dev(v, dtype)
+        else:
+            Q, K, V = device_fn(t)
+        F = Q.shape[1]
+        out = torch.empty_like(Q)
         if checked:
             st0 = cache.export_layer(layer)
             if t > 0:
-                check_state_invariants(st0, bits, F, t, L_max)
-            load_oracle_state(ref, st0, t, F)
+                check_state_invariants(st0, bits, F_first, F_prev, tokens_seen, T_expected)
+            load_oracle_state(ref, st0, t, F_first)
         for l in range(layers):            # other layers take the same inputs; only `layer` is verified
             cache.step(l, Q, K, V, out)
         torch.cuda.synchronize()
-        assert cache.len(layer) == orc.expected_cache_len(t + 1, F, L_max)
+        if t == 0:
+            F_first = F
+        T_expected = orc.next_cache_len(t + 1, T_expected, F_first, F, L_max)
+        tokens_seen += F
+        F_prev = F
+        assert cache.len(layer) == T_expected
         if not checked:
             continue
         S_gpu = cache.last_scores()
@@ -117,3 +143,39 @@ def run_stream(stream, frames, L_max, bits, check_steps=None, impl=binding.ATTN_
     assert worst["kv_bytes"] == ref.kv_bytes_packed()
     cache.destroy()
     return worst
+
+
+def device_stream(H, F, dtype, seed, d=64, pool=4, drift_rho=None):
+    """Inputs for unchecked steps, drawn on the device with the recipe of synth.Stream (Q, V ~ N(0,1); K with a
+    per-channel offset and four ten-fold channels per head; optionally AR(1) drifting means).  Returns device_fn."""
+    g = torch.Generator(device="cuda:0")
+    g.manual_seed(seed)
+    td = torch_dtype(dtype)
+    mu = torch.randn(H, 1, d, device="cuda:0", generator=g) * 0.5
+    m = torch.ones(H, 1, d, device="cuda:0")
+    for h in range(H):
+        m[h, 0, torch.randperm(d, device="cuda:0", generator=g)[:4]] = 10.0
+    state = {"t": -1, "dq": None, "dk": None, "dv": None}
+    frames = []
+
+    def fn(t):
+        if drift_rho is None:
+            if not frames:
+                for _ in range(pool):
+                    q = torch.randn(H, F, d, device="cuda:0", generator=g)
+                    k = (torch.randn(H, F, d, device="cuda:0", generator=g) + mu) * m
+                    v = torch.randn(H, F, d, device="cuda:0", generator=g)
+                    frames.append(tuple(x.to(td).contiguous() for x in (q, k, v)))
+            return frames[t % pool]
+        rho, innov = drift_rho, (1.0 - drift_rho ** 2) ** 0.5 * 0.5
+        while state["t"] < t:                                    # the means advance frame by frame
+            for key in ("dq", "dk", "dv"):
+                eps = torch.randn(H, 1, d, device="cuda:0", generator=g)
+                state[key] = eps * 0.5 if state[key] is None else rho * state[key] + innov * eps
+            state["t"] += 1
+        q = torch.randn(H, F, d, device="cuda:0", generator=g) + state["dq"]
+        k = (torch.randn(H, F, d, device="cuda:0", generator=g) + mu + state["dk"]) * m
+        v = torch.randn(H, F, d, device="cuda:0", generator=g) + state["dv"]
+        return tuple(x.to(td).contiguous() for x in (q, k, v))
+
+    return fn

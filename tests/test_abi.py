@@ -37,3 +37,9 @@ def test_host_side_argument_checks_need_no_gpu():
     assert lib.xsv_step(None, 0, None, None, None, 1, 0, None, None) == 1
     assert lib.xsv_strerror(6) == b"bounded device-side wait ran out"
     lib.xsv_cache_destroy(None)
+
+
+def test_per_device_table_keeps_devices_apart():
+    # kernel attributes are per CUDA device; the table that remembers them must not let one device's
+    # entry stand for another's (host-only self-test inside the library)
+    assert binding.load().xsv_selftest_device_table() == 0

@@ -205,8 +205,8 @@ def test_api_errors_and_bytes_constant():
     with pytest.raises(binding.XsvError) as e:
         c.set_options(n_special=3)                    # options after the first step
     assert e.value.code == 3
-    Q2 = torch.randn(16, 100, 64, device="cuda", dtype=torch.float16)
-    assert lib.xsv_step(c._h, 1, Q2.data_ptr(), Q2.data_ptr(), Q2.data_ptr(), 100, 0, out.data_ptr(), None) == 2
+    Q2 = torch.randn(16, 300, 64, device="cuda", dtype=torch.float16)      # more tokens than the largest frame allowed
+    assert lib.xsv_step(c._h, 1, Q2.data_ptr(), Q2.data_ptr(), Q2.data_ptr(), 300, 0, out.data_ptr(), None) == 2
     assert lib.xsv_step(c._h, 1, Q.data_ptr(), Q.data_ptr(), Q.data_ptr(), 261, 1, out.data_ptr(), None) == 2
     c.step(1, Q, Q, Q, out)
     b0 = c.bytes()
@@ -258,22 +258,22 @@ def test_bounded_wait_times_out_and_reports():
 
 
 def test_long_horizon_stream_stays_flat():
-    # config-3 shape (1374 tokens/frame, budget 10992, 2-bit), fewer layers and frames than the full run:
-    # once pruning has started the cache bytes, the cache length and the per-frame time must stay flat
+    # config-3 shape (1374 tokens/frame, budget 10992, 2-bit, per-channel means drifting as an AR(1) process),
+    # fewer layers and frames than the full run: once pruning has started the cache bytes and the cache length stay
+    # constant and the per-frame time does not drift
+    from tests.gpu_harness import device_stream
     H, F, L, bits, layers, frames = 16, 1374, 10992, 2, 4, 300
-    g = torch.Generator(device="cuda")
-    g.manual_seed(3)
-    pool = [tuple(torch.randn(H, F, 64, device="cuda", generator=g).to(torch.bfloat16) for _ in range(3)) for _ in range(5)]
+    feeds = [device_stream(H, F, "bf16", seed=40 + l, drift_rho=0.95) for l in range(layers)]
     out = torch.empty(H, F, 64, device="cuda", dtype=torch.bfloat16)
     c = binding.Cache(layers, H, 64, L, bits)
-    times, ev = [], [torch.cuda.Event(enable_timing=True) for _ in range(frames + 1)]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * frames)]
     bytes_seen = set()
-    ev[0].record()
     for t in range(frames):
-        q, k, v = pool[t % len(pool)]
+        inputs = [feeds[l](t) for l in range(layers)]          # drawn before the clock starts
+        ev[2 * t].record()
         for l in range(layers):
-            c.step(l, q, k, v, out)
-        ev[t + 1].record()
+            c.step(l, *inputs[l], out)
+        ev[2 * t + 1].record()
         if t >= 9:
             bytes_seen.add(c.bytes())
             assert c.len(layers - 1) == L
@@ -281,10 +281,58 @@ def test_long_horizon_stream_stays_flat():
     assert c.status() == 0
     assert len(bytes_seen) == 1                                   # constant device memory
     assert torch.isfinite(out.float()).all()
-    times = [ev[t].elapsed_time(ev[t + 1]) for t in range(frames)]
-    steady = sorted(times[20:])
-    p50, p99 = steady[len(steady) // 2], steady[int(len(steady) * 0.99)]
-    first, last = sum(times[20:60]) / 40, sum(times[-40:]) / 40
-    assert p99 < 1.5 * p50, (p50, p99)
-    assert abs(last - first) < 0.15 * first, (first, last)        # no drift of the per-frame time
+    times = [ev[2 * t].elapsed_time(ev[2 * t + 1]) for t in range(frames)]
+    med = lambda xs: sorted(xs)[len(xs) // 2]
+    early, late = med(times[20:60]), med(times[-40:])
+    assert abs(late - early) < 0.10 * early, (early, late)        # medians: robust against a neighbour's burst
     c.destroy()
+
+
+def test_host_step_with_joins_between_calls():
+    # deferred join + host buffers + xsv_cache_join between the calls and no device synchronisation: a staging slot
+    # must not be refilled while the side-stream kernels of the step that read it are still running
+    st = synth.Stream(H=4, d=64, F=200, dtype="bf16", layer=14)
+    a = binding.Cache(1, 4, 64, 700, 4)
+    b = binding.Cache(1, 4, 64, 700, 4)
+    a.set_deferred_join(True)
+    hosts, devs = [], []
+    for t in range(9):
+        q, k, v = (torch.from_numpy(x).to(torch.bfloat16) for x in st.frame(t))
+        Qh, Kh, Vh = q.pin_memory(), k.pin_memory(), v.pin_memory()
+        oh = torch.empty_like(Qh).pin_memory()
+        a.step_host(0, Qh, Kh, Vh, oh)
+        a.join()                                       # the caller's stream waits; the copy stream must still be held back
+        hosts.append((Qh, Kh, Vh, oh))
+        Q, K, V = q.cuda(), k.cuda(), v.cuda()
+        od = torch.empty_like(Q)
+        b.step(0, Q, K, V, od)
+        devs.append(od)
+    torch.cuda.synchronize()
+    for (_, _, _, oh), od in zip(hosts, devs):
+        assert torch.equal(oh, od.cpu())
+    sa, sb = a.export_layer(0), b.export_layer(0)
+    for key in sa:
+        assert np.array_equal(sa[key], sb[key])
+    a.destroy(); b.destroy()
+
+
+def test_two_devices_in_one_process():
+    # kernel attributes (opt-in shared memory) are set per device: a cache on a second GPU of the same process works
+    if torch.cuda.device_count() < 2:
+        pytest.skip("one GPU visible")
+    st = synth.Stream(H=2, d=64, F=150, dtype="fp16", layer=15)
+    outs = []
+    for dev in (0, 1):
+        torch.cuda.set_device(dev)
+        c = binding.Cache(1, 2, 64, 400, 4)
+        o = None
+        for t in range(5):
+            q, k, v = (torch.from_numpy(x).to(f"cuda:{dev}", torch.float16).contiguous() for x in st.frame(t))
+            o = torch.empty_like(q)
+            c.step(0, q, k, v, o)
+        torch.cuda.synchronize()
+        assert c.status() == 0
+        outs.append(o.cpu())
+        c.destroy()
+    torch.cuda.set_device(0)
+    assert torch.equal(outs[0], outs[1])

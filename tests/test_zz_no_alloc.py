@@ -26,9 +26,14 @@ def _inputs(H, F, n_keys, dtype, layer):
             torch.from_numpy(np.ascontiguousarray(keys)).to("cuda:0", td).contiguous())
 
 
+def _host(x):
+    return x.float().cpu().numpy().astype(np.float64)
+
+
 def test_static_scratch_entry_point_matches_allocating_one_twice():
     # two calls in a row, the second with fewer heads and other data, so that anything the
     # first call left in the shared array would show up if it were read
+    from oracle import xsv_oracle as orc
     for H, F, n_keys, dtype, layer in ((16, 1374, 4000, "bf16", 11), (4, 261, 777, "fp16", 12)):
         Q, keys = _inputs(H, F, n_keys, dtype, layer)
         want = binding.importance_scores(Q, keys)
@@ -42,6 +47,23 @@ def test_static_scratch_entry_point_matches_allocating_one_twice():
         w, g = want.cpu().numpy(), got.cpu().numpy()
         assert np.all(np.isfinite(g))
         assert np.max(np.abs(g - w)) <= TOL * np.max(np.abs(w))
+        # and against the definition itself (Eq. 3-7), not only against the other entry point
+        ref = orc.importance_scores(_host(Q), _host(keys), 5, 16)
+        assert np.max(np.abs(g - ref)) <= TOL * np.max(np.abs(ref))
+
+
+def test_static_scratch_entry_point_allocates_nothing_once_set_up():
+    # the first call on a device for an input type is set-up (the symbol's address is looked up and, with lazy
+    # loading, the module is loaded); from the second call on the free memory must not move, with no allocating
+    # call in between
+    Q, keys = _inputs(8, 300, 1500, "bf16", 13)
+    got = torch.empty(1500, device="cuda:0", dtype=torch.float32)
+    assert binding.importance_scores_static(Q, keys, got) == 0      # set-up call
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    assert binding.importance_scores_static(Q, keys, got) == 0
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before
 
 
 def test_static_scratch_entry_point_rejects_sizes_beyond_its_limit():
