@@ -10,7 +10,9 @@
  * top-k pruning that always keeps the first and the current frame (Eq. 8),
  * and dimension-adaptive quantisation of the resulting cache (Eq. 9-11:
  * keys per channel over groups of 64 tokens, values per token over 64
- * channels).  Every step of that path runs in CUDA kernels for sm_100a;
+ * channels; the quantiser subtracts the group minimum, as the quantiser of
+ * KIVI that section 4.1 names does: code = round((x - min) / s),
+ * x~ = code * s + min).  Every step of that path runs in CUDA kernels for sm_100a;
  * there is no CPU fallback.
  *
  * Conventions
@@ -62,7 +64,7 @@ typedef enum {
     XSV_ERR_OOM = 4,     /* device or host allocation failed                          */
     XSV_ERR_CUDA = 5,    /* a CUDA runtime call failed                                */
     XSV_ERR_TIMEOUT = 6, /* a bounded device-side wait ran out (status word)          */
-    XSV_ERR_RANGE = 7,   /* a zero-point left int32, or an input the fp16 range (status word) */
+    XSV_ERR_RANGE = 7,   /* an input lay beyond the fp16 range (status word)          */
     XSV_ERR_CAPACITY = 8,/* unbounded cache grew past max_cache_tokens                */
     XSV_ERR_LIMIT = 9    /* size beyond the fixed maximum of a no-allocation entry point */
 } xsv_status;
@@ -206,7 +208,6 @@ xsv_status xsv_importance_scores(const void* Q, const void* keys, int heads, int
  * (x - x~)^2 over all elements, accumulated in float64, is written to
  * *mse_host (HOST).  bits: 2, 4 or 8.  Allocates and frees its scratch on
  * `stream` (stream-ordered allocator) and synchronises `stream`.
- * XSV_ERR_RANGE: a zero-point left the int32 range.
  */
 xsv_status xsv_quantization_mse(const void* x, int heads, long long n_tokens, xsv_dtype dtype, int bits,
                                 int per_channel, double* mse_host, void* stream);
@@ -239,11 +240,11 @@ xsv_status xsv_importance_scores_static(const void* Q, const void* keys, int hea
                                         long long n_keys, xsv_dtype dtype, int n_special,
                                         int pool_group, float* scores, void* stream);
 
-/* Device bytes held now: codes, scales, zero-points, origin ids of all layer
+/* Device bytes held now: codes, scales, offsets, origin ids of all layer
  * buffers plus the spare buffer and scratch (section 4.6's memory figure). */
 size_t xsv_cache_bytes(const xsv_cache* c);
 
-/* Bytes of one layer's packed KV at its current length (codes + scales + zero-points). */
+/* Bytes of one layer's packed KV at its current length (codes + scales + offsets). */
 size_t xsv_cache_layer_kv_bytes(const xsv_cache* c, int layer);
 
 void xsv_cache_destroy(xsv_cache* c);
@@ -262,14 +263,15 @@ long long xsv_cache_frames(const xsv_cache* c, int layer);
  * Copy one layer's logical state to HOST arrays (synchronises `stream`).
  * Any pointer may be NULL to skip it.  With T = xsv_cache_len, H heads, d = head_dim:
  *   k_codes, v_codes : unsigned char [H][T][d], one code per byte (bits < 16);
- *   k_scale / k_zero : float / int [H][ceil(T/64)][d]  (Eq. 10, per channel per 64-token group);
- *   v_scale / v_zero : float / int [H][T]              (per token);
+ *   k_scale / k_zero : float [H][ceil(T/64)][d]  (Eq. 10, per channel per 64-token group: the scale and
+ *                      the offset, i.e. the group's minimum; a value is code * scale + offset, Eq. 12);
+ *   v_scale / v_zero : float [H][T]              (the same per token);
  *   origin           : long long [T], the running index in the stream of the token in each slot
  *                      (tokens of all earlier frames + its index in its frame);
  *   k_raw, v_raw     : unsigned short [H][T][d], the 16-bit cache when bits == 16.
  */
 xsv_status xsv_cache_export_layer(xsv_cache* c, int layer, unsigned char* k_codes, float* k_scale,
-                                  int* k_zero, unsigned char* v_codes, float* v_scale, int* v_zero,
+                                  float* k_zero, unsigned char* v_codes, float* v_scale, float* v_zero,
                                   long long* origin, unsigned short* k_raw, unsigned short* v_raw,
                                   void* stream);
 
@@ -291,8 +293,8 @@ xsv_status xsv_cache_export_layer(xsv_cache* c, int layer, unsigned char* k_code
  */
 xsv_status xsv_cache_import_layer(xsv_cache* c, int layer, long long n_cached, long long frames_done,
                                   int frame_tokens, xsv_dtype dtype, const unsigned char* k_codes,
-                                  const float* k_scale, const int* k_zero, const unsigned char* v_codes,
-                                  const float* v_scale, const int* v_zero, const long long* origin,
+                                  const float* k_scale, const float* k_zero, const unsigned char* v_codes,
+                                  const float* v_scale, const float* v_zero, const long long* origin,
                                   const unsigned short* k_raw, const unsigned short* v_raw, void* stream);
 
 /*

@@ -11,8 +11,8 @@ pooling group, G the quantisation group, b the bit width, n = 2^b - 1.
 
 Arithmetic: attention, pooling, scoring are accumulated in float64.  The
 quantiser (Eq. 9-10) and dequantiser (Eq. 12) are carried out in IEEE float32
-with one operation per rounding, because their results are integers (codes,
-zero-points) or float32 scales that the GPU must reproduce bit for bit.
+with one operation per rounding, because their results are integer codes and
+float32 scales and offsets that the GPU must reproduce bit for bit.
 
 Pins (tests/test_oracle_*.py): block-causal attention against a library
 softmax-attention routine; attention after pruning against attention over the
@@ -29,49 +29,58 @@ import numpy as np
 
 F32 = np.float32
 TINY = F32(2.0 ** -126)
-I32_MIN, I32_MAX = -(2 ** 31), 2 ** 31 - 1
 
 
 # --------------------------------------------------------------------------
 # Eq. 9-10: asymmetric uniform quantiser, one group at a time (vectorised over
 # leading axes; the group is the LAST axis of `x`).
+#
+# Form.  Section 3.3 prints the quantiser with an integer zero-point,
+# code = round(x / s) + z with z = round(-x_min / s); section 4.1 says the
+# quantisation is carried out with KIVI, whose quantiser subtracts the group
+# minimum instead: code = round((x - x_min) / s), x~ = code * s + x_min.  The two
+# differ by the rounding of the zero-point, i.e. by a shift of the whole grid of
+# up to s/2.  The cache is quantised again after every pruning step (section
+# 3.3: quantisation is applied to the final cache, kept and new entries alike),
+# and under that repetition the difference decides: with the minimum subtracted
+# a group's extremes are reproduced exactly, so ranges never outgrow the data;
+# with the rounded zero-point every pass shifts them, the selection keeps the
+# keys with the largest projections, and at 2 bits key magnitudes were measured
+# to grow tenfold within a few hundred frames.  The minimum-offset form is the
+# reading taken here; `z` below is that offset (a float32 in value units).
 # --------------------------------------------------------------------------
 def quantize_groups(x, bits):
-    """Quantise each row of x[..., m] as one group (Eq. 9-10).
+    """Quantise each row of x[..., m] as one group (Eq. 9-10, minimum-offset form).
 
-    s = (x_max - x_min) / (2^b - 1); z = round(-x_min / s);
-    code = clamp(round(x / s) + z, 0, 2^b - 1); round = nearest, ties to even.
-    All in float32: one subtraction, true divisions.  z is not clamped to the
-    code range (Eq. 10 has no clamp).  Degenerate group (s below the smallest
-    normal float32, which includes x_max == x_min): s := |x_min| if x_min != 0
-    else 1, after which the same formulas give code 0 everywhere and the
+    s = (x_max - x_min) / (2^b - 1); z = x_min;
+    code = clamp(round((x - z) / s), 0, 2^b - 1); round = nearest, ties to even.
+    All in float32, one rounding per operation: one subtraction for the range,
+    one true division for s, then per element one subtraction and one true
+    division.  Degenerate group (s below the smallest normal float32, which
+    includes x_max == x_min): s := 1, which gives code 0 everywhere and the
     dequantised value x_min exactly.
-    Returns (codes uint8 [..., m], s float32 [...], z int32 [...]).
+    Returns (codes uint8 [..., m], s float32 [...], z float32 [...]).
     """
     x = np.asarray(x, dtype=F32)
     n = (1 << bits) - 1
-    mn = x.min(axis=-1)
-    mx = x.max(axis=-1)
+    mn = x.min(axis=-1).astype(F32)
+    mx = x.max(axis=-1).astype(F32)
     with np.errstate(divide="ignore", invalid="ignore", over="ignore"):
-        s = (mx - mn).astype(F32) / F32(n)
-        s = s.astype(F32)
-        degenerate = ~(s >= TINY)
-        s_deg = np.where(mn != 0, np.abs(mn), F32(1.0)).astype(F32)
-        s = np.where(degenerate, s_deg, s).astype(F32)
-        zf = np.rint((-mn).astype(F32) / s).astype(F32)
-        z = np.clip(zf.astype(np.float64), I32_MIN, I32_MAX).astype(np.int64)
-        q = np.rint(x / s[..., None]).astype(F32)
-        q = np.clip(q.astype(np.float64), I32_MIN, I32_MAX).astype(np.int64)
-    codes = np.clip(q + z[..., None], 0, n).astype(np.uint8)
-    return codes, s, z.astype(np.int32)
+        s = ((mx - mn).astype(F32) / F32(n)).astype(F32)
+        s = np.where(s >= TINY, s, F32(1.0)).astype(F32)
+        y = (x - mn[..., None]).astype(F32)
+        q = np.rint((y / s[..., None]).astype(F32))
+    codes = np.clip(q.astype(np.float64), 0, n).astype(np.uint8)
+    return codes, s, mn
 
 
 def dequantize(codes, s, z):
-    """Eq. 12 (inverse of Eq. 9): x~ = (code - z) * s, one float32 multiply.
+    """Eq. 12 (inverse of Eq. 9): x~ = code * s + z, a float32 multiply followed by a float32 add
+    (two roundings; no fused multiply-add).
 
     codes [..., m]; s, z broadcastable to codes' shape."""
-    diff = codes.astype(np.int64) - np.asarray(z).astype(np.int64)
-    return (diff.astype(F32) * np.asarray(s, dtype=F32)).astype(F32)
+    prod = (codes.astype(F32) * np.asarray(s, dtype=F32)).astype(F32)
+    return (prod + np.asarray(z, dtype=F32)).astype(F32)
 
 
 def quantization_mse(x, bits, granularity, G=64):
@@ -197,9 +206,9 @@ def keep_positions(S, T_first, T_current, T, L_max):
 class LayerCache:
     """State of one layer's cache in its logical (unpacked) form.
 
-    bits in {2,4,8}: Kc/Vc uint8 codes [H,T,d]; Ks float32 / Kz int32
+    bits in {2,4,8}: Kc/Vc uint8 codes [H,T,d]; Ks / Kz float32 (scale, offset)
     [H, ceil(T/G), d] (per channel, groups of G consecutive tokens, Eq. 11);
-    Vs float32 / Vz int32 [H, T, d/G] (per token, groups of G channels).
+    Vs / Vz float32 [H, T, d/G] (per token, groups of G channels).
     bits == 16: quantisation off, Kc/Vc hold the 16-bit inputs as float32.
     origin[T] = running index of the token in the stream (tokens of all earlier frames + its index in its
     frame; frame_index * F + token_index when every frame holds F tokens) -- a label by which kept sets
@@ -219,9 +228,9 @@ class LayerCache:
         self.Kc = np.zeros((H, 0, d), cdt)
         self.Vc = np.zeros((H, 0, d), cdt)
         self.Ks = np.zeros((H, 0, d), F32)
-        self.Kz = np.zeros((H, 0, d), np.int32)
+        self.Kz = np.zeros((H, 0, d), F32)
         self.Vs = np.zeros((H, 0, d // G), F32)
-        self.Vz = np.zeros((H, 0, d // G), np.int32)
+        self.Vz = np.zeros((H, 0, d // G), F32)
         self.origin = np.zeros((0,), np.int64)
         self.last_scores = None
         self.last_keep = None
@@ -313,7 +322,7 @@ class LayerCache:
         K_vals = np.concatenate([Kd[:, from_cache], K], axis=1)      # float32 [H,T_new,d]
         Kc_new = np.zeros((H, T_new, d), np.uint8)
         Ks_new = np.zeros((H, n_groups, d), F32)
-        Kz_new = np.zeros((H, n_groups, d), np.int32)
+        Kz_new = np.zeros((H, n_groups, d), F32)
         fz = frozen_groups
         Kc_new[:, :fz * G] = self.Kc[:, :fz * G]
         Ks_new[:, :fz] = self.Ks[:, :fz]
@@ -336,14 +345,14 @@ class LayerCache:
         self.T = int(origin.shape[0])
         cdt = F32 if self.bits == 16 else np.uint8
         self.Kc, self.Vc = np.asarray(Kc, cdt), np.asarray(Vc, cdt)
-        self.Ks, self.Kz = np.asarray(Ks, F32), np.asarray(Kz, np.int32)
-        self.Vs, self.Vz = np.asarray(Vs, F32), np.asarray(Vz, np.int32)
+        self.Ks, self.Kz = np.asarray(Ks, F32), np.asarray(Kz, F32)
+        self.Vs, self.Vz = np.asarray(Vs, F32), np.asarray(Vz, F32)
         self.origin = np.asarray(origin, np.int64)
         self.tokens_seen = int(self.origin[-1]) + 1 if self.T else 0     # the last frame's last token is always kept
 
     def kv_bytes_packed(self):
         """Bytes of the packed representation: b-bit codes + float32 scale +
-        int32 zero-point per group (the figure the memory claim is about)."""
+        float32 offset per group (the figure the memory claim is about)."""
         if self.bits == 16:
             return 2 * self.H * self.T * self.d * 2
         code = 2 * self.H * self.T * self.d * self.bits // 8

@@ -164,8 +164,8 @@ class Cache:
             ptrs = [None] * 6 + [st["origin"], st["Kraw"], st["Vraw"]]
         else:
             st.update(Kc=np.zeros((H, T, d), np.uint8), Ks=np.zeros((H, ng, d), np.float32),
-                      Kz=np.zeros((H, ng, d), np.int32), Vc=np.zeros((H, T, d), np.uint8),
-                      Vs=np.zeros((H, T), np.float32), Vz=np.zeros((H, T), np.int32))
+                      Kz=np.zeros((H, ng, d), np.float32), Vc=np.zeros((H, T, d), np.uint8),
+                      Vs=np.zeros((H, T), np.float32), Vz=np.zeros((H, T), np.float32))
             ptrs = [st["Kc"], st["Ks"], st["Kz"], st["Vc"], st["Vs"], st["Vz"], st["origin"], None, None]
         args = [a.ctypes.data_as(C.c_void_p) if a is not None else None for a in ptrs]
         _check(self._lib.xsv_cache_export_layer(self._h, layer, *args, _stream_ptr(stream)),

@@ -53,7 +53,7 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t add
 __device__ __forceinline__ uint32_t tile_off(int row, int chunk) { return (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4)); }
 
 // Unpack + dequantise 16 consecutive codes starting at channel c0 (bit offset
-// c0*BITS of the row), using per-channel (ks, kz) or per-token (s, z).
+// c0*BITS of the row), using per-channel (ks, kz) or per-token (s, z) scale and offset: code * s + z (Eq. 12).
 template <int BITS, bool PER_CHANNEL>
 __device__ __forceinline__ void dequant16(const uint8_t* rowptr, int c0, const float* ks, const float* kz, float s,
                                           float z, uint32_t (&out)[8]) {
@@ -76,11 +76,11 @@ __device__ __forceinline__ void dequant16(const uint8_t* rowptr, int c0, const f
         float c_b = (float)((w[(e + 1) / CPW] >> (((e + 1) % CPW) * BITS)) & M);
         float a, b;
         if (PER_CHANNEL) {
-            a = __fmul_rn(c_a - kz[c0 + e], ks[c0 + e]);
-            b = __fmul_rn(c_b - kz[c0 + e + 1], ks[c0 + e + 1]);
+            a = __fadd_rn(__fmul_rn(c_a, ks[c0 + e]), kz[c0 + e]);
+            b = __fadd_rn(__fmul_rn(c_b, ks[c0 + e + 1]), kz[c0 + e + 1]);
         } else {
-            a = __fmul_rn(c_a - z, s);
-            b = __fmul_rn(c_b - z, s);
+            a = __fadd_rn(__fmul_rn(c_a, s), z);
+            b = __fadd_rn(__fmul_rn(c_b, s), z);
         }
         out[e / 2] = pack_h2(a, b);
     }
@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(256) attn_mma_kernel(LayerView lv, int T_c, co
         __syncthreads();   // previous tile fully consumed
         if (cached && BITS < 16) {
             if (tid < 64) sKs[tid] = lv.kscale[((size_t)h * lv.capg + t) * 64 + tid];
-            else if (tid < 128) sKz[tid - 64] = (float)lv.kzero[((size_t)h * lv.capg + t) * 64 + tid - 64];
+            else if (tid < 128) sKz[tid - 64] = lv.kzero[((size_t)h * lv.capg + t) * 64 + tid - 64];
             __syncthreads();
         }
         {
@@ -141,7 +141,7 @@ __global__ void __launch_bounds__(256) attn_mma_kernel(LayerView lv, int T_c, co
                     const size_t r = (size_t)h * lv.cap + base + row;
                     dequant16<BITS < 16 ? BITS : 4, true>(lv.kcodes + r * ROWB, qtr * 16, sKs, sKz, 0.f, 0.f, kk);
                     dequant16<BITS < 16 ? BITS : 4, false>(lv.vcodes + r * ROWB, qtr * 16, nullptr, nullptr,
-                                                               lv.vscale[r], (float)lv.vzero[r], vv);
+                                                               lv.vscale[r], lv.vzero[r], vv);
                 } else {
                     const uint4 *kp, *vp;
                     if (cached) {

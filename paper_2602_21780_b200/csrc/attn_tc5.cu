@@ -51,7 +51,7 @@ constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 // shared-memory map (from a 1024-byte aligned base)
 constexpr uint32_t OFF_Q = 0;                                  // 2 tiles
 constexpr uint32_t OFF_KV = 2 * TILE_BYTES;                    // NSTAGE x (K tile, V tile)
-constexpr uint32_t OFF_META = OFF_KV + NSTAGE * 2 * TILE_BYTES;   // key parameters as halves: [producer warp][offset | scale | bias][64]
+constexpr uint32_t OFF_META = OFF_KV + NSTAGE * 2 * TILE_BYTES;   // key parameters as halves: [producer warp][scale | offset][64]
 constexpr uint32_t OFF_BAR = OFF_META + 3072;
 constexpr uint32_t BAR_BYTES = 512;
 constexpr uint32_t SMEM_BYTES = OFF_BAR + BAR_BYTES + 1024;    // + alignment slack
@@ -65,7 +65,7 @@ static_assert(B_COUNT * 8 + 16 <= BAR_BYTES, "barrier block");
 __host__ __device__ constexpr uint32_t TM_S(int x, int b) { return (uint32_t)((x * NBUF + b) * SUB); }
 constexpr uint32_t TM_O0 = 2 * NBUF * SUB;
 static_assert(TM_O0 + 2 * XSV_D <= 512, "tensor memory columns");
-static_assert(NPROD * 3 * 64 * 2 <= 3072, "staging area of the key parameters");
+static_assert(NPROD * 2 * 64 * 2 <= 3072, "staging area of the key parameters");
 
 struct Params {
     LayerView lv;
@@ -322,7 +322,6 @@ template <int BITS> __host__ __device__ constexpr int unpack_shift(int i) {   //
 template <int BITS> __host__ __device__ constexpr int unpack_tb(int i) {      // mantissa bit of the code afterwards
     return BITS == 4 ? 4 * (i & 1) : BITS == 2 ? (i < 5 ? 2 * i : 2 * (i - 5)) : 0;
 }
-template <int BITS> __host__ __device__ constexpr int unpack_off(int i) { return 1024 >> unpack_tb<BITS>(i); }
 
 // half2 (OFF_i + code_i, OFF_i + code_{i + W/2}) of packed word w; i is a compile-time
 // constant after unrolling
@@ -333,32 +332,19 @@ __device__ __forceinline__ uint32_t code_pair(uint32_t w, int i) {
     const uint32_t magic = (uint32_t)(25 - tb) << 10;
     return ((w >> unpack_shift<BITS>(i)) & (m1 | (m1 << 16))) | (magic | (magic << 16));
 }
-// Eq. 12 on a pair of codes: ((OFF + code) - a) * s + b.  For a zero-point z with
-// OFF + z exactly representable in fp16 (|OFF + z| <= 2047) a = OFF + z, b = 0:
-// the subtraction is exact and the error is that of rounding s and the product.
-// Otherwise (the group lies far from zero) a = 0, b = -(OFF + z) * s, whose
-// rounding is about one unit in the last place of the values themselves.
+// Eq. 12 on a pair of codes: ((OFF + code) - OFF) * s + z with s the scale and z the offset of the group, both
+// rounded to fp16.  The subtraction is exact (OFF is the power of two that code_pair put into the exponent), so the
+// error is that of rounding s, z and the result: about one unit in the last place of the values themselves.
 template <int BITS>
-__device__ __forceinline__ uint32_t dq_pair(uint32_t w, int i, uint32_t a2, uint32_t s2, uint32_t b2) {
-    return hfma2_u(hsub2_u(code_pair<BITS>(w, i), a2), s2, b2);
+__device__ __forceinline__ uint32_t dq_pair(uint32_t w, int i, uint32_t s2, uint32_t z2) {
+    const uint32_t off = (uint32_t)(25 - unpack_tb<BITS>(i)) << 10;          // fp16 OFF
+    return hfma2_u(hsub2_u(code_pair<BITS>(w, i), off | (off << 16)), s2, z2);
 }
 
 __device__ __forceinline__ uint16_t f2h_sat(float x) {
     uint16_t h;
     asm("cvt.rn.satfinite.f16.f32 %0, %1;" : "=h"(h) : "f"(x));
     return h;
-}
-// the fp16 parameters (a, s, b) of dq_pair for scale s, zero-point z and offset off
-__device__ __forceinline__ void dq_params(float s, int z, int off, uint16_t& ah, uint16_t& sh, uint16_t& bh) {
-    const int zo = z > 0x70000000 ? z : z + off;   // no overflow; such a z takes the far branch anyway
-    sh = f2h_sat(s);
-    if (zo >= -2047 && zo <= 2047) {
-        ah = f2h_sat((float)zo);      // exact
-        bh = 0;
-    } else {
-        ah = 0;
-        bh = f2h_sat(-(float)zo * s);   // from the float32 scale: the rounding error of sh times a large zero-point would be of the order of the values
-    }
 }
 
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
@@ -468,8 +454,7 @@ __device__ __forceinline__ void tile_iter_next(const Params& p, int b, int u_las
 template <int NW>
 struct SlabRegs {
     uint32_t w[NW];
-    float s0, s1;
-    int z0, z1;
+    float s0, s1, z0, z1;
     bool valid;
 };
 
@@ -495,9 +480,8 @@ __device__ __noinline__ void producer_loop(const Params& p, const Cta c) {
     const int F = p.F, n_ct = p.n_ct, T_c = p.T_c;
     int* const status = p.status;
     const LayerView lv = p.lv;
-    uint16_t* const mA = reinterpret_cast<uint16_t*>(smem + OFF_META) + pw * 192;   // this warp's [offset | scale | bias][64]
-    uint16_t* const mS = mA + 64;
-    uint16_t* const mB = mA + 128;
+    uint16_t* const mS = reinterpret_cast<uint16_t*>(smem + OFF_META) + pw * 128;   // this warp's [scale | offset][64] as fp16
+    uint16_t* const mB = mS + 64;
 
     // slab g of the CTA: tile g / 8, slab g % 8; this warp owns g = pw, pw + NPROD, ...
     auto fetch = [&](const TileIter& ti, int sl, SlabRegs<NW>& r) {
@@ -514,7 +498,7 @@ __device__ __noinline__ void producer_loop(const Params& p, const Cta c) {
         if (sl < 4) {                       // key parameters of the channels at positions lane and lane + 32
             const int grp = ti.kv * 2 + ((sl & 3) >> 1);
             r.s0 = r.s1 = 0.f;
-            r.z0 = r.z1 = 0;
+            r.z0 = r.z1 = 0.f;
             if (grp * XSV_G < T_c) {
                 const size_t m = ((size_t)ti.h * lv.capg + grp) * 64;
                 r.s0 = lv.kscale[m + perm<W>(lane)];
@@ -560,45 +544,34 @@ __device__ __noinline__ void producer_loop(const Params& p, const Cta c) {
             if (sl < 4) {
                 // keys: stage the group's per-channel parameters (fp16, position order), then unpack the row
                 __syncwarp();                      // the previous slab's reads of the staging area are over
-                dq_params(rc.s0, rc.z0, unpack_off<UB>((lane >> 1) % SPW), mA[lane], mS[lane], mB[lane]);
-                dq_params(rc.s1, rc.z1, unpack_off<UB>(((lane + 32) >> 1) % SPW), mA[lane + 32], mS[lane + 32], mB[lane + 32]);
+                mS[lane] = f2h_sat(rc.s0); mB[lane] = f2h_sat(rc.z0);
+                mS[lane + 32] = f2h_sat(rc.s1); mB[lane + 32] = f2h_sat(rc.z1);
                 __syncwarp();
-                const uint4* a4p = reinterpret_cast<const uint4*>(mA);
                 const uint4* s4p = reinterpret_cast<const uint4*>(mS);
                 const uint4* b4p = reinterpret_cast<const uint4*>(mB);
 #pragma unroll
                 for (int ck = 0; ck < 8; ++ck) {   // 16-byte chunk = half2 slots 4ck .. 4ck+3
-                    const uint4 a4 = a4p[ck], s4 = s4p[ck], b4 = b4p[ck];
-                    const uint32_t av[4] = {a4.x, a4.y, a4.z, a4.w}, sv[4] = {s4.x, s4.y, s4.z, s4.w},
-                                   bv[4] = {b4.x, b4.y, b4.z, b4.w};
+                    const uint4 s4 = s4p[ck], b4 = b4p[ck];
+                    const uint32_t sv[4] = {s4.x, s4.y, s4.z, s4.w}, bv[4] = {b4.x, b4.y, b4.z, b4.w};
                     uint32_t o[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         const int slot = 4 * ck + q;
-                        o[q] = dq_pair<UB>(rc.w[(slot / SPW) % NW], slot % SPW, av[q], sv[q], bv[q]);
+                        o[q] = dq_pair<UB>(rc.w[(slot / SPW) % NW], slot % SPW, sv[q], bv[q]);
                     }
                     *reinterpret_cast<uint4*>(tile + swz(row, ck)) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
             } else {
-                // values: the row's own parameters, one offset variant per code position inside a word
-                uint32_t a2[SPW], s2, b2[SPW];
-                {
-                    uint16_t ah, sh, bh;
-#pragma unroll
-                    for (int i = 0; i < SPW; ++i) {
-                        dq_params(rc.s0, rc.z0, unpack_off<UB>(i), ah, sh, bh);
-                        a2[i] = (uint32_t)ah | ((uint32_t)ah << 16);
-                        b2[i] = (uint32_t)bh | ((uint32_t)bh << 16);
-                        s2 = (uint32_t)sh | ((uint32_t)sh << 16);
-                    }
-                }
+                // values: the row's own scale and offset
+                const uint32_t sh = f2h_sat(rc.s0), zh = f2h_sat(rc.z0);
+                const uint32_t s2 = sh | (sh << 16), z2 = zh | (zh << 16);
 #pragma unroll
                 for (int ck = 0; ck < 8; ++ck) {
                     uint32_t o[4];
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         const int slot = 4 * ck + q;
-                        o[q] = dq_pair<UB>(rc.w[(slot / SPW) % NW], slot % SPW, a2[slot % SPW], s2, b2[slot % SPW]);
+                        o[q] = dq_pair<UB>(rc.w[(slot / SPW) % NW], slot % SPW, s2, z2);
                     }
                     *reinterpret_cast<uint4*>(tile + swz(row, ck)) = make_uint4(o[0], o[1], o[2], o[3]);
                 }

@@ -99,8 +99,8 @@ __global__ void __launch_bounds__(1024) qtilde_final_kernel(float* __restrict__ 
 
 // ---------------------------------------------------------------------------
 // Eq. 5-7: S[j] = (1/H) sum_h q~ . K~[h, T_first + j, :] over the middle segment.
-// By linearity q~ . K~[h,p,:] = sum_c (q~_c s_c) code_c - sum_c q~_c s_c z_c, with
-// (s, z) the parameters of the key group of p: one block per key group, so the
+// By linearity q~ . K~[h,p,:] = sum_c (q~_c s_c) code_c + sum_c q~_c z_c, with
+// (s, z) the scale and offset of the key group of p: one block per key group, so the
 // weights q~_c s_c and the bias are prepared once per head and a token costs one
 // multiply-add per code.  256 threads = 64 tokens x 4 head slices; a warp reads
 // 32 consecutive packed rows of one head.  A thread first issues the loads of
@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
     constexpr uint32_t NMAX = (1u << BITS) - 1u;
     extern __shared__ __align__(16) float sm[];
     float* sW = sm;                             // [H][64] weights q~_c * s_c * 2^-(bits * position of c in its sub-word)
-    float* sB = sW + (size_t)H * 64;            // [H] bias sum_c q~_c s_c z_c
+    float* sB = sW + (size_t)H * 64;            // [H] bias sum_c q~_c z_c
     float* part = sB + ((H + 3) & ~3);          // [4][64] per-slice sums
 
     const int g = (T_first >> 6) + blockIdx.x;  // key group of this block
@@ -153,8 +153,7 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
             const float q0 = qfinal[lane] * qnorm, q1 = qfinal[lane + 32] * qnorm;
             const float pos = __int_as_float((127 - BITS * ((lane & 7) % SUB)) << 23);
             for (int h0 = warp; h0 < H; h0 += 2 * (SCORE_TPB / 32)) {     // two heads per pass: eight loads in flight
-                float sc[2][2];
-                int zz[2][2];
+                float sc[2][2], zz[2][2];
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     const int h = h0 + t * (SCORE_TPB / 32);
@@ -166,7 +165,7 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
                 for (int t = 0; t < 2; ++t) {
                     const int h = h0 + t * (SCORE_TPB / 32);
                     const float w0 = q0 * sc[t][0], w1 = q1 * sc[t][1];
-                    float b = w0 * (float)zz[t][0] + w1 * (float)zz[t][1];
+                    float b = q0 * zz[t][0] + q1 * zz[t][1];
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) b += __shfl_xor_sync(0xFFFFFFFFu, b, o);
                     if (h < H) {
@@ -213,7 +212,7 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
                         }
                     }
                 }
-                acc += a - sB[h];
+                acc += a + sB[h];
             }
         }
     }
@@ -601,9 +600,9 @@ __global__ void __launch_bounds__(1024) select_reg_kernel(const float* __restric
 // The arithmetic is arranged for the pipes it runs on (integer and min/max
 // instructions issue at half the rate of float multiply-adds):
 //  * a code is not shifted down before it is widened: (word & mask_k) | 2^23,
-//    read as a float, is 2^23 + code * 2^(bits k); the staged constants are
-//    -(2^23 + z * 2^(bits k)) and s * 2^-(bits k), so one add and one multiply
-//    give (code - z) * s with the same single rounding as Eq. 12;
+//    read as a float, is 2^23 + code * 2^(bits k); minus 2^23 and times the
+//    staged s * 2^-(bits k) that is code * s with the rounding of Eq. 12's
+//    multiply, and the group's offset is added in a second operation;
 //  * the clamp of Eq. 9 is a saturating multiply by 1/n, and a row's codes are
 //    summed into 16-bit sub-words by multiply-adds (n * 2^(bits k) each) and
 //    converted once per sub-word.
@@ -616,9 +615,8 @@ struct RqCfg {
     static constexpr int ROWB = XSV_D * BITS / 8;
     static constexpr int SUB = (BITS == 8) ? 2 : (BITS == 4 ? 4 : 8);   // codes per 16-bit sub-word
     static constexpr int NSUB = 8 / SUB;                                // sub-words per lane (8 codes)
-    static constexpr int ZLIM = 1 << (22 - BITS * (SUB - 1));           // |z| below this: 2^23 + z * 2^(bits k) is exact
     static constexpr int CODE_WORDS = XSV_G * ROWB / 4;
-    // per warp, in 4-byte words: old scale and offset constants, new scale / reciprocal / z as float / z,
+    // per warp, in 4-byte words: old scales and offsets, new scale / reciprocal / offset (+ 64 spare),
     // old positions, packed rows
     static constexpr int WORDS = 2 * RQ_WIN * 64 + 4 * 64 + 64 + CODE_WORDS;
     static constexpr int OFF_CODES = 2 * RQ_WIN * 64 + 4 * 64 + 64;
@@ -647,7 +645,7 @@ __device__ __forceinline__ uint32_t rq_sub(uint64_t ch, int j) { return (uint32_
 // General form of Eq. 12 for a row whose old group is outside the staged window or has parameters the fast
 // form cannot take: parameters from memory, one conversion per code.
 template <int BITS>
-__device__ __forceinline__ void rq_fetch_slow(const float* __restrict__ ks, const int* __restrict__ kz, uint64_t ch, float (&x)[8]) {
+__device__ __forceinline__ void rq_fetch_slow(const float* __restrict__ ks, const float* __restrict__ kz, uint64_t ch, float (&x)[8]) {
     constexpr uint32_t NMAX = (1u << BITS) - 1u;
 #pragma unroll
     for (int e = 0; e < 8; ++e) x[e] = xsv_dequant((int)((uint32_t)(ch >> (e * BITS)) & NMAX), kz[e], ks[e]);
@@ -665,16 +663,6 @@ __device__ __forceinline__ void rq_fetch_fresh(const T* __restrict__ row, float 
         x[2 * e] = xsv_to_float<T>(lo);
         x[2 * e + 1] = xsv_to_float<T>(hi);
     }
-}
-
-// General form of Eq. 9 for the 8 codes of one (token, channel octet).
-template <int BITS>
-__device__ __forceinline__ uint64_t rq_codes_slow(const float (&x)[8], const float* ns, const float* ni, const int* nz) {
-    uint64_t out = 0;
-#pragma unroll
-    for (int e = 0; e < 8; ++e)
-        out |= (uint64_t)(uint32_t)xsv_quant_code(x[e], ns[e], ni[e], nz[e], (1 << BITS) - 1) << (e * BITS);
-    return out;
 }
 
 // Values of kept tokens move verbatim (codes row, scale, zero-point, origin): one warp per (64 new positions, head).
@@ -740,9 +728,8 @@ __device__ __forceinline__ void rq_quant_v_item(const LayerView& dst, const T* _
             mn = fminf(mn, __shfl_xor_sync(0xFFFFFFFFu, mn, o));
             mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
         }
-        float s;
-        int z;
-        xsv_quant_params(mn, mx, NMAX, s, z, status);
+        float s, z;
+        xsv_quant_params(mn, mx, NMAX, s, z);
         const float inv_s = __frcp_rn(s);
         const uint32_t c0 = (uint32_t)xsv_quant_code(x0, s, inv_s, z, NMAX), c1 = (uint32_t)xsv_quant_code(x1, s, inv_s, z, NMAX);
         uint32_t w = (c0 | (c1 << BITS)) << (2 * BITS * (lane % LPW));
@@ -790,9 +777,8 @@ __global__ void __launch_bounds__(RQ_THREADS, 3) requant_k_kernel(LayerView src,
     float* w_zc = w_s + RQ_WIN * 64;
     float* n_s = w_zc + RQ_WIN * 64;
     float* n_i = n_s + 64;
-    float* n_zf = n_i + 64;
-    int* n_z = reinterpret_cast<int*>(n_zf + 64);
-    int* s_sp = n_z + 64;
+    float* n_zf = n_i + 64;                                   // the new groups' offsets
+    int* s_sp = reinterpret_cast<int*>(n_zf + 128);
     uint8_t* s_codes = reinterpret_cast<uint8_t*>(w_s + C::OFF_CODES);
     const int fz = fz_dev ? *fz_dev : fz_host;
     const bool same = (src.kcodes == dst.kcodes);
@@ -861,18 +847,18 @@ __global__ void __launch_bounds__(RQ_THREADS, 3) requant_k_kernel(LayerView src,
             // parameters of the staged old groups: lane l takes channels l and l + 32 of each row
             bool slow[RQ_WIN];
             const float* ksp = src.kscale + ((size_t)h * src.capg + g_lo) * 64 + lane;
-            const int* kzp = src.kzero + ((size_t)h * src.capg + g_lo) * 64 + lane;
+            const float* kzp = src.kzero + ((size_t)h * src.capg + g_lo) * 64 + lane;
 #pragma unroll
             for (int r = 0; r < RQ_WIN; ++r) {
                 slow[r] = false;
                 if (g_lo + r < src.capg) {
 #pragma unroll
                     for (int k = 0; k < 2; ++k) {
-                        const int z = kzp[r * 64 + 32 * k];
+                        const float z = kzp[r * 64 + 32 * k];
                         const float sc = ksp[r * 64 + 32 * k];
-                        const bool ok = z > -C::ZLIM && z < C::ZLIM && sc >= 7.8886090522101181e-31f /* 2^-100 */;
+                        const bool ok = sc >= 7.8886090522101181e-31f /* 2^-100: the scaling by 2^-(bits k) stays exact */;
                         w_s[r * 64 + 32 * k + lane] = sc * pos_scale;
-                        w_zc[r * 64 + 32 * k + lane] = -(float)(8388608 + (ok ? (z << pos_shift) : 0));
+                        w_zc[r * 64 + 32 * k + lane] = z;
                         slow[r] |= !ok;
                     }
                 }
@@ -918,7 +904,7 @@ __global__ void __launch_bounds__(RQ_THREADS, 3) requant_k_kernel(LayerView src,
 #pragma unroll
                         for (int e = 0; e < 8; ++e) {
                             const uint32_t m = (rq_sub<BITS>(ch, e / SUB) & ((uint32_t)NMAX << (BITS * (e % SUB)))) | 0x4B000000u;
-                            x[e] = __fmul_rn(__fadd_rn(__uint_as_float(m), cv[e]), sv[e]);
+                            x[e] = __fadd_rn(__fmul_rn(__fadd_rn(__uint_as_float(m), -8388608.f), sv[e]), cv[e]);
                         }
                     };
 #pragma unroll 1
@@ -973,22 +959,19 @@ __global__ void __launch_bounds__(RQ_THREADS, 3) requant_k_kernel(LayerView src,
             mx[e] = fmaxf(mx[e], __shfl_xor_sync(FULL, mx[e], 16));
         }
         // Eq. 10: this lane derives the parameters of channels 8w + 2tq and 8w + 2tq + 1
-        float s2[2];
-        int z2[2];
+        float s2[2], z2[2];
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
             const float a = tq == 0 ? mn[k] : tq == 1 ? mn[2 + k] : tq == 2 ? mn[4 + k] : mn[6 + k];
             const float b = tq == 0 ? mx[k] : tq == 1 ? mx[2 + k] : tq == 2 ? mx[4 + k] : mx[6 + k];
-            xsv_quant_params(a, b, NMAX, s2[k], z2[k], status);
+            xsv_quant_params(a, b, NMAX, s2[k], z2[k]);
             const int c = 8 * w + 2 * tq + k;
             n_s[c] = s2[k];
             n_i[c] = __frcp_rn(s2[k]);
-            n_z[c] = z2[k];
-            n_zf[c] = (z2[k] > -2097152 && z2[k] < 2097152) ? (float)z2[k] : __int_as_float(0x7FC00000);
+            n_zf[c] = z2[k];
         }
         __syncwarp();
         float iv[8], fv[8], ns[8];
-        bool slow_lane = false;
         {
             const float4 i0 = *reinterpret_cast<const float4*>(n_i + 8 * w), i1 = *reinterpret_cast<const float4*>(n_i + 8 * w + 4);
             const float4 f0 = *reinterpret_cast<const float4*>(n_zf + 8 * w), f1 = *reinterpret_cast<const float4*>(n_zf + 8 * w + 4);
@@ -996,34 +979,30 @@ __global__ void __launch_bounds__(RQ_THREADS, 3) requant_k_kernel(LayerView src,
             iv[0] = i0.x; iv[1] = i0.y; iv[2] = i0.z; iv[3] = i0.w; iv[4] = i1.x; iv[5] = i1.y; iv[6] = i1.z; iv[7] = i1.w;
             fv[0] = f0.x; fv[1] = f0.y; fv[2] = f0.z; fv[3] = f0.w; fv[4] = f1.x; fv[5] = f1.y; fv[6] = f1.z; fv[7] = f1.w;
             ns[0] = -a0.x; ns[1] = -a0.y; ns[2] = -a0.z; ns[3] = -a0.w; ns[4] = -a1.x; ns[5] = -a1.y; ns[6] = -a1.z; ns[7] = -a1.w;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) slow_lane |= (fv[e] != fv[e]);
         }
         uint8_t* const obase = dst.kcodes + ((size_t)h * dst.cap + p0 + tq) * ROWB + w * BITS;
         auto put = [&](int i, const float (&x)[8]) {
-            // Eq. 9 in the float domain.  Re-quantised values sit on rounding boundaries of the new grid whenever the
-            // old and new scales are in a small rational ratio, so the quotient must be the IEEE one every time: with
-            // 1/s correctly rounded, y0 = x (1/s) followed by two remainder corrections y += (x - y s) (1/s), each one
-            // fused multiply-add pair, is the correctly rounded x / s (the first correction makes y faithful, the
-            // second exact).  Then: round to nearest even by adding and subtracting 1.5 * 2^23, add the zero-point
-            // (exact: both are integers below 2^22), clamp to [0, n] by a saturating multiply with 1/n, and sum
+            // Eq. 9 in the float domain: d = x - offset (one subtraction), then round(d / s).  Re-quantised values sit
+            // on rounding boundaries of the new grid whenever the old and new scales are in a small rational ratio, so
+            // the quotient must be the IEEE one every time: with 1/s correctly rounded, y0 = d (1/s) followed by two
+            // remainder corrections y += (d - y s) (1/s), each one fused multiply-add pair, is the correctly rounded
+            // d / s (the first correction makes y faithful, the second exact).  Then: round to nearest even by adding
+            // and subtracting 1.5 * 2^23, clamp to [0, n] by a saturating multiply with 1/n, and sum
             // n * u * 2^(bits k) into the sub-word (the sum is within 2^-6 of the integer it stands for, so the
-            // conversion restores it).  A lane whose zero-points are too large for this takes the general routine
-            // (quotients beyond 2^21 imply such a zero-point, since code = quotient + z lies in [0, n]).
+            // conversion restores it).  The quotient lies in [0, n] up to rounding, far inside the exact range.
             uint64_t out;
-            if (slow_lane) {
-                out = rq_codes_slow<BITS>(x, n_s + 8 * w, n_i + 8 * w, n_z + 8 * w);
-            } else {
+            {
                 float acc[NSUB];
 #pragma unroll
                 for (int j = 0; j < NSUB; ++j) acc[j] = 0.f;
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    float y = __fmul_rn(x[e], iv[e]);
-                    y = __fmaf_rn(__fmaf_rn(y, ns[e], x[e]), iv[e], y);
-                    y = __fmaf_rn(__fmaf_rn(y, ns[e], x[e]), iv[e], y);
+                    const float d = __fsub_rn(x[e], fv[e]);
+                    float y = __fmul_rn(d, iv[e]);
+                    y = __fmaf_rn(__fmaf_rn(y, ns[e], d), iv[e], y);
+                    y = __fmaf_rn(__fmaf_rn(y, ns[e], d), iv[e], y);
                     const float r = __fadd_rn(__fadd_rn(y, 12582912.f), -12582912.f);
-                    const float u = rq_mul_sat(__fadd_rn(r, fv[e]), KINV);
+                    const float u = rq_mul_sat(r, KINV);
                     acc[e / SUB] = __fmaf_rn(u, (float)(NMAX << (BITS * (e % SUB))), acc[e / SUB]);
                 }
                 out = 0;
@@ -1038,7 +1017,7 @@ __global__ void __launch_bounds__(RQ_THREADS, 3) requant_k_kernel(LayerView src,
         walk(put, [&](int i, const float (&x0)[8], const float (&x1)[8]) { put(i, x0); put(i + 1, x1); });
         // the parameters go out last: in place, the group's old parameters may still have been read from memory above
         *reinterpret_cast<float2*>(dst.kscale + prm + 8 * w + 2 * tq) = make_float2(s2[0], s2[1]);
-        *reinterpret_cast<int2*>(dst.kzero + prm + 8 * w + 2 * tq) = make_int2(z2[0], z2[1]);
+        *reinterpret_cast<float2*>(dst.kzero + prm + 8 * w + 2 * tq) = make_float2(z2[0], z2[1]);
         __syncwarp();   // the staged rows are rewritten by the next item
     }
 }

@@ -163,9 +163,9 @@ xsv_status allocate(xsv_cache* c) {
         b.view.kcodes = base + off[0];
         b.view.vcodes = base + off[1];
         b.view.kscale = (float*)(base + off[2]);
-        b.view.kzero = (int*)(base + off[3]);
+        b.view.kzero = (float*)(base + off[3]);
         b.view.vscale = (float*)(base + off[4]);
-        b.view.vzero = (int*)(base + off[5]);
+        b.view.vzero = (float*)(base + off[5]);
         b.view.origin = (long long*)(base + off[6]);
         b.view.cap = cap;
         b.view.capg = (int)((cap + XSV_G - 1) / XSV_G);
@@ -268,7 +268,7 @@ const char* xsv_strerror(xsv_status s) {
         case XSV_ERR_OOM: return "out of memory";
         case XSV_ERR_CUDA: return "CUDA runtime error";
         case XSV_ERR_TIMEOUT: return "bounded device-side wait ran out";
-        case XSV_ERR_RANGE: return "value outside the supported range (zero-point beyond int32, or a 16-bit input beyond +-65504)";
+        case XSV_ERR_RANGE: return "a 16-bit input beyond the supported range of +-65504";
         case XSV_ERR_CAPACITY: return "unbounded cache exceeded max_cache_tokens";
         case XSV_ERR_LIMIT: return "size exceeds the fixed maximum of this no-allocation entry point";
     }
@@ -710,8 +710,8 @@ long long xsv_cache_frames(const xsv_cache* c, int layer) {
     return c->frames[layer];
 }
 
-xsv_status xsv_cache_export_layer(xsv_cache* c, int layer, unsigned char* k_codes, float* k_scale, int* k_zero,
-                                  unsigned char* v_codes, float* v_scale, int* v_zero, long long* origin,
+xsv_status xsv_cache_export_layer(xsv_cache* c, int layer, unsigned char* k_codes, float* k_scale, float* k_zero,
+                                  unsigned char* v_codes, float* v_scale, float* v_zero, long long* origin,
                                   unsigned short* k_raw, unsigned short* v_raw, void* stream) {
     if (!c || layer < 0 || layer >= c->layers) return XSV_ERR_ARG;
     cudaStream_t st = (cudaStream_t)stream;
@@ -755,8 +755,8 @@ xsv_status xsv_cache_export_layer(xsv_cache* c, int layer, unsigned char* k_code
 }
 
 xsv_status xsv_cache_import_layer(xsv_cache* c, int layer, long long n_cached, long long frames_done, int frame_tokens,
-                                  xsv_dtype dtype, const unsigned char* k_codes, const float* k_scale, const int* k_zero,
-                                  const unsigned char* v_codes, const float* v_scale, const int* v_zero,
+                                  xsv_dtype dtype, const unsigned char* k_codes, const float* k_scale, const float* k_zero,
+                                  const unsigned char* v_codes, const float* v_scale, const float* v_zero,
                                   const long long* origin, const unsigned short* k_raw, const unsigned short* v_raw,
                                   void* stream) {
     if (!c || layer < 0 || layer >= c->layers || n_cached < 0 || frames_done < 0 || frame_tokens <= 0 || !origin) return XSV_ERR_ARG;

@@ -27,16 +27,17 @@
 //                                  at bit offset c*bits of the row (little endian);
 //                                  rowb = 64*bits/8 bytes.  bits == 16: the raw
 //                                  16-bit elements.
-//   kscale/kzero  [H][capg][64]  : Eq. 10 parameters per channel per 64-token group.
-//   vscale/vzero  [H][cap]       : Eq. 10 parameters per token (64 channels).
+//   kscale/kzero  [H][capg][64]  : Eq. 10 parameters per channel per 64-token group: the scale and the
+//                                  offset (the group's minimum, in value units).
+//   vscale/vzero  [H][cap]       : the same per token (64 channels).
 //   origin        [cap]          : frame_index * F + token_index of each slot.
 struct LayerView {
     uint8_t* kcodes;
     float* kscale;
-    int* kzero;
+    float* kzero;
     uint8_t* vcodes;
     float* vscale;
-    int* vzero;
+    float* vzero;
     long long* origin;
     long long cap;
     int capg;
@@ -69,31 +70,29 @@ __device__ __forceinline__ float xsv_small_int_to_float(int v) {
     return __fadd_rn(__int_as_float(0x4B400000 + v), -12582912.f);
 }
 
-// Eq. 12: x~ = (code - z) * s, one float32 multiply.
-__device__ __forceinline__ float xsv_dequant(int code, int z, float s) {
-    const int v = code - z;
-    const float f = (v > -4194304 && v < 4194304) ? xsv_small_int_to_float(v) : __int2float_rn(v);
-    return __fmul_rn(f, s);
+// Eq. 12 in the minimum-offset form: x~ = code * s + z, a float32 multiply then a float32 add (two roundings,
+// never a fused multiply-add: the re-quantisation of kept keys starts from these values and must see the same
+// bits everywhere).
+__device__ __forceinline__ float xsv_dequant(int code, float z, float s) {
+    return __fadd_rn(__fmul_rn(xsv_small_int_to_float(code), s), z);
 }
 
-// Eq. 10 in float32, one rounding per operation; degenerate groups
-// (s below the smallest normal) take s = |mn| (or 1 when mn == 0).
-__device__ __forceinline__ void xsv_quant_params(float mn, float mx, int n, float& s, int& z, int* status) {
+// Eq. 10 in float32, one rounding per operation: s = (mx - mn) / n, offset z = mn; degenerate groups
+// (s below the smallest normal, which includes mx == mn) take s = 1.
+__device__ __forceinline__ void xsv_quant_params(float mn, float mx, int n, float& s, float& z) {
     s = __fdiv_rn(__fsub_rn(mx, mn), __int2float_rn(n));
-    if (!(s >= 1.17549435e-38f)) s = (mn != 0.f) ? fabsf(mn) : 1.f;
-    float zf = rintf(__fdiv_rn(-mn, s));
-    if (!(fabsf(zf) < 2147483648.f)) atomicOr(status, XSV_DEV_RANGE);
-    z = __float2int_rn(zf);   // saturates at the int32 limits
+    if (!(s >= 1.17549435e-38f)) s = 1.f;
+    z = mn;
 }
 
-// Eq. 9: clamp(round(x / s) + z, 0, n), round = nearest-even, with x / s the
-// IEEE float32 quotient.  inv_s = 1 / s (correctly rounded).  x * inv_s lies
-// within 2^-22 |x / s| of the true quotient, as does the rounded quotient
-// itself; unless x * inv_s comes within 2^-20 |x / s| of a rounding boundary
-// (a half-integer) both therefore round to the same integer, and the division
-// is skipped.  Near a boundary the exact division decides.
-__device__ __forceinline__ int xsv_quant_code(float x, float s, float inv_s, int z, int n) {
-    const float y = __fmul_rn(x, inv_s);
+// Eq. 9: clamp(round((x - z) / s), 0, n), round = nearest-even, with (x - z) one float32 subtraction and the
+// quotient the IEEE float32 one.  inv_s = 1 / s (correctly rounded).  y * inv_s lies within 2^-22 |y / s| of
+// the true quotient, as does the rounded quotient itself; unless y * inv_s comes within 2^-20 |y / s| of a
+// rounding boundary (a half-integer) both therefore round to the same integer, and the division is skipped.
+// Near a boundary the exact division decides.
+__device__ __forceinline__ int xsv_quant_code(float x, float s, float inv_s, float z, int n) {
+    const float d = __fsub_rn(x, z);
+    const float y = __fmul_rn(d, inv_s);
     int q;
     if (fabsf(y) < 2097152.f) {
         // round to nearest even by adding and subtracting 1.5 * 2^23 (exact for |y| < 2^21); the integer is
@@ -101,12 +100,11 @@ __device__ __forceinline__ int xsv_quant_code(float x, float s, float inv_s, int
         const float t = __fadd_rn(y, 12582912.f);
         const float r = __fadd_rn(t, -12582912.f);
         q = __float_as_int(t) - 0x4B400000;
-        if (fabsf(fabsf(y - r) - 0.5f) < fabsf(y) * 9.5367431640625e-7f) q = __float2int_rn(rintf(__fdiv_rn(x, s)));
+        if (fabsf(fabsf(y - r) - 0.5f) < fabsf(y) * 9.5367431640625e-7f) q = __float2int_rn(rintf(__fdiv_rn(d, s)));
     } else {
-        q = __float2int_rn(rintf(__fdiv_rn(x, s)));   // saturating
+        q = __float2int_rn(rintf(__fdiv_rn(d, s)));   // saturating
     }
-    const long long v = (long long)q + (long long)z;
-    return (int)(v < 0 ? 0 : (v > n ? n : v));
+    return q < 0 ? 0 : (q > n ? n : q);
 }
 
 // Programmatic dependent launch.  A kernel launched with xsv_launch_dep may be scheduled while the kernel before

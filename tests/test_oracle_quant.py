@@ -21,12 +21,12 @@ def test_hand_worked_examples(golden_dir):
         x = np.array([float(v) for v in xs.split()], np.float32)
         c, s_o, z_o = orc.quantize_groups(x[None, :], int(bits))
         assert float(s_o[0]) == float(s)
-        assert int(z_o[0]) == int(z)
+        assert float(z_o[0]) == float(z)
         assert c[0].tolist() == [int(v) for v in codes.split()]
         d = orc.dequantize(c, s_o[:, None], z_o[:, None])
         assert d[0].tolist() == [float(v) for v in deq.split()]
         n += 1
-    assert n >= 8
+    assert n >= 11
 
 
 @pytest.mark.parametrize("bits", [2, 4, 8])
@@ -43,7 +43,7 @@ def test_error_bound_min_max_and_range(bits, offset):
     assert np.all(c[r, amin] == 0)
     assert np.all(c[r, amax] >= n - 1)
     # |x - DQ(Q(x))| <= s/2 (float64 evaluation on the stored float32 s), plus the
-    # float32 rounding of the quotient x/s and of the product (code - z) * s, each
+    # float32 roundings of x - offset, of the quotient and of code * s + offset, each
     # at most 2^-24 |x|, which matters only for groups far from zero.
     d = orc.dequantize(c, s[:, None], z[:, None]).astype(np.float64)
     x64 = x.astype(np.float64)
@@ -55,19 +55,39 @@ def test_error_bound_min_max_and_range(bits, offset):
     assert np.all(np.diff(cs, axis=1) >= 0)
 
 
-def test_scale_and_zero_point_formulas_fp32():
-    # s and z are the printed formulas evaluated in float32 (independent re-evaluation
-    # with Python floats rounded to float32 at each operation).
+def test_scale_and_offset_formulas_fp32():
+    # s and the offset are the formulas evaluated in float32 (independent re-evaluation
+    # with Python floats rounded to float32 at each operation), and so are the codes.
     rng = np.random.default_rng(3)
     for bits in (2, 4, 8):
         n = (1 << bits) - 1
         for _ in range(200):
             x = rng.standard_normal(64).astype(np.float32) * np.float32(rng.uniform(0.1, 5))
             c, s, z = orc.quantize_groups(x[None], bits)
-            mn, mx = float(x.min()), float(x.max())
+            mn, mx = np.float32(x.min()), np.float32(x.max())
             s_ref = np.float32(np.float32(mx - mn) / np.float32(n))
-            z_ref = int(np.rint(np.float32(np.float32(-mn) / s_ref)))
-            assert float(s[0]) == float(s_ref) and int(z[0]) == z_ref
+            assert float(s[0]) == float(s_ref) and float(z[0]) == float(mn)
+            for i in (0, 17, 63):
+                q = np.rint(np.float32(np.float32(x[i] - mn) / s_ref))
+                assert int(c[0, i]) == int(min(max(q, 0), n))
+
+
+def test_extremes_are_reproduced_and_requantisation_is_idempotent():
+    # the property that keeps repeated quantisation of the cache stable: a group's minimum dequantises to itself
+    # exactly and its maximum to within the float32 rounding of n * s; quantising the dequantised group again
+    # changes neither the codes nor (beyond that rounding) the parameters
+    rng = np.random.default_rng(11)
+    for bits in (2, 4, 8):
+        n = (1 << bits) - 1
+        x = (rng.standard_normal((500, 64)) * rng.uniform(0.01, 30, (500, 1)) + rng.uniform(-50, 50, (500, 1))).astype(np.float32)
+        c, s, z = orc.quantize_groups(x, bits)
+        d = orc.dequantize(c, s[:, None], z[:, None])
+        r = np.arange(500)
+        assert np.array_equal(d[r, x.argmin(axis=1)], x.min(axis=1))
+        assert np.all(np.abs(d.max(axis=1).astype(np.float64) - x.max(axis=1)) <= 2.0 ** -22 * np.abs(x).max(axis=1))
+        c2, s2, z2 = orc.quantize_groups(d, bits)
+        assert np.array_equal(c2, c) and np.array_equal(z2, z)
+        assert np.all(np.abs(s2.astype(np.float64) - s) <= 2.0 ** -21 * s)
 
 
 def test_constant_and_tiny_groups_are_exact():
@@ -144,12 +164,12 @@ def test_mse_is_zero_for_values_on_the_grid():
 
 
 def test_mse_hand_worked_example():
-    # 2 bits (n = 3).  Token 0: [0, 1, 3] -> s = 1, z = 0, exact.  Token 1: [0, 0.4, 3] -> s = 1, 0.4 rounds to 0.
+    # 2 bits (n = 3).  Token 0: [0, 1, 3] -> s = 1, offset 0, exact.  Token 1: [0, 0.4, 3] -> s = 1, 0.4 rounds to 0.
     x = np.array([[[0.0, 1.0, 3.0], [0.0, 0.4, 3.0]]], dtype=np.float32)
     want = float(np.float64(np.float32(0.4)) ** 2) / 6.0
     assert orc.quantization_mse(x, 2, "token") == pytest.approx(want, rel=1e-12)
-    # per channel over the (partial) group of the two tokens: channel 1 is [1, 0.4] -> s = 0.2, z = round(-0.4/0.2) = -2,
-    # codes 3 and 0, dequantised (3+2)*0.2 = 1.0 and 0.4 up to float32 rounding; channels 0 and 2 are constant
+    # per channel over the (partial) group of the two tokens: channel 1 is [1, 0.4] -> s = 0.2, offset 0.4,
+    # codes 3 and 0, dequantised 3 * 0.2 + 0.4 = 1.0 (up to float32 rounding) and 0.4; channels 0 and 2 are constant
     got = orc.quantization_mse(x, 2, "channel")
     assert got < 1e-14
 

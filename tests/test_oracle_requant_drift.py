@@ -4,7 +4,10 @@ quantised again from their members' dequantised values).
 
 Each pass may move a value by up to half a step of the new grid, so the error of a long-lived key is not the one-shot
 bound s/2.  This measurement on a drifting stream shows that it grows over the first tens of frames and then
-saturates at a small multiple of s/2; the numbers are quoted in the design notes next to the reading."""
+saturates at a small multiple of s/2, and that key magnitudes never outgrow the inputs (the minimum-offset
+quantiser reproduces a group's extremes exactly; with a rounded integer zero-point the whole grid shifts by up to
+s/2 per pass and at 2 bits the magnitudes were measured to grow twelve-fold in 400 frames).  The numbers are quoted
+in the design notes next to the reading."""
 import numpy as np
 import pytest
 
@@ -16,8 +19,10 @@ def _age_profile(bits, frames=120, H=2, F=70, budget_frames=8):
     st = synth.Stream(H=H, d=64, F=F, dtype="bf16", layer=7, drift_rho=0.95)
     cache = orc.LayerCache(H, 64, budget_frames * F, bits)
     original = {}
+    k_in = 0.0
     for t in range(frames):
         Q, K, V = st.frame(t)
+        k_in = max(k_in, float(np.abs(K).max()))
         cache.step(Q, K, V)
         for i in range(F):
             original[t * F + i] = K[:, i, :]
@@ -27,7 +32,7 @@ def _age_profile(bits, frames=120, H=2, F=70, budget_frames=8):
     half_step = 0.5 * cache.Ks[:, np.arange(cache.T) // 64, :].astype(np.float64)
     err = np.abs(cache.dequant_K().astype(np.float64) - K0) / half_step      # in units of the current s/2
     middle = o >= F
-    out = {}
+    out = {"magnitude": (k_in, float(np.abs(cache.dequant_K()).max()), float(cache.Ks.max()))}
     for name, lo, hi in (("fresh", 0, 1), ("young", 1, 5), ("mid", 5, 20), ("old", 20, 10 ** 9)):
         m = middle & (age >= lo) & (age < hi)
         out[name] = (int(m.sum()), float(np.sqrt(np.mean(err[:, m] ** 2))) if m.any() else 0.0,
@@ -49,3 +54,7 @@ def test_requantisation_error_saturates(bits):
     assert prof["old"][1] <= 3.0
     # the worst single error is a few steps (at 2 bits the whole range is only 3 steps = 6 half-steps)
     assert prof["old"][2] <= (6.0 if bits == 2 else 16.0)
+    # the cached keys never exceed the largest input magnitude, and no group's range exceeds the inputs' spread
+    k_in, k_cached, s_max = prof["magnitude"]
+    assert k_cached <= k_in * (1 + 1e-6)
+    assert s_max * ((1 << bits) - 1) <= 2 * k_in * (1 + 1e-6)
