@@ -8,6 +8,10 @@ layer, 4-bit KV, bf16), in steady state (the cache is filled to its budget by
 untimed prefill frames first).  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+  python bench.py --config 3      long horizon: 24 layers x 1000 frames, budget 10992, 2-bit, drifting means;
+                                  per-frame latency p50 / p99 over frames 100-1000, its slope, bytes at start and end
+  python bench.py --config 4      one layer: budgets {4096, 16384, 65536} x bits {2, 4, 8} x frames {32, 256}, and the
+                                  uncompressed bf16 cache grown to a share of the free memory, timed at checkpoints
 
 N > 1 (under torchrun): the path does not shard -- every rank runs an independent
 replica (its own stream of frames); value = all ranks' frames / max-over-ranks time.
@@ -37,21 +41,27 @@ def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         m = json.load(open(p))
-        return dict(tflops=float(m.get("bf16_tflops_sustained", m.get("bf16_tflops"))), hbm=float(m["hbm_gbs"]),
+        return dict(tflops=float(m.get("bf16_tflops_sustained", m.get("bf16_tflops"))),
+                    tflops_burst=float(m.get("bf16_tflops", m.get("bf16_tflops_sustained"))), hbm=float(m["hbm_gbs"]),
                     source="measured (MEASURED_PEAKS.json, sustained bf16)")
-    return dict(tflops=1400.0, hbm=6650.0, source="fallback (no MEASURED_PEAKS.json)")
+    return dict(tflops=1400.0, tflops_burst=1590.0, hbm=6650.0, source="fallback (no MEASURED_PEAKS.json)")
 
 
-def attn_traffic_bytes():
-    """DRAM bytes per attention launch from the committed ncu summary, if any."""
-    p = os.path.join(ROOT, "profiles", "attention_config2_traffic.txt")
+TRAFFIC_FILE = os.path.join("profiles", "attention_config2_traffic.txt")
+
+
+def attn_traffic():
+    """DRAM bytes per attention launch from the committed ncu summary (with the capture it came from), if any."""
+    out = {"bytes": None, "source": None}
     try:
-        for line in open(p):
+        for line in open(os.path.join(ROOT, TRAFFIC_FILE)):
             if line.startswith("traffic_bytes_per_launch:"):
-                return float(line.split(":")[1])
+                out["bytes"] = float(line.split(":")[1])
+            elif line.startswith("captured:"):
+                out["source"] = f"{TRAFFIC_FILE} ({line.split(':', 1)[1].strip()})"
     except OSError:
         pass
-    return None
+    return out
 
 
 class ClockSampler:
@@ -152,6 +162,55 @@ def oracle_layer_step_seconds(repeats=1):
     return best
 
 
+def oracle_config_times(max_seconds=60.0):
+    """One steady-state layer-step of the oracle per configuration, on all BLAS threads and on one thread.
+    The one-thread run takes a sample of the heads (scaled up by the head ratio; heads are independent in every
+    step of the oracle except the head mean of the scores, which is a small share) so that it stays bounded."""
+    import numpy as np
+    from oracle import xsv_oracle as orc
+    from paper_2602_21780_b200 import synth
+    try:
+        from threadpoolctl import threadpool_limits
+    except Exception:
+        threadpool_limits = None
+    out = {}
+    t_begin = time.perf_counter()
+    shapes = {"config0": (16, 261, 1044, 4, "fp16", 1), "config1/2": (16, F, 21984, 4, "bf16", 1),
+              "config3": (16, F, 10992, 2, "bf16", 1)}
+    for name, (Hc, Fc, Lc, bc, dt, _) in shapes.items():
+        entry = {}
+        for threads, heads in (("all", Hc), ("one", 2)):
+            if time.perf_counter() - t_begin > max_seconds:
+                break
+            st = synth.Stream(H=heads, d=D, F=Fc, dtype=dt)
+            ref = orc.LayerCache(heads, D, Lc, bc)
+            n_pre = Lc // Fc
+            pre = [st.frame(t) for t in range(n_pre)]
+            K, V = np.concatenate([f[1] for f in pre], axis=1), np.concatenate([f[2] for f in pre], axis=1)
+            T = K.shape[1]
+            ng = -(-T // 64)
+            pad = ng * 64 - T
+            Kp = np.concatenate([K, np.repeat(K[:, -1:, :], pad, axis=1)], axis=1) if pad else K
+            kc, ks, kz = orc.quantize_groups(Kp.reshape(heads, ng, 64, D).transpose(0, 1, 3, 2), bc)
+            kc = kc.transpose(0, 1, 3, 2).reshape(heads, ng * 64, D)[:, :T]
+            vc, vs, vz = orc.quantize_groups(V.reshape(heads, T, 1, D), bc)
+            ref.load_state(n_pre, Fc, kc, ks, kz, vc.reshape(heads, T, D), vs, vz, np.arange(T))
+            q, k, v = st.frame(n_pre)
+            ctx = threadpool_limits(limits=1) if (threads == "one" and threadpool_limits) else None
+            t0 = time.perf_counter()
+            if ctx:
+                with ctx:
+                    ref.step(q, k, v)
+            else:
+                ref.step(q, k, v)
+            dt_s = (time.perf_counter() - t0) * (Hc / heads)
+            entry[threads + "_threads_s"] = dt_s
+            if threads == "one":
+                entry["one_thread_sample"] = f"{heads} of {Hc} heads, scaled by {Hc // heads}"
+        out[name] = entry
+    return out
+
+
 def replica_seed(base, rank):
     """Every rank streams its own frames: the path does not shard, ranks are independent replicas."""
     return base + rank
@@ -199,6 +258,174 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+class DriftFeed:
+    """Per-layer inputs of configuration 3, drawn on the device: the recipe of gen_frames plus per-channel means of
+    Q, K and V that follow an AR(1) process (rho = 0.95, stationary standard deviation 0.5), advanced frame by frame."""
+
+    def __init__(self, torch, dev, layers, seed, rho=0.95):
+        self.torch, self.dev, self.layers, self.rho = torch, dev, layers, rho
+        self.g = torch.Generator(device=dev)
+        self.g.manual_seed(seed)
+        self.mu = torch.randn(layers, H, 1, D, device=dev, generator=self.g) * 0.5
+        self.m = torch.ones(layers, H, 1, D, device=dev)
+        for l in range(layers):
+            for h in range(H):
+                self.m[l, h, 0, torch.randperm(D, device=dev, generator=self.g)[:4]] = 10.0
+        self.drift = [torch.randn(layers, H, 1, D, device=dev, generator=self.g) * 0.5 for _ in range(3)]
+        self.innov = (1.0 - rho * rho) ** 0.5 * 0.5
+
+    def frame(self):
+        """(Q, K, V), each [layers, H, F, D] bf16, for the next frame."""
+        t = self.torch
+        for i in range(3):
+            self.drift[i] = self.rho * self.drift[i] + self.innov * t.randn(self.layers, H, 1, D, device=self.dev, generator=self.g)
+        shp = (self.layers, H, F, D)
+        q = (t.randn(shp, device=self.dev, generator=self.g) + self.drift[0]).to(t.bfloat16)
+        k = ((t.randn(shp, device=self.dev, generator=self.g) + self.mu + self.drift[1]) * self.m).to(t.bfloat16)
+        v = (t.randn(shp, device=self.dev, generator=self.g) + self.drift[2]).to(t.bfloat16)
+        return q, k, v
+
+
+def run_config3(args, torch, binding, dev, stream):
+    """24 layers x 1000 frames, budget 10992, 2-bit, drifting means: frames/s, per-frame latency distribution over
+    frames 100-1000 and its slope, device bytes at the start of the steady state and at the end."""
+    layers, frames, L, bits = args.layers, args.frames or 1000, 10992, 2
+    feed = DriftFeed(torch, dev, layers, seed=20260221 + 3)
+    out = torch.empty(H, F, D, device=dev, dtype=torch.bfloat16)
+    cache = binding.Cache(layers, H, D, L, bits)
+    cache.set_deferred_join(True)
+    sp = stream.cuda_stream
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(frames)]
+    bytes_at = {}
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    launches0 = binding.kernel_launches()
+    t_wall = time.perf_counter()
+    for f in range(frames):
+        q, k, v = feed.frame()                           # drawn before the frame's clock starts
+        ev[f][0].record(stream)
+        for l in range(layers):
+            rc = cache.step_raw(l, q[l].data_ptr(), k[l].data_ptr(), v[l].data_ptr(), F, binding.BF16, out.data_ptr(), sp)
+            if rc != 0:
+                raise RuntimeError(f"xsv_step failed: status {rc}")
+        cache.join(stream)
+        ev[f][1].record(stream)
+        if f in (9, 99, frames - 1):
+            bytes_at[f + 1] = cache.bytes()
+        if f % 50 == 49:
+            torch.cuda.synchronize()                     # bounds the queue of pending launches and inputs
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t_wall
+    clocks = sampler.stop()
+    assert cache.status() == 0, "device status word set"
+    ms = [a.elapsed_time(b) for a, b in ev]
+    lo = min(100, frames // 2)
+    steady = sorted(ms[lo:])
+    n = len(steady)
+    xs = list(range(lo, frames))
+    mx, my = sum(xs) / n, sum(ms[lo:]) / n
+    slope = sum((x - mx) * (y - my) for x, y in zip(xs, ms[lo:])) / max(1e-9, sum((x - mx) ** 2 for x in xs))
+    total_ms = sum(ms[lo:])
+    line = {"metric": "frames/s of compressed-KV causal attention step (24 layers), long horizon", "value": n / (total_ms * 1e-3),
+            "unit": "frames/s", "n_gpus": 1, "steps": n, "warmup": lo, "ms_per_step": total_ms / n, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"config3: {layers} layers x (16 heads x 64), 1374 tokens/frame, {frames} frames, budget {L} "
+                                   f"tokens/layer, {bits}-bit KV, bf16, AR(1) drift (rho 0.95) of the per-channel means of Q, K, V "
+                                   "drawn on the device", "deferred_join": True,
+                       "l2": "each frame touches 203 MB of fresh inputs + 203 MB of cache (> 126 MB L2); no flush"},
+            "clocks": clocks, "gpu_launches": binding.kernel_launches() - launches0,
+            "latency_ms_per_frame": {"frames": f"{lo}-{frames}", "p50": steady[n // 2], "p99": steady[min(n - 1, int(n * 0.99))],
+                                     "min": steady[0], "max": steady[-1], "slope_ms_per_frame": slope,
+                                     "slope_over_run_fraction_of_p50": slope * n / steady[n // 2]},
+            "cache_bytes_at_frame": bytes_at, "cache_bytes_constant": len(set(bytes_at.values())) == 1,
+            "kv_bytes_per_layer": cache.layer_kv_bytes(0), "cache_len": cache.len(0), "wall_s_incl_input_generation": wall}
+    cache.destroy()
+    print(json.dumps(line), flush=True)
+
+
+def run_config4(args, torch, binding, dev, stream):
+    """One layer at paper shape: the budget x bits x frames sweep, then the uncompressed bf16 cache grown towards a
+    share of the free device memory and timed at checkpoints (frames between checkpoints are appended without their
+    attention, so the run does not pay for every step before a checkpoint)."""
+    sp = stream.cuda_stream
+    frames_pool = gen_frames(torch, dev, 1, POOL, seed=20260221 + 4)[0]
+    out = torch.empty(H, F, D, device=dev, dtype=torch.bfloat16)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    peaks = measured_peaks()
+    rows = []
+    for budget in (4096, 16384, 65536):
+        for bits in (2, 4, 8):
+            for n_frames in (32, 256):
+                c = binding.Cache(1, H, D, budget, bits)
+                c.set_deferred_join(True)
+                times = []
+                for f in range(n_frames):
+                    q, k, v = frames_pool[f % POOL]
+                    timed = f >= n_frames - 8                       # the last 8 frames of the run
+                    if timed:
+                        e0.record(stream)
+                    rc = c.step_raw(0, q.data_ptr(), k.data_ptr(), v.data_ptr(), F, binding.BF16, out.data_ptr(), sp)
+                    if rc != 0:
+                        raise RuntimeError(f"xsv_step failed: status {rc}")
+                    if timed:
+                        c.join(stream)
+                        e1.record(stream)
+                        torch.cuda.synchronize()
+                        times.append(e0.elapsed_time(e1))
+                assert c.status() == 0
+                ms = sorted(times)[len(times) // 2]
+                T = c.len(0) + F
+                rows.append({"budget": budget, "bits": bits, "frames": n_frames, "cache_len": c.len(0),
+                             "pruning": c.len(0) >= max(budget, 2 * F) and n_frames * F > budget,
+                             "ms_per_layer_step": ms, "layer_steps_per_s": 1e3 / ms,
+                             "attention_tflops_if_all_time_were_attention": 4.0 * F * T * D * H / (ms * 1e-3) / 1e12,
+                             "kv_bytes": c.layer_kv_bytes(0), "device_bytes": c.bytes()})
+                c.destroy()
+    # ---- the uncompressed reference point: no pruning, no quantisation, cache as large as the memory allows
+    free, total = torch.cuda.mem_get_info()
+    tok_bytes = 2 * H * D * 2                                        # K and V rows, bf16
+    limit = min(0.85 * free, args.max_gb * 1e9)
+    max_frames = int((limit - 2e9) // (tok_bytes * F))               # 2 GB kept for scratch and inputs
+    checkpoints = [n for n in (32, 256, 1000, 4000, 16000) if n < max_frames] + [max_frames]
+    c = binding.Cache(1, H, D, 0, 16)
+    c.set_options(max_frame_tokens=F, max_cache_tokens=(max_frames + 2) * F)
+    grown = []
+    done = 0
+    for cp in checkpoints:
+        while done < cp - 1:                                         # bulk append up to the frame before the checkpoint
+            q, k, v = frames_pool[done % POOL]
+            c.append(0, k, v, stream)
+            done += 1
+        torch.cuda.synchronize()
+        times = []
+        for r in range(3):                                           # the checkpoint's own step, timed; repeated on
+            q, k, v = frames_pool[(done + r) % POOL]                 # the following frames (the cache grows by three)
+            e0.record(stream)
+            rc = c.step_raw(0, q.data_ptr(), k.data_ptr(), v.data_ptr(), F, binding.BF16, out.data_ptr(), sp)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            if rc != 0:
+                raise RuntimeError(f"xsv_step failed: status {rc}")
+            times.append(e0.elapsed_time(e1))
+        done += 3
+        ms = sorted(times)[1]
+        T = done * F
+        grown.append({"frames": done, "cache_tokens": c.len(0), "kv_bytes": c.layer_kv_bytes(0), "ms_per_layer_step": ms,
+                      "attention_tflops": 4.0 * F * T * D * H / (ms * 1e-3) / 1e12,
+                      "frac_of_bf16_sustained": 4.0 * F * T * D * H / (ms * 1e-3) / 1e12 / peaks["tflops"]})
+    assert c.status() == 0
+    dev_bytes = c.bytes()
+    c.destroy()
+    line = {"metric": "one-layer sweep: ms per layer-step over budget x bits x frames; uncompressed bf16 cache growth",
+            "value": None, "unit": "ms per layer-step", "n_gpus": 1, "higher_is_better": False, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "config4: one layer, 16 heads x 64, 1374 tokens/frame, bf16; median of the last 8 frames of "
+                                   "each run; uncompressed run: bits = 16, no budget, frames between checkpoints appended "
+                                   "without attention (xsv_cache_append)",
+                       "uncompressed_memory_limit_bytes": limit, "free_bytes": free, "total_bytes": total},
+            "sweep": rows, "uncompressed": grown, "uncompressed_device_bytes": dev_bytes}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     global LAYERS, WORKLOAD, L_MAX, BITS, PREFILL
     ap = argparse.ArgumentParser()
@@ -215,6 +442,11 @@ def main():
                     help="cache budget in frames (default 16 = the benchmark; other values: the cache-length sweep)")
     ap.add_argument("--bits", type=int, default=BITS, choices=[2, 4, 8, 16],
                     help="bits per cached element (default 4 = the benchmark; 16 = quantisation off, pruning only)")
+    ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4],
+                    help="2: the benchmark (default); 3: the long-horizon run; 4: the one-layer sweep and the uncompressed cache")
+    ap.add_argument("--frames", type=int, default=0, help="--config 3: frames to stream (default 1000)")
+    ap.add_argument("--max-gb", type=float, default=120.0,
+                    help="--config 4: cap in GB on the uncompressed cache (it also stays below 85 %% of the free memory)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -246,6 +478,10 @@ def main():
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
+    if args.config in (3, 4):
+        if rank == 0:
+            (run_config3 if args.config == 3 else run_config4)(args, torch, binding, dev, torch.cuda.current_stream())
+        return
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
@@ -305,13 +541,22 @@ def main():
     launches = binding.kernel_launches() - launches0
     clocks = sampler.stop()
     prof = cache.profile_read(reset=True)
-    # the other phases, in a short pass of their own after the timed region (events around every phase slow the step)
-    cache.set_profiling(1)
+    # the other phases, in short passes of their own after the timed region (events around every phase slow the step):
+    # once as the step runs (selection and quantisation on the library's own streams: spans that include waiting for
+    # free multiprocessors) and once with every kernel on the caller's stream in order (spans = kernel durations)
     n_phase_frames = max(1, min(3, args.steps))
-    for f in range(n_phase_frames):
-        frame_step(cache, PREFILL + args.warmup + args.steps + f)
-    torch.cuda.synchronize()
-    prof_all = cache.profile_read(reset=True)
+    prof_all, prof_serial = None, None
+    for mode in (1, 4):
+        cache.set_profiling(mode)
+        cache.profile_read(reset=True)
+        for f in range(n_phase_frames):
+            frame_step(cache, PREFILL + args.warmup + args.steps + f)
+        cache.join(stream)
+        torch.cuda.synchronize()
+        if mode == 1:
+            prof_all = cache.profile_read(reset=True)
+        else:
+            prof_serial = cache.profile_read(reset=True)
     cache.set_profiling(0)
     assert cache.status() == 0, "device status word set"
     assert cache.bytes() == bytes_before, "cache bytes changed in steady state"
@@ -327,9 +572,12 @@ def main():
     T_all = L_MAX + F
     flops = 4.0 * F * T_all * D * H
     achieved = flops / (attn_ms / attn_n * 1e-3) / 1e12 if attn_n else None
+    traffic = attn_traffic()
     roofline = {"bound": "tensor", "kernel": "fused dequant+attention", "achieved": achieved,
                 "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"] if achieved else None,
-                "traffic": None if sweep else attn_traffic_bytes(), "peak_source": peaks["source"],
+                "peak_burst": peaks["tflops_burst"], "frac_of_burst_peak": achieved / peaks["tflops_burst"] if achieved else None,
+                "traffic": None if sweep else traffic["bytes"], "traffic_source": None if sweep else traffic["source"],
+                "peak_source": peaks["source"],
                 "flops_per_launch": flops, "avg_launch_ms": attn_ms / attn_n if attn_n else None,
                 "launches_timed": attn_n, "launches_total": args.steps * LAYERS,
                 "kernels_per_launch": attn_launches / attn_n if attn_n else None}
@@ -340,18 +588,22 @@ def main():
     score_bytes = n_mid * (H * D * BITS // 8 + H * 8) + H * F * D * 2
     quant_bytes = n_mid * tok_b + 2 * H * F * D * 2 + (L_MAX - F) * tok_b
     phases = {}
+    steps_n = n_phase_frames * LAYERS
     for name, nbytes in (("score", score_bytes), ("select", n_mid * 4 + k_keep * 4), ("quant", quant_bytes)):
-        pms, pn = prof_all[name]
-        steps_n = n_phase_frames * LAYERS
+        pms, pn = prof_serial[name]
+        oms, _ = prof_all[name]
         if steps_n and pms > 0:
             per = pms / steps_n
             phases[name] = {"avg_ms": per, "algorithmic_bytes": nbytes, "GB/s": nbytes / (per * 1e-3) / 1e9,
-                            "frac_of_hbm": nbytes / (per * 1e-3) / 1e9 / peaks["hbm"], "launches_per_step": pn / steps_n}
-    phases["attn"] = {"avg_ms": attn_ms / attn_n if attn_n else None}
-    phases["note"] = (f"score/select/quant: events around every phase, {n_phase_frames} frames after the timed region; "
-                      "select and quant run on the library's second stream under the tail of the attention kernel, so "
-                      "their spans start when the scores are ready and include the wait for free multiprocessors: the "
-                      "phases overlap and do not add up to the step")
+                            "frac_of_hbm": nbytes / (per * 1e-3) / 1e9 / peaks["hbm"], "launches_per_step": pn / steps_n,
+                            "span_ms_when_overlapped": oms / steps_n if oms > 0 else None}
+    phases["attn"] = {"avg_ms": attn_ms / attn_n if attn_n else None,
+                      "avg_ms_serial_pass": prof_serial["attn"][0] / steps_n if steps_n else None}
+    phases["note"] = (f"score/select/quant: {n_phase_frames} frames after the timed region with every kernel of the step on one "
+                      "stream in order and events around each phase, so avg_ms is the duration of the phase's kernels "
+                      "(24 layers x 700 MB of cache between two visits of a layer: nothing of it is still in the L2); "
+                      "span_ms_when_overlapped is the same phase as the benchmark runs it, on the library's own streams "
+                      "beside the attention kernel, where the span includes waiting for free multiprocessors")
     cache.destroy()
 
     # ---- end to end: same metric through the C ABI with HOST buffers (copies inside the timed region)
@@ -395,7 +647,9 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sec = oracle_layer_step_seconds()
         cpu = {"value": 1.0 / (LAYERS * sec), "unit": "frames/s", "cores": blas_threads(), "kind": "oracle",
-               "sample": f"one steady-state layer-step (T_c={L_MAX}) = 1/24 frame: {sec:.2f} s, extrapolated x24"}
+               "nproc": os.cpu_count(),
+               "sample": f"one steady-state layer-step (T_c={L_MAX}) = 1/24 frame: {sec:.2f} s on all threads, extrapolated x24",
+               "layer_step_seconds_by_config": oracle_config_times()}
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": "frames/s", "n_gpus": world, "steps": args.steps,

@@ -139,6 +139,39 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
                     int n_tokens, xsv_dtype dtype, void* out, void* stream);
 
 /*
+ * One step for several independent video streams at once (no counterpart in
+ * the paper, which streams one video; this is how a server fills the GPU when
+ * one stream's step is too small to, e.g. with the paper's own budget of about
+ * two frames).  caches[i] is stepped on layer `layer` with the frame
+ * Q[i], K[i], V[i] of n_tokens[i] tokens and writes out[i]; each call argument
+ * is a HOST array of n entries (device pointers for Q, K, V, out), n at most
+ * XSV_MAX_BATCH.  The attention of all n streams is ONE kernel launch (plus one
+ * merge launch) whose CTAs are dealt to the streams in proportion to their
+ * work; scores, selection and quantisation run per stream, the selection and
+ * quantisation on each cache's own streams side by side.  Results and cache
+ * states are those of n xsv_step calls.  The caches must be distinct, on one
+ * device, with equal heads and bit width (XSV_ERR_SHAPE otherwise) and use the
+ * default attention kernel; every cache is checked before anything is launched,
+ * so an argument, shape or order error leaves all of them unchanged.
+ */
+#define XSV_MAX_BATCH 8
+xsv_status xsv_step_batch(xsv_cache* const* caches, int n, int layer, const void* const* Q,
+                          const void* const* K, const void* const* V, const int* n_tokens,
+                          xsv_dtype dtype, void* const* out, void* stream);
+
+/*
+ * The cache update of a step without its attention (no counterpart in the
+ * paper: a way to fill a cache quickly, e.g. to measure the attention over a
+ * long uncompressed cache without paying for every step before it).  Appends
+ * the frame's keys and values as xsv_step would, quantised if the cache is.
+ * Only for steps that do not prune (the first frame, an unbounded cache, or
+ * T_c + n_tokens <= L_max): a pruning step needs the frame's queries and
+ * returns XSV_ERR_ORDER here.  Counts as the layer's step for this frame.
+ */
+xsv_status xsv_cache_append(xsv_cache* c, int layer, const void* K, const void* V, int n_tokens,
+                            xsv_dtype dtype, void* stream);
+
+/*
  * Deferred join (off by default).  With on != 0, `stream` does not wait at the
  * end of a pruning step for the selection and re-quantisation kernels on the
  * cache's own streams: they finish under whatever `stream` runs next (the next
@@ -321,8 +354,11 @@ int xsv_cache_status_word(xsv_cache* c, void* stream);
  * phase on the step's stream; on = 2: around the attention phase only (each
  * pair of events costs the stream a few microseconds, which matters when the
  * whole step is being timed as well); on = 3: around every seventh attention
- * phase (a sample that walks through the layers of a 24-layer stack); on = 0:
- * none.  xsv_cache_profile_read
+ * phase (a sample that walks through the layers of a 24-layer stack); on = 4:
+ * as 1, and every kernel of the step runs on `stream` in order (the cache's own
+ * streams are not used), so that the recorded spans are kernel durations and
+ * not spans that include waiting for free multiprocessors; on = 0: none.
+ * xsv_cache_profile_read
  * synchronises the recorded events, adds their durations to per-phase totals,
  * and returns the totals (milliseconds) and launch counts accumulated since
  * the last reset.  Events are created when profiling is switched on and, if

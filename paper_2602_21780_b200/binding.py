@@ -24,6 +24,8 @@ SYMBOLS = {
     "xsv_cache_set_options": (_i, [_vp, _i, _i, _i, _i, _ll]),
     "xsv_cache_set_attn_impl": (_i, [_vp, _i]),
     "xsv_step": (_i, [_vp, _i, _vp, _vp, _vp, _i, _i, _vp, _vp]),
+    "xsv_step_batch": (_i, [_vp, _i, _i, _vp, _vp, _vp, _vp, _i, _vp, _vp]),
+    "xsv_cache_append": (_i, [_vp, _i, _vp, _vp, _i, _i, _vp]),
     "xsv_step_host": (_i, [_vp, _i, _vp, _vp, _vp, _i, _i, _vp, _vp]),
     "xsv_cache_set_host_pipelining": (_i, [_vp, _i]),
     "xsv_cache_host_flush": (_i, [_vp, _vp]),
@@ -69,6 +71,17 @@ def load():
     return _lib
 
 
+def step_batch(caches, layer, Qs, Ks, Vs, outs, stream=None):
+    """One step of several caches in one call (see xsv_step_batch): lists of CUDA tensors, one per cache."""
+    n = len(caches)
+    lib = load()
+    arr = lambda xs: (C.c_void_p * n)(*[x.data_ptr() for x in xs])
+    handles = (C.c_void_p * n)(*[c._h.value for c in caches])
+    ntok = (C.c_int * n)(*[int(q.shape[1]) for q in Qs])
+    _check(lib.xsv_step_batch(handles, n, layer, arr(Qs), arr(Ks), arr(Vs), ntok, _dtype_code(Qs[0]), arr(outs),
+                              _stream_ptr(stream)), "xsv_step_batch")
+
+
 class XsvError(RuntimeError):
     def __init__(self, code, where):
         self.code = code
@@ -110,6 +123,11 @@ class Cache:
     def set_options(self, n_special=-1, pool_group=-1, quant_group=-1, max_frame_tokens=0, max_cache_tokens=-1):
         _check(self._lib.xsv_cache_set_options(self._h, n_special, pool_group, quant_group, max_frame_tokens,
                                                int(max_cache_tokens)), "xsv_cache_set_options")
+
+    def append(self, layer, K, V, stream=None):
+        """The cache update of a step without its attention (steps that do not prune)."""
+        _check(self._lib.xsv_cache_append(self._h, layer, K.data_ptr(), V.data_ptr(), K.shape[1], _dtype_code(K),
+                                          _stream_ptr(stream)), "xsv_cache_append")
 
     def set_attn_impl(self, impl):
         _check(self._lib.xsv_cache_set_attn_impl(self._h, impl), "xsv_cache_set_attn_impl")

@@ -84,6 +84,16 @@ struct Params {
 
 constexpr int PART_STRIDE = 256 * 66;   // floats per (CTA, slot)
 
+// Several independent streams (caches) in one launch: stream s owns the CTAs [cta_base[s], cta_base[s + 1]) and the
+// units [unit_base[s], unit_base[s + 1]) of the merge grid; each stream's Params carries its own CTA count G, its
+// slice of the workspace and its own status word, so inside a CTA everything is as for a launch of that stream alone.
+struct BatchParams {
+    int n;
+    int cta_base[XSV_MAX_BATCH + 1];
+    int unit_base[XSV_MAX_BATCH + 1];
+    Params p[XSV_MAX_BATCH];
+};
+
 // ------------------------------------------------------------------ work split
 struct Span { int kv0, kv1; };
 
@@ -895,7 +905,10 @@ __device__ __noinline__ void mma_loop(const Params& p, const Cta c, const int x)
 
 // ------------------------------------------------------------------ the kernel
 template <typename T, int BITS>
-__global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_constant__ Params p) {
+__global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_constant__ BatchParams bp) {
+    int s_idx = 0;
+    while (s_idx + 1 < bp.n && (int)blockIdx.x >= bp.cta_base[s_idx + 1]) ++s_idx;    // uniform: this CTA's stream
+    const Params& p = bp.p[s_idx];
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t smem_base = smem_u32(smem);
@@ -905,7 +918,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_cons
     auto BAR = [&](int i) { return bar_base + 8u * (uint32_t)i; };
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int b = blockIdx.x;
+    const int b = (int)blockIdx.x - bp.cta_base[s_idx];
     const long long tick0 = cta_tick(p, b), tick1 = cta_tick(p, b + 1);
     if (tick0 >= tick1) {                             // uniform: nothing to do, nothing allocated
         xsv_dep_sync();                               // every block waits for the kernel before it, so that the order of the chain holds
@@ -961,12 +974,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_cons
 // that a row's 256 bytes are read by 16 consecutive threads.
 constexpr int MAX_PARTS = 256;         // a unit can be shared by as many CTAs as there are; the launcher keeps G <= MAX_PARTS
 template <typename T>
-__global__ void __launch_bounds__(256) attn_combine_kernel(const Params p) {
+__global__ void __launch_bounds__(256) attn_combine_kernel(const __grid_constant__ BatchParams bp) {
     xsv_dep_release();
+    int s_idx = 0;
+    while (s_idx + 1 < bp.n && (int)blockIdx.y >= bp.unit_base[s_idx + 1]) ++s_idx;
+    const Params& p = bp.p[s_idx];
     __shared__ int s_slot[MAX_PARTS];
     __shared__ int s_cand[MAX_PARTS];      // per candidate CTA: -1 nothing of this unit, -2 the whole unit, else its slot
     __shared__ int s_n, s_b0, s_nb;
-    const int u = blockIdx.y;
+    const int u = (int)blockIdx.y - bp.unit_base[s_idx];
     if (threadIdx.x == 0) {
         long long base;
         int cost;
@@ -1064,9 +1080,9 @@ __global__ void wait_selftest_kernel(int* status) {
 }
 
 template <typename T, int BITS>
-cudaError_t launch(const Params& p, bool merge_only, cudaStream_t st) {
+cudaError_t launch(const BatchParams& bp, bool merge_only, cudaStream_t st) {
     if (merge_only) {
-        xsv_launch_dep(attn_combine_kernel<T>, dim3(16, p.H * p.npair), dim3(256), 0, st, p);
+        xsv_launch_dep(attn_combine_kernel<T>, dim3(16, bp.unit_base[bp.n]), dim3(256), 0, st, bp);
         xsv_count_launch(1);
         return cudaGetLastError();
     }
@@ -1077,7 +1093,7 @@ cudaError_t launch(const Params& p, bool merge_only, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         attr_set.set(dev, 1);
     }
-    xsv_launch_dep(attn_tc5_kernel<T, BITS>, dim3(p.G), dim3(NTHREADS), SMEM_BYTES, st, p);
+    xsv_launch_dep(attn_tc5_kernel<T, BITS>, dim3(bp.cta_base[bp.n]), dim3(NTHREADS), SMEM_BYTES, st, bp);
     xsv_count_launch(1);
     return cudaGetLastError();
 }
@@ -1093,12 +1109,10 @@ cudaError_t xsv_launch_wait_selftest(int* status, cudaStream_t st) {
 size_t xsv_attn_tc5_workspace_bytes() { return (size_t)xsv_sm_count() * 2 * PART_STRIDE * sizeof(float); }
 
 namespace {
-cudaError_t launch_tc5(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V, void* out,
-                       int dtype, int H, int F, float* workspace, int* status, int spare_sms, bool merge_only,
-                       cudaStream_t st) {
-    if (!workspace) return cudaErrorNotSupported;
-    Params p{};
-    p.lv = lv; p.Q = Q; p.K = K; p.V = V; p.out = out; p.part = workspace; p.status = status;
+// The work of one stream (everything of Params but the CTA count and the workspace slice).
+void fill_params(Params& p, const LayerView& lv, int T_c, const void* Q, const void* K, const void* V, void* out, int H,
+                 int F, int* status) {
+    p.lv = lv; p.Q = Q; p.K = K; p.V = V; p.out = out; p.status = status;
     p.T_c = T_c; p.F = F; p.H = H;
     p.n_ct = (T_c + BN - 1) / BN;
     p.nkv = p.n_ct + (F + BN - 1) / BN;
@@ -1106,20 +1120,44 @@ cudaError_t launch_tc5(const LayerView& lv, int T_c, const void* Q, const void* 
     p.n_full = ((p.npair - 1) * 2 * BM + BM < F) ? p.npair : p.npair - 1;
     p.ticks_head = p.n_full * unit_len(p, true) + (p.npair - p.n_full) * unit_len(p, false);
     p.total = p.ticks_head * H;
-    const long long steps = (long long)H * p.npair * p.nkv;
-    const int sms = xsv_sm_count() - spare_sms > 0 ? xsv_sm_count() - spare_sms : 1;   // multiprocessors left to another kernel
-    p.G = (int)(steps < sms ? steps : sms);
-    if (p.G > MAX_PARTS) p.G = MAX_PARTS;
-#define XSV_TC5(TT, B) return launch<TT, B>(p, merge_only, st)
+}
+
+// CTAs of the launch dealt to the streams in proportion to their work (at least one each, never more than a
+// stream has steps); the CTAs of one stream then split that stream's steps among themselves as in a launch of its own.
+void deal_ctas(BatchParams& bp, float* workspace, int sms) {
+    long long total = 0;
+    for (int i = 0; i < bp.n; ++i) total += bp.p[i].total;
+    int used = 0;
+    for (int i = 0; i < bp.n; ++i) {
+        Params& p = bp.p[i];
+        const long long steps = (long long)p.H * p.npair * p.nkv;
+        long long g = total > 0 ? (p.total * sms + total / 2) / total : 1;
+        const int left = sms - used - (bp.n - 1 - i);              // keep one for every stream still to come
+        if (g > left) g = left;
+        if (g > steps) g = steps;
+        if (g > MAX_PARTS) g = MAX_PARTS;
+        if (g < 1) g = 1;
+        p.G = (int)g;
+        p.part = workspace + (size_t)used * 2 * PART_STRIDE;
+        bp.cta_base[i] = used;
+        used += p.G;
+    }
+    bp.cta_base[bp.n] = used;
+    bp.unit_base[0] = 0;
+    for (int i = 0; i < bp.n; ++i) bp.unit_base[i + 1] = bp.unit_base[i] + bp.p[i].H * bp.p[i].npair;
+}
+
+cudaError_t launch_tc5(const BatchParams& bp, int dtype, int bits, bool merge_only, cudaStream_t st) {
+#define XSV_TC5(TT, B) return launch<TT, B>(bp, merge_only, st)
     if (dtype == 0) {
-        switch (lv.bits) {
+        switch (bits) {
             case 2: XSV_TC5(__half, 2);
             case 4: XSV_TC5(__half, 4);
             case 8: XSV_TC5(__half, 8);
             case 16: XSV_TC5(__half, 16);
         }
     } else {
-        switch (lv.bits) {
+        switch (bits) {
             case 2: XSV_TC5(__nv_bfloat16, 2);
             case 4: XSV_TC5(__nv_bfloat16, 4);
             case 8: XSV_TC5(__nv_bfloat16, 8);
@@ -1129,15 +1167,42 @@ cudaError_t launch_tc5(const LayerView& lv, int T_c, const void* Q, const void* 
 #undef XSV_TC5
     return cudaErrorInvalidValue;
 }
+
+cudaError_t launch_one(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V, void* out, int dtype,
+                       int H, int F, float* workspace, int* status, int spare_sms, bool merge_only, cudaStream_t st) {
+    if (!workspace) return cudaErrorNotSupported;
+    BatchParams bp{};
+    bp.n = 1;
+    fill_params(bp.p[0], lv, T_c, Q, K, V, out, H, F, status);
+    const int sms = xsv_sm_count() - spare_sms > 0 ? xsv_sm_count() - spare_sms : 1;   // multiprocessors left to another kernel
+    deal_ctas(bp, workspace, sms);
+    return launch_tc5(bp, dtype, lv.bits, merge_only, st);
+}
 }  // namespace
 
 cudaError_t xsv_launch_attn_tc5(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V, void* out,
                                 int dtype, int H, int F, float* workspace, int* status, int spare_sms, cudaStream_t st) {
-    return launch_tc5(lv, T_c, Q, K, V, out, dtype, H, F, workspace, status, spare_sms, false, st);
+    return launch_one(lv, T_c, Q, K, V, out, dtype, H, F, workspace, status, spare_sms, false, st);
 }
 
 cudaError_t xsv_launch_attn_tc5_merge(const LayerView& lv, int T_c, const void* Q, const void* K, const void* V,
                                       void* out, int dtype, int H, int F, float* workspace, int* status,
                                       int spare_sms, cudaStream_t st) {
-    return launch_tc5(lv, T_c, Q, K, V, out, dtype, H, F, workspace, status, spare_sms, true, st);
+    return launch_one(lv, T_c, Q, K, V, out, dtype, H, F, workspace, status, spare_sms, true, st);
+}
+
+cudaError_t xsv_launch_attn_tc5_batch(int n, const LayerView* lvs, const int* T_cs, const void* const* Qs,
+                                      const void* const* Ks, const void* const* Vs, void* const* outs, int dtype, int H,
+                                      const int* Fs, float* workspace, int* const* statuses, cudaStream_t st) {
+    if (!workspace || n < 1 || n > XSV_MAX_BATCH) return cudaErrorInvalidValue;
+    BatchParams bp{};
+    bp.n = n;
+    for (int i = 0; i < n; ++i) {
+        if (lvs[i].bits != lvs[0].bits) return cudaErrorInvalidValue;
+        fill_params(bp.p[i], lvs[i], T_cs[i], Qs[i], Ks[i], Vs[i], outs[i], H, Fs[i], statuses[i]);
+    }
+    deal_ctas(bp, workspace, xsv_sm_count());
+    cudaError_t e = launch_tc5(bp, dtype, lvs[0].bits, false, st);
+    if (e != cudaSuccess) return e;
+    return launch_tc5(bp, dtype, lvs[0].bits, true, st);
 }

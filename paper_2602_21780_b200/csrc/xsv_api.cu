@@ -88,7 +88,7 @@ struct xsv_cache {
 
     size_t bytes = 0;
 
-    int profiling = 0;          // 0 off, 1 events around every phase, 2 around the attention phase only, 3 around every 7th one
+    int profiling = 0;          // 0 off, 1 events around every phase, 2 around the attention phase only, 3 around every 7th one, 4 as 1 with every kernel on the caller's stream
     unsigned long long attn_calls = 0;
     std::vector<PendingEvent> pending;
     std::vector<cudaEvent_t> free_events;
@@ -238,7 +238,7 @@ struct PhaseTimer {
     bool on;
     PhaseTimer(xsv_cache* c_, cudaStream_t st_, int phase_) : c(c_), st(st_), phase(phase_) {
         launches0 = g_launches.load(std::memory_order_relaxed);
-        on = c->profiling == 1 || (c->profiling == 2 && phase == XSV_PHASE_ATTN) ||
+        on = c->profiling == 1 || c->profiling == 4 || (c->profiling == 2 && phase == XSV_PHASE_ATTN) ||
              (c->profiling == 3 && phase == XSV_PHASE_ATTN && (c->attn_calls++ % 7ull) == 0ull);
         if (on) {
             a = get_event(c);
@@ -325,12 +325,30 @@ xsv_status xsv_cache_set_attn_impl(xsv_cache* c, xsv_attn_impl impl) {
     return XSV_OK;
 }
 
-xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const void* V, int n_tokens,
-                    xsv_dtype dtype, void* out, void* stream) {
+}  // extern "C"
+
+namespace {
+
+// What one step of one cache comes to, worked out on the host before anything is launched.
+struct StepPlan {
+    xsv_cache* c;
+    int layer;
+    const void *Q, *K, *V;
+    void* out;
+    int dtype, F, H;
+    long long T_c, T, t, origin0;
+    bool prune, side_select, append_only;
+    int cur, T_first, n_mid, k;
+};
+
+// Argument, shape and order checks, allocation on the first step, and the step's quantities.  Launches nothing.
+xsv_status plan_step(xsv_cache* c, int layer, const void* Q, const void* K, const void* V, int n_tokens, xsv_dtype dtype,
+                     void* out, bool append_only, StepPlan& p) {
     if (!c || !Q || !K || !V || !out) return XSV_ERR_ARG;
     if (layer < 0 || layer >= c->layers || n_tokens <= 0) return XSV_ERR_ARG;
     if (dtype != XSV_F16 && dtype != XSV_BF16) return XSV_ERR_ARG;
-    if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)out) & 15) return XSV_ERR_SHAPE;
+    if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V) & 15) return XSV_ERR_SHAPE;
+    if (!append_only && ((uintptr_t)out & 15)) return XSV_ERR_SHAPE;
     if (out == Q || out == K || out == V) return XSV_ERR_ARG;
     if (c->F_max != 0 && n_tokens > c->F_max) return XSV_ERR_SHAPE;   // frames may differ in size up to max_frame_tokens
     if (c->dtype >= 0 && (int)dtype != c->dtype) return XSV_ERR_SHAPE;
@@ -338,40 +356,46 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
     long long min_frames = c->frames[0];
     for (int l = 1; l < c->layers; ++l) min_frames = c->frames[l] < min_frames ? c->frames[l] : min_frames;
     if (c->frames[layer] > min_frames) return XSV_ERR_ORDER;   // this layer already took the current frame
-
-    cudaStream_t st = (cudaStream_t)stream;
     if (!c->allocated) {
         c->F_max = n_tokens;          // not told otherwise: no later frame is larger than the first
         cudaSetDevice(c->device);
         xsv_status s = allocate(c);
         if (s != XSV_OK) { c->F_max = 0; return s; }
     }
-    const int F = n_tokens, H = c->H;
-    const long long T_c = c->len[layer];
-    const long long T = T_c + F;
-    const long long t = c->frames[layer] + 1;
-    const bool prune = t >= 2 && c->L_max > 0 && T > c->L_max;
-    if (!prune && T > c->cap) return XSV_ERR_CAPACITY;
-    c->dtype = (int)dtype;
-    c->stepped = true;
-
-    const int cur = c->buf_of_layer[layer];
-    const LayerView& lv = c->bufs[cur].view;
-    cudaError_t e;
-
+    p.c = c; p.layer = layer; p.Q = Q; p.K = K; p.V = V; p.out = out; p.dtype = (int)dtype; p.append_only = append_only;
+    p.F = n_tokens; p.H = c->H;
+    p.T_c = c->len[layer];
+    p.T = p.T_c + p.F;
+    p.t = c->frames[layer] + 1;
+    p.prune = p.t >= 2 && c->L_max > 0 && p.T > c->L_max;
+    if (!p.prune && p.T > c->cap) return XSV_ERR_CAPACITY;
+    if (append_only && p.prune) return XSV_ERR_ORDER;      // a step that prunes needs the frame's queries (Eq. 3-7)
+    p.cur = c->buf_of_layer[layer];
     // Eq. 8 with the sizes of the first and of the current frame as separate quantities:
     // k = max(0, L_max - T_first - T_current) of the middle segment's T_c - T_first tokens are kept.
-    const long long origin0 = c->tokens_seen[layer];
-    const int T_first = t == 1 ? F : c->F_first[layer];
-    const int n_mid = (int)(T_c - T_first);
-    const long long kk = c->L_max - T_first - F;
-    const int k = (int)(kk > 0 ? kk : 0);
+    p.origin0 = c->tokens_seen[layer];
+    p.T_first = p.t == 1 ? p.F : c->F_first[layer];
+    p.n_mid = (int)(p.T_c - p.T_first);
+    const long long kk = c->L_max - p.T_first - p.F;
+    p.k = (int)(kk > 0 ? kk : 0);
     // The scores (Eq. 3-7) need the frame's queries and the cached keys only, so they come first; the selection
     // (Eq. 8), one block that is bound by latency, then runs on a stream of its own: it takes the first multiprocessor
     // that an attention CTA leaves (the CTAs' finishing times are spread over some tens of microseconds) and what
     // follows it takes the next ones.  (Keeping one multiprocessor free of attention CTAs for that stream from the
     // start gives 0.7 % more frames per second and 3 % less throughput of the attention kernel; not done.)
-    const bool side_select = prune && side_select_enabled() && c->attn_impl != XSV_ATTN_MMA && c->attn_ws != nullptr;
+    p.side_select = p.prune && side_select_enabled() && c->profiling != 4 && c->attn_impl != XSV_ATTN_MMA && c->attn_ws != nullptr;
+    return XSV_OK;
+}
+
+// Everything of the step that comes before the attention kernel on the caller's stream: the waits for earlier
+// side-stream work, the scores, and (on the cache's own streams) the selection and the re-quantisation.
+xsv_status launch_before_attention(const StepPlan& p, cudaStream_t st) {
+    xsv_cache* c = p.c;
+    const int layer = p.layer, F = p.F, H = p.H, T_first = p.T_first, k = p.k;
+    const LayerView& lv = c->bufs[p.cur].view;
+    cudaError_t e;
+    c->dtype = p.dtype;
+    c->stepped = true;
     // Deferred join: side-stream work of earlier steps may still be running.  This layer's own must have ended before
     // its cache is read, and the last selection before the score buffer is rewritten.
     if (!c->side_pending.empty() && c->side_pending[layer]) {
@@ -383,74 +407,89 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
         if ((e = cudaStreamWaitEvent(st, c->ev_picked, 0)) != cudaSuccess) return cuda_fail(e);
         c->select_outstanding = false;
     }
-    if (prune) {
-        {   // ---- Eq. 3-7
-            PhaseTimer pt(c, st, XSV_PHASE_SCORE);
-            e = xsv_launch_qtilde(Q, (int)dtype, H, F, c->n_special, c->g, c->qpart, st);
-            if (e != cudaSuccess) return cuda_fail(e);
-            const int n_pooled = c->n_special + (F - c->n_special + c->g - 1) / c->g;
-            const float qnorm = 1.0f / ((float)H * (float)n_pooled);
-            if (c->bits == 16) e = xsv_launch_score_raw(lv, (int)dtype, H, T_first, (int)T_c, c->qpart, qnorm, c->scores, st);
-            else e = xsv_launch_score(lv, H, T_first, (int)T_c, c->qpart, qnorm, c->scores, st);
-            if (e != cudaSuccess) return cuda_fail(e);
-        }
-        cudaStream_t sel_st = st;
-        if (side_select) {
-            // the new selection overwrites the kept-position map that the values of the previous step may still read
-            if (c->defer_join && (e = cudaStreamWaitEvent(c->cs_sel, c->ev_values, 0)) != cudaSuccess) return cuda_fail(e);
-            if ((e = cudaEventRecord(c->ev_scored, st)) != cudaSuccess) return cuda_fail(e);
-            if ((e = cudaStreamWaitEvent(c->cs_sel, c->ev_scored, 0)) != cudaSuccess) return cuda_fail(e);
-            sel_st = c->cs_sel;
-        }
-        {   // ---- Eq. 8
-            PhaseTimer pt(c, sel_st, XSV_PHASE_SELECT);
-            e = xsv_launch_select(c->scores, n_mid, k, T_first, (int)T_c, c->srcmap, c->dscal, sel_st);
-            if (e != cudaSuccess) return cuda_fail(e);
-        }
-        if (side_select) {
-            // Eq. 9-11 need the selection only, not the attention output: they follow it into the spare buffer -- the keys
-            // on its stream, the values (two short kernels: kept rows move verbatim, the frame's rows are quantised)
-            // on a third one, so that neither waits for the other -- on the multiprocessors that the attention CTAs
-            // leave one by one, and beside the merge kernel.  The caller's stream waits for both below, so the step ends
-            // when all of it has.
-            if (c->bits < 16) {
-                const LayerView& dv = c->bufs[c->spare].view;
-                if ((e = cudaEventRecord(c->ev_picked, c->cs_sel)) != cudaSuccess) return cuda_fail(e);
-                if ((e = cudaStreamWaitEvent(c->cs_val, c->ev_picked, 0)) != cudaSuccess) return cuda_fail(e);
-                {
-                    PhaseTimer pt(c, c->cs_val, XSV_PHASE_QUANT);
-                    e = xsv_launch_values(lv, dv, V, (int)dtype, H, F, T_first + k, T_first, c->srcmap, origin0, c->status, c->cs_val);
-                    if (e != cudaSuccess) return cuda_fail(e);
-                }
-                if ((e = cudaEventRecord(c->ev_values, c->cs_val)) != cudaSuccess) return cuda_fail(e);
-                PhaseTimer pt(c, sel_st, XSV_PHASE_QUANT);
-                e = xsv_launch_compress(lv, dv, K, V, (int)dtype, H, F, T_first + k, T_first + k + F, T_first, c->srcmap,
-                                        c->dscal, 0, origin0, false, c->status, sel_st);
+    if (!p.prune) return XSV_OK;
+    {   // ---- Eq. 3-7
+        PhaseTimer pt(c, st, XSV_PHASE_SCORE);
+        e = xsv_launch_qtilde(p.Q, p.dtype, H, F, c->n_special, c->g, c->qpart, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+        const int n_pooled = c->n_special + (F - c->n_special + c->g - 1) / c->g;
+        const float qnorm = 1.0f / ((float)H * (float)n_pooled);
+        if (c->bits == 16) e = xsv_launch_score_raw(lv, p.dtype, H, T_first, (int)p.T_c, c->qpart, qnorm, c->scores, st);
+        else e = xsv_launch_score(lv, H, T_first, (int)p.T_c, c->qpart, qnorm, c->scores, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    cudaStream_t sel_st = st;
+    if (p.side_select) {
+        // the new selection overwrites the kept-position map that the values of the previous step may still read
+        if (c->defer_join && (e = cudaStreamWaitEvent(c->cs_sel, c->ev_values, 0)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventRecord(c->ev_scored, st)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamWaitEvent(c->cs_sel, c->ev_scored, 0)) != cudaSuccess) return cuda_fail(e);
+        sel_st = c->cs_sel;
+    }
+    {   // ---- Eq. 8
+        PhaseTimer pt(c, sel_st, XSV_PHASE_SELECT);
+        e = xsv_launch_select(c->scores, p.n_mid, k, T_first, (int)p.T_c, c->srcmap, c->dscal, sel_st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (p.side_select) {
+        // Eq. 9-11 need the selection only, not the attention output: they follow it into the spare buffer -- the keys
+        // on its stream, the values (two short kernels: kept rows move verbatim, the frame's rows are quantised)
+        // on a third one, so that neither waits for the other -- on the multiprocessors that the attention CTAs
+        // leave one by one, and beside the merge kernel.  The caller's stream waits for both afterwards, so the step
+        // ends when all of it has.
+        if (c->bits < 16) {
+            const LayerView& dv = c->bufs[c->spare].view;
+            if ((e = cudaEventRecord(c->ev_picked, c->cs_sel)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaStreamWaitEvent(c->cs_val, c->ev_picked, 0)) != cudaSuccess) return cuda_fail(e);
+            {
+                PhaseTimer pt(c, c->cs_val, XSV_PHASE_QUANT);
+                e = xsv_launch_values(lv, dv, p.V, p.dtype, H, F, T_first + k, T_first, c->srcmap, p.origin0, c->status, c->cs_val);
                 if (e != cudaSuccess) return cuda_fail(e);
             }
-            if ((e = cudaEventRecord(c->ev_selected, c->cs_sel)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaEventRecord(c->ev_values, c->cs_val)) != cudaSuccess) return cuda_fail(e);
+            PhaseTimer pt(c, sel_st, XSV_PHASE_QUANT);
+            e = xsv_launch_compress(lv, dv, p.K, p.V, p.dtype, H, F, T_first + k, T_first + k + F, T_first, c->srcmap,
+                                    c->dscal, 0, p.origin0, false, c->status, sel_st);
+            if (e != cudaSuccess) return cuda_fail(e);
         }
+        if ((e = cudaEventRecord(c->ev_selected, c->cs_sel)) != cudaSuccess) return cuda_fail(e);
     }
+    return XSV_OK;
+}
 
-    // ---- Eq. 2 / Eq. 12: attention over [cache ; frame]
+// ---- Eq. 2 / Eq. 12: attention of one cache's frame over [cache ; frame]
+xsv_status launch_attention(const StepPlan& p, cudaStream_t st) {
+    xsv_cache* c = p.c;
+    const LayerView& lv = c->bufs[p.cur].view;
+    cudaError_t e;
     bool tc5 = false;
     {
         PhaseTimer pt(c, st, XSV_PHASE_ATTN);      // the attention kernel proper; the merge of shared tiles follows
         e = cudaErrorNotSupported;
         if (c->attn_impl != XSV_ATTN_MMA)
-            e = xsv_launch_attn_tc5(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, c->attn_ws, c->status, 0, st);
+            e = xsv_launch_attn_tc5(lv, (int)p.T_c, p.Q, p.K, p.V, p.out, p.dtype, p.H, p.F, c->attn_ws, c->status, 0, st);
         tc5 = (e == cudaSuccess);
         if (e == cudaErrorNotSupported) {
             if (c->attn_impl == XSV_ATTN_TC5) return XSV_ERR_ARG;
-            e = xsv_launch_attn_mma(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, st);
+            e = xsv_launch_attn_mma(lv, (int)p.T_c, p.Q, p.K, p.V, p.out, p.dtype, p.H, p.F, st);
         }
         if (e != cudaSuccess) return cuda_fail(e);
     }
     if (tc5) {
-        e = xsv_launch_attn_tc5_merge(lv, (int)T_c, Q, K, V, out, (int)dtype, H, F, c->attn_ws, c->status, 0, st);
+        e = xsv_launch_attn_tc5_merge(lv, (int)p.T_c, p.Q, p.K, p.V, p.out, p.dtype, p.H, p.F, c->attn_ws, c->status, 0, st);
         if (e != cudaSuccess) return cuda_fail(e);
     }
-    const bool deferred = side_select && c->defer_join && c->bits < 16;
+    return XSV_OK;
+}
+
+// What follows the attention: the join with the cache's own streams (or its deferral), the cache update of a
+// step that does not prune, and the bookkeeping.
+xsv_status launch_after_attention(const StepPlan& p, cudaStream_t st) {
+    xsv_cache* c = p.c;
+    const int layer = p.layer, F = p.F, H = p.H, T_first = p.T_first, k = p.k;
+    const LayerView& lv = c->bufs[p.cur].view;
+    cudaError_t e = cudaSuccess;
+    const bool deferred = p.side_select && c->defer_join && c->bits < 16;
     if (deferred) {
         // the caller's stream goes on; it waits for this layer's side-stream work when the layer is stepped again
         // (or in xsv_cache_join)
@@ -459,46 +498,111 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
         c->side_pending[layer] = 1;
         c->select_outstanding = true;
     } else {
-        if (side_select && (e = cudaStreamWaitEvent(st, c->ev_selected, 0)) != cudaSuccess) return cuda_fail(e);
-        if (side_select && c->bits < 16 && (e = cudaStreamWaitEvent(st, c->ev_values, 0)) != cudaSuccess) return cuda_fail(e);
+        if (p.side_select && (e = cudaStreamWaitEvent(st, c->ev_selected, 0)) != cudaSuccess) return cuda_fail(e);
+        if (p.side_select && c->bits < 16 && (e = cudaStreamWaitEvent(st, c->ev_values, 0)) != cudaSuccess) return cuda_fail(e);
     }
-
-    if (prune) {
+    if (p.prune) {
         const int n_old_new = T_first + k;
         const int T_new = n_old_new + F;
         const LayerView& dv = c->bufs[c->spare].view;
         {   // ---- Eq. 9-11 on the new order [first ; kept ; current], written to the spare buffer
             PhaseTimer pt(c, st, XSV_PHASE_QUANT);
             if (c->bits == 16) {
-                e = xsv_launch_raw_update(lv, dv, K, V, H, F, n_old_new, T_first, c->srcmap, origin0, st);
+                e = xsv_launch_raw_update(lv, dv, p.K, p.V, H, F, n_old_new, T_first, c->srcmap, p.origin0, st);
             } else {
-                if (!side_select)
-                    e = xsv_launch_compress(lv, dv, K, V, (int)dtype, H, F, n_old_new, T_new, T_first, c->srcmap, c->dscal, 0,
-                                            origin0, true, c->status, st);
+                if (!p.side_select)
+                    e = xsv_launch_compress(lv, dv, p.K, p.V, p.dtype, H, F, n_old_new, T_new, T_first, c->srcmap, c->dscal, 0,
+                                            p.origin0, true, c->status, st);
             }
             if (e != cudaSuccess) return cuda_fail(e);
         }
         c->buf_of_layer[layer] = c->spare;
-        c->spare = cur;
+        c->spare = p.cur;
         c->len[layer] = T_new;
-        c->last_scores_n = n_mid;
+        c->last_scores_n = p.n_mid;
     } else {
         // append in place: cached tokens keep their slots; the partial tail key
         // group (if any) is rebuilt together with the fresh tokens
         PhaseTimer pt(c, st, XSV_PHASE_QUANT);
         if (c->bits == 16) {
-            e = xsv_launch_raw_update(lv, lv, K, V, H, F, (int)T_c, F, nullptr, origin0, st);
+            e = xsv_launch_raw_update(lv, lv, p.K, p.V, H, F, (int)p.T_c, F, nullptr, p.origin0, st);
         } else {
-            e = xsv_launch_compress(lv, lv, K, V, (int)dtype, H, F, (int)T_c, (int)T, F, nullptr, nullptr,
-                                    (int)(T_c / XSV_G), origin0, true, c->status, st);
+            e = xsv_launch_compress(lv, lv, p.K, p.V, p.dtype, H, F, (int)p.T_c, (int)p.T, F, nullptr, nullptr,
+                                    (int)(p.T_c / XSV_G), p.origin0, true, c->status, st);
         }
         if (e != cudaSuccess) return cuda_fail(e);
-        c->len[layer] = T;
+        c->len[layer] = p.T;
         c->last_scores_n = 0;
     }
-    c->frames[layer] = t;
-    c->tokens_seen[layer] = origin0 + F;
-    if (t == 1) c->F_first[layer] = F;
+    c->frames[layer] = p.t;
+    c->tokens_seen[layer] = p.origin0 + F;
+    if (p.t == 1) c->F_first[layer] = F;
+    return XSV_OK;
+}
+
+xsv_status step_impl(xsv_cache* c, int layer, const void* Q, const void* K, const void* V, int n_tokens,
+                     xsv_dtype dtype, void* out, void* stream, bool append_only) {
+    StepPlan p{};
+    xsv_status s = plan_step(c, layer, Q, K, V, n_tokens, dtype, out, append_only, p);
+    if (s != XSV_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    if ((s = launch_before_attention(p, st)) != XSV_OK) return s;
+    if (!append_only && (s = launch_attention(p, st)) != XSV_OK) return s;
+    return launch_after_attention(p, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const void* V, int n_tokens,
+                    xsv_dtype dtype, void* out, void* stream) {
+    return step_impl(c, layer, Q, K, V, n_tokens, dtype, out, stream, false);
+}
+
+xsv_status xsv_cache_append(xsv_cache* c, int layer, const void* K, const void* V, int n_tokens, xsv_dtype dtype,
+                            void* stream) {
+    // Q and out are not touched on this path; K stands in for them in the argument checks
+    return step_impl(c, layer, K, K, V, n_tokens, dtype, c, stream, true);
+}
+
+xsv_status xsv_step_batch(xsv_cache* const* caches, int n, int layer, const void* const* Q, const void* const* K,
+                          const void* const* V, const int* n_tokens, xsv_dtype dtype, void* const* out, void* stream) {
+    if (!caches || !Q || !K || !V || !n_tokens || !out || n <= 0 || n > XSV_MAX_BATCH) return XSV_ERR_ARG;
+    StepPlan plans[XSV_MAX_BATCH];
+    for (int i = 0; i < n; ++i) {
+        for (int j = 0; j < i; ++j)
+            if (caches[i] == caches[j]) return XSV_ERR_ARG;
+        const xsv_status s = plan_step(caches[i], layer, Q[i], K[i], V[i], n_tokens[i], dtype, out[i], false, plans[i]);
+        if (s != XSV_OK) return s;                      // nothing has been launched: every cache is unchanged
+        const xsv_cache* a = caches[0];
+        const xsv_cache* b = caches[i];
+        if (b->device != a->device || b->H != a->H || b->bits != a->bits) return XSV_ERR_SHAPE;
+        if (b->attn_impl == XSV_ATTN_MMA || !b->attn_ws) return XSV_ERR_ARG;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    xsv_status s;
+    for (int i = 0; i < n; ++i)
+        if ((s = launch_before_attention(plans[i], st)) != XSV_OK) return s;
+    {   // one attention launch and one merge launch for all streams
+        LayerView lvs[XSV_MAX_BATCH];
+        int T_cs[XSV_MAX_BATCH], Fs[XSV_MAX_BATCH];
+        const void *Qs[XSV_MAX_BATCH], *Ks[XSV_MAX_BATCH], *Vs[XSV_MAX_BATCH];
+        void* outs[XSV_MAX_BATCH];
+        int* statuses[XSV_MAX_BATCH];
+        for (int i = 0; i < n; ++i) {
+            lvs[i] = caches[i]->bufs[plans[i].cur].view;
+            T_cs[i] = (int)plans[i].T_c; Fs[i] = plans[i].F;
+            Qs[i] = Q[i]; Ks[i] = K[i]; Vs[i] = V[i]; outs[i] = out[i];
+            statuses[i] = caches[i]->status;
+        }
+        PhaseTimer pt(caches[0], st, XSV_PHASE_ATTN);
+        cudaError_t e = xsv_launch_attn_tc5_batch(n, lvs, T_cs, Qs, Ks, Vs, outs, (int)dtype, caches[0]->H, Fs,
+                                                  caches[0]->attn_ws, statuses, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    for (int i = 0; i < n; ++i)
+        if ((s = launch_after_attention(plans[i], st)) != XSV_OK) return s;
     return XSV_OK;
 }
 
@@ -860,7 +964,7 @@ int xsv_cache_status_word(xsv_cache* c, void* stream) {
 
 xsv_status xsv_cache_set_profiling(xsv_cache* c, int on) {
     if (!c) return XSV_ERR_ARG;
-    if (on < 0 || on > 3) return XSV_ERR_ARG;
+    if (on < 0 || on > 4) return XSV_ERR_ARG;
     if (on && c->free_events.empty() && c->pending.empty()) {
         // a pool of timing events, so that the steps that follow create none
         cudaSetDevice(c->device);

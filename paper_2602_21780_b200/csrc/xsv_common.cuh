@@ -9,6 +9,9 @@
 
 #define XSV_D 64   // channels per head (head_dim)
 #define XSV_G 64   // quantisation group size (tokens for K, channels for V)
+#ifndef XSV_MAX_BATCH
+#define XSV_MAX_BATCH 8   // streams per batched launch (also in the public header)
+#endif
 
 // Bits of the sticky device status word.
 #define XSV_DEV_TIMEOUT 1

@@ -71,6 +71,12 @@ cudaError_t xsv_launch_attn_tc5_merge(const LayerView& lv, int T_c, const void* 
                                       void* out, int dtype, int H, int F, float* workspace, int* status,
                                       int spare_sms, cudaStream_t st);
 
+// The attention of several independent streams (each with its own cache view, inputs, output and status word) and
+// the merge that follows, as one launch each; all streams share dtype, bit width and head count.  `workspace` as above.
+cudaError_t xsv_launch_attn_tc5_batch(int n, const LayerView* lvs, const int* T_cs, const void* const* Qs,
+                                      const void* const* Ks, const void* const* Vs, void* const* outs, int dtype, int H,
+                                      const int* Fs, float* workspace, int* const* statuses, cudaStream_t st);
+
 // One small kernel whose only wait can never be satisfied: it must come back after the
 // attention kernel's wait limit with XSV_DEV_TIMEOUT set in *status (device int).
 cudaError_t xsv_launch_wait_selftest(int* status, cudaStream_t st);

@@ -188,3 +188,72 @@ def device_stream(H, F, dtype, seed, d=64, pool=4, drift_rho=None):
         return tuple(x.to(td).contiguous() for x in (q, k, v))
 
     return fn
+
+
+def run_batch(streams, frames, L_max, bits, starts=None, check_steps=None, deferred_join=False):
+    """Several independent streams stepped together through xsv_step_batch, each verified against its own oracle
+    with the step-locked protocol of run_stream.  streams: synth.Stream objects (same heads and dtype; frame sizes
+    may differ); starts[i]: the frame at which stream i joins (so that lengths differ and some streams prune while
+    others still append).  Returns the worst errors over all streams."""
+    B = len(streams)
+    starts = starts or [0] * B
+    H, d, dtype = streams[0].H, streams[0].d, streams[0].dtype
+    caches = [binding.Cache(1, H, d, L_max, bits) for _ in range(B)]
+    for c in caches:
+        c.set_deferred_join(deferred_join)
+    refs = [orc.LayerCache(H, d, L_max, bits) for _ in range(B)]
+    for r in refs:
+        r._dtype = dtype
+    track = [dict(F_first=0, F_prev=0, seen=0, T=0, t=0) for _ in range(B)]
+    worst = dict(attn=0.0, score=0.0, pruned_steps=0, checked=0, batched_calls=0)
+    for t in range(frames):
+        active = [i for i in range(B) if t >= starts[i]]
+        data = {i: streams[i].frame(t - starts[i]) for i in active}
+        dev = {i: tuple(to_dev(x, dtype) for x in data[i]) for i in active}
+        outs = {i: torch.empty_like(dev[i][0]) for i in active}
+        checked = check_steps is None or t in check_steps
+        if checked:
+            for i in active:
+                st0 = caches[i].export_layer(0)
+                tr = track[i]
+                if tr["t"] > 0:
+                    check_state_invariants(st0, bits, tr["F_first"], tr["F_prev"], tr["seen"], tr["T"])
+                load_oracle_state(refs[i], st0, tr["t"], tr["F_first"])
+        binding.step_batch([caches[i] for i in active], 0, [dev[i][0] for i in active], [dev[i][1] for i in active],
+                           [dev[i][2] for i in active], [outs[i] for i in active])
+        worst["batched_calls"] += 1
+        torch.cuda.synchronize()
+        for i in active:
+            tr = track[i]
+            F = data[i][0].shape[1]
+            if tr["t"] == 0:
+                tr["F_first"] = F
+            tr["T"] = orc.next_cache_len(tr["t"] + 1, tr["T"], tr["F_first"], F, L_max)
+            tr["seen"] += F
+            tr["F_prev"] = F
+            tr["t"] += 1
+            assert caches[i].len(0) == tr["T"]
+        if not checked:
+            continue
+        for i in active:
+            q, k, v = data[i]
+            ref = refs[i]
+            S_gpu = caches[i].last_scores()
+            o_ref = ref.step(q, k, v, select_on=S_gpu.astype(np.float64) if S_gpu.size else None)
+            o_gpu = outs[i].float().cpu().numpy().astype(np.float64)
+            assert np.all(np.isfinite(o_gpu)), f"step {t}, stream {i}: non-finite attention output"
+            e = float(np.max(np.abs(o_gpu - o_ref)) / np.max(np.abs(o_ref)))
+            worst["attn"] = max(worst["attn"], e)
+            assert e <= ATTN_TOL, f"step {t}, stream {i}: attention error {e:.3e} of max|out|"
+            if ref.last_scores is not None and ref.last_scores.size:
+                assert S_gpu.shape == ref.last_scores.shape
+                es = float(np.max(np.abs(S_gpu - ref.last_scores)) / np.max(np.abs(ref.last_scores)))
+                worst["score"] = max(worst["score"], es)
+                assert es <= SCORE_TOL, f"step {t}, stream {i}: score error {es:.3e} of max|S|"
+                worst["pruned_steps"] += 1
+            compare_states(caches[i].export_layer(0), ref, bits, f"step {t}, stream {i}")
+            worst["checked"] += 1
+    for c in caches:
+        assert c.status() == 0
+        c.destroy()
+    return worst

@@ -6,7 +6,7 @@ import torch
 
 from oracle import xsv_oracle as orc
 from paper_2602_21780_b200 import binding, synth
-from tests.gpu_harness import device_stream, run_stream, to_dev
+from tests.gpu_harness import device_stream, run_batch, run_stream, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -202,6 +202,35 @@ def test_config3_long_horizon_samples(bits):
                    device_fn=device_stream(c["H"], c["F"], c["dtype"], seed=103, drift_rho=c["drift_rho"]))
     assert w["checked"] == 3 and w["pruned_steps"] == 3
     assert w["attn_skipped"] == 0 and w["key_magnitude"] < 128.0
+
+
+@pytest.mark.parametrize("B", [2, 4, 8])
+def test_several_streams_in_one_launch(B):
+    # B independent video streams stepped together: one attention launch for all of them, every stream compared with
+    # its own oracle at every step.  The streams join one frame apart, so that their cache lengths differ and some
+    # prune while others still append; frame sizes differ between streams as well
+    streams = [synth.Stream(H=4, d=64, F=200 - 15 * (i % 3), dtype="bf16", layer=60 + i) for i in range(B)]
+    w = run_batch(streams, 7 + B // 2, 640, 4, starts=[i // 2 for i in range(B)])
+    assert w["pruned_steps"] >= 2 * B and w["checked"] >= 5 * B
+
+
+def test_two_streams_at_paper_shape_and_two_bits():
+    streams = [synth.Stream(H=16, d=64, F=F_PAPER, dtype="bf16", layer=70 + i) for i in range(2)]
+    w = run_batch(streams, 5, 3 * F_PAPER, 2, starts=[0, 1], check_steps={3, 4}, deferred_join=True)
+    assert w["pruned_steps"] >= 3
+
+
+def test_batch_rejects_mismatched_caches_before_launching():
+    a, b = binding.Cache(1, 4, 64, 500, 4), binding.Cache(1, 4, 64, 500, 2)
+    Q = torch.zeros(4, 100, 64, device="cuda", dtype=torch.float16)
+    outs = [torch.empty_like(Q), torch.empty_like(Q)]
+    with pytest.raises(binding.XsvError) as e:
+        binding.step_batch([a, b], 0, [Q, Q], [Q, Q], [Q, Q], outs)
+    assert e.value.code == 2 and a.len(0) == 0 and b.len(0) == 0           # different bit widths: nothing was stepped
+    with pytest.raises(binding.XsvError) as e:
+        binding.step_batch([a, a], 0, [Q, Q], [Q, Q], [Q, Q], outs)
+    assert e.value.code == 1 and a.len(0) == 0
+    a.destroy(); b.destroy()
 
 
 def test_config1_every_step():
