@@ -12,6 +12,8 @@ untimed prefill frames first).  Prints ONE JSON line.
                                   per-frame latency p50 / p99 over frames 100-1000, its slope, bytes at start and end
   python bench.py --config 4      one layer: budgets {4096, 16384, 65536} x bits {2, 4, 8} x frames {32, 256}, and the
                                   uncompressed bf16 cache grown to a share of the free memory, timed at checkpoints
+  python bench.py --batch B       B independent streams stepped together (xsv_step_batch) against the same B streams
+                                  stepped one after the other, at the benchmark's budget and at a budget of 4096
 
 N > 1 (under torchrun): the path does not shard -- every rank runs an independent
 replica (its own stream of frames); value = all ranks' frames / max-over-ranks time.
@@ -426,6 +428,57 @@ def run_config4(args, torch, binding, dev, stream):
     print(json.dumps(line), flush=True)
 
 
+def run_batch_bench(args, torch, binding, dev, stream):
+    """B independent streams, `layers` layers each, in steady state: frames/s of all streams together when every
+    layer-step is one xsv_step_batch call over the B streams, against the same streams stepped one after the other."""
+    B, layers, n_frames = args.batch, min(args.layers, 4), max(args.steps, 10)
+    sp = stream.cuda_stream
+    pools = [gen_frames(torch, dev, layers, 2, seed=20260221 + 10 + b) for b in range(B)]
+    outs = [torch.empty(H, F, D, device=dev, dtype=torch.bfloat16) for _ in range(B)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rows = []
+    for budget in (L_MAX, 4096):
+        res = {}
+        for mode in ("sequential", "batched"):
+            caches = [binding.Cache(layers, H, D, budget, BITS) for _ in range(B)]
+
+            def frame(f):
+                if mode == "sequential":
+                    for b in range(B):
+                        for l in range(layers):
+                            q, k, v = pools[b][l][f % 2]
+                            rc = caches[b].step_raw(l, q.data_ptr(), k.data_ptr(), v.data_ptr(), F, binding.BF16, outs[b].data_ptr(), sp)
+                            if rc != 0:
+                                raise RuntimeError(f"xsv_step failed: status {rc}")
+                else:
+                    for l in range(layers):
+                        qkv = [pools[b][l][f % 2] for b in range(B)]
+                        binding.step_batch(caches, l, [x[0] for x in qkv], [x[1] for x in qkv], [x[2] for x in qkv], outs, stream)
+
+            prefill = budget // F + 3
+            for f in range(prefill):
+                frame(f)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for f in range(n_frames):
+                frame(prefill + f)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+            for c in caches:
+                assert c.status() == 0
+                c.destroy()
+            res[mode] = B * n_frames / (ms * 1e-3)          # frames of all streams per second (of a `layers`-layer stack)
+        rows.append({"budget": budget, "streams": B, "layers": layers, "frames_per_s_sequential": res["sequential"],
+                     "frames_per_s_batched": res["batched"], "ratio": res["batched"] / res["sequential"]})
+    line = {"metric": f"frames/s of {B} streams stepped together vs one after the other ({layers}-layer stacks)", "value": rows[0]["ratio"],
+            "unit": "ratio batched / sequential at the benchmark's budget", "n_gpus": 1, "steps": n_frames, "higher_is_better": True,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"{B} streams x {layers} layers x (16 heads x 64), 1374 tokens/frame, {BITS}-bit KV, bf16, steady state"},
+            "rows": rows}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     global LAYERS, WORKLOAD, L_MAX, BITS, PREFILL
     ap = argparse.ArgumentParser()
@@ -445,6 +498,7 @@ def main():
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4],
                     help="2: the benchmark (default); 3: the long-horizon run; 4: the one-layer sweep and the uncompressed cache")
     ap.add_argument("--frames", type=int, default=0, help="--config 3: frames to stream (default 1000)")
+    ap.add_argument("--batch", type=int, default=0, help="streams stepped together (2-8): the batched-against-sequential comparison")
     ap.add_argument("--max-gb", type=float, default=120.0,
                     help="--config 4: cap in GB on the uncompressed cache (it also stays below 85 %% of the free memory)")
     args = ap.parse_args()
@@ -478,9 +532,10 @@ def main():
 
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if args.config in (3, 4):
+    if args.config in (3, 4) or args.batch:
         if rank == 0:
-            (run_config3 if args.config == 3 else run_config4)(args, torch, binding, dev, torch.cuda.current_stream())
+            fn = run_batch_bench if args.batch else (run_config3 if args.config == 3 else run_config4)
+            fn(args, torch, binding, dev, torch.cuda.current_stream())
         return
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)

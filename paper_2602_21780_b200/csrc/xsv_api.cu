@@ -338,6 +338,7 @@ struct StepPlan {
     int dtype, F, H;
     long long T_c, T, t, origin0;
     bool prune, side_select, append_only;
+    bool scores_on_side;      // the scores run on the cache's own stream too (several caches stepped together)
     int cur, T_first, n_mid, k;
 };
 
@@ -408,22 +409,33 @@ xsv_status launch_before_attention(const StepPlan& p, cudaStream_t st) {
         c->select_outstanding = false;
     }
     if (!p.prune) return XSV_OK;
+    const bool side_scores = p.side_select && p.scores_on_side;
+    if (side_scores) {
+        // Several caches stepped together: each cache's scores run on its own stream, side by side with the other
+        // caches', from the point the caller's stream has reached (the inputs are ready there).
+        if (c->defer_join && (e = cudaStreamWaitEvent(c->cs_sel, c->ev_values, 0)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaEventRecord(c->ev_scored, st)) != cudaSuccess) return cuda_fail(e);
+        if ((e = cudaStreamWaitEvent(c->cs_sel, c->ev_scored, 0)) != cudaSuccess) return cuda_fail(e);
+    }
     {   // ---- Eq. 3-7
-        PhaseTimer pt(c, st, XSV_PHASE_SCORE);
-        e = xsv_launch_qtilde(p.Q, p.dtype, H, F, c->n_special, c->g, c->qpart, st);
+        cudaStream_t sc_st = side_scores ? c->cs_sel : st;
+        PhaseTimer pt(c, sc_st, XSV_PHASE_SCORE);
+        e = xsv_launch_qtilde(p.Q, p.dtype, H, F, c->n_special, c->g, c->qpart, sc_st);
         if (e != cudaSuccess) return cuda_fail(e);
         const int n_pooled = c->n_special + (F - c->n_special + c->g - 1) / c->g;
         const float qnorm = 1.0f / ((float)H * (float)n_pooled);
-        if (c->bits == 16) e = xsv_launch_score_raw(lv, p.dtype, H, T_first, (int)p.T_c, c->qpart, qnorm, c->scores, st);
-        else e = xsv_launch_score(lv, H, T_first, (int)p.T_c, c->qpart, qnorm, c->scores, st);
+        if (c->bits == 16) e = xsv_launch_score_raw(lv, p.dtype, H, T_first, (int)p.T_c, c->qpart, qnorm, c->scores, sc_st);
+        else e = xsv_launch_score(lv, H, T_first, (int)p.T_c, c->qpart, qnorm, c->scores, sc_st);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     cudaStream_t sel_st = st;
     if (p.side_select) {
-        // the new selection overwrites the kept-position map that the values of the previous step may still read
-        if (c->defer_join && (e = cudaStreamWaitEvent(c->cs_sel, c->ev_values, 0)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaEventRecord(c->ev_scored, st)) != cudaSuccess) return cuda_fail(e);
-        if ((e = cudaStreamWaitEvent(c->cs_sel, c->ev_scored, 0)) != cudaSuccess) return cuda_fail(e);
+        if (!side_scores) {
+            // the new selection overwrites the kept-position map that the values of the previous step may still read
+            if (c->defer_join && (e = cudaStreamWaitEvent(c->cs_sel, c->ev_values, 0)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaEventRecord(c->ev_scored, st)) != cudaSuccess) return cuda_fail(e);
+            if ((e = cudaStreamWaitEvent(c->cs_sel, c->ev_scored, 0)) != cudaSuccess) return cuda_fail(e);
+        }
         sel_st = c->cs_sel;
     }
     {   // ---- Eq. 8
@@ -579,6 +591,7 @@ xsv_status xsv_step_batch(xsv_cache* const* caches, int n, int layer, const void
         const xsv_cache* b = caches[i];
         if (b->device != a->device || b->H != a->H || b->bits != a->bits) return XSV_ERR_SHAPE;
         if (b->attn_impl == XSV_ATTN_MMA || !b->attn_ws) return XSV_ERR_ARG;
+        plans[i].scores_on_side = n > 1;
     }
     cudaStream_t st = (cudaStream_t)stream;
     xsv_status s;
