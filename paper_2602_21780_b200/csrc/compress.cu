@@ -72,29 +72,23 @@ __global__ void __launch_bounds__(256) qtilde_partial_kernel(const T* __restrict
     }
 }
 
-// Fixed-order sum of the n_part partial rows, written over the first row: qpart[0..64) = sum_h sum_i w_i Q[h,i,:].
-// 1024 threads: 16 per channel, each sums every 16th row (loads issued eight at a time), then a fixed-order sum of the 16.
-__global__ void __launch_bounds__(1024) qtilde_final_kernel(float* __restrict__ qpart, int n_part) {
-    xsv_dep_release();
-    xsv_dep_sync();
-    __shared__ float red[16][64];
+// q~ = sum_h sum_i w_i Q[h,i,:] from the n_part partial rows, summed in one fixed order by every block that needs
+// it (the partial rows are 32 KB and stay in the L2; a kernel of its own for this sum cost more than the reads).
+// 256 threads: four per channel, each sums every fourth row with its loads eight at a time; qt[64] in shared memory.
+__device__ __forceinline__ void qtilde_sum(const float* __restrict__ qpart, int n_part, float qnorm, float (*red)[64], float* qt) {
     const int c = threadIdx.x & 63, part = threadIdx.x >> 6;
     float s = 0.f;
-    for (int k0 = part; k0 < n_part; k0 += 16 * 8) {
+    for (int k0 = part; k0 < n_part; k0 += 4 * 8) {
         float v[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = (k0 + 16 * j < n_part) ? qpart[(size_t)(k0 + 16 * j) * 64 + c] : 0.f;
+        for (int j = 0; j < 8; ++j) v[j] = (k0 + 4 * j < n_part) ? qpart[(size_t)(k0 + 4 * j) * 64 + c] : 0.f;
 #pragma unroll
         for (int j = 0; j < 8; ++j) s += v[j];
     }
     red[part][c] = s;
-    __syncthreads();       // every partial row has been read
-    if (threadIdx.x < 64) {
-        float t = 0.f;
-#pragma unroll
-        for (int k = 0; k < 16; ++k) t += red[k][c];
-        qpart[c] = t;
-    }
+    __syncthreads();
+    if (threadIdx.x < 64) qt[c] = (((red[0][c] + red[1][c]) + red[2][c]) + red[3][c]) * qnorm;
+    __syncthreads();
 }
 
 // ---------------------------------------------------------------------------
@@ -114,10 +108,14 @@ constexpr int SCORE_ROWS = 4;              // rows a thread holds in registers a
 
 template <int BITS>
 __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, int T_first, int T_c,
-                                                          const float* __restrict__ qfinal, float qnorm,
+                                                          const float* __restrict__ qpart, int n_part, float qnorm,
                                                           float* __restrict__ scores) {
     xsv_dep_release();
-    xsv_dep_sync();
+    // The kernels before this one in the stream (the partial sums of the queries, the merge of the previous step's
+    // attention) do not touch the cache: the packed rows and the groups' parameters are loaded before the wait for
+    // them, and only the partial sums are read after it.
+    __shared__ float q_red[4][64];
+    __shared__ __align__(16) float q_t[64];
     constexpr int ROWB = XSV_D * BITS / 8;
     constexpr int NV = ROWB / 16;              // 16-byte loads per row
     constexpr int SUB = (BITS == 8) ? 2 : (BITS == 4 ? 4 : 8);   // codes per 16-bit sub-word
@@ -148,9 +146,11 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
             }
         }
         if (hb == 0) {
+            xsv_dep_sync();
+            qtilde_sum(qpart, n_part, qnorm, q_red, q_t);
             // weights and bias: one warp per head at a time, lane l takes channels l and l + 32 (same position in
             // their sub-words)
-            const float q0 = qfinal[lane] * qnorm, q1 = qfinal[lane + 32] * qnorm;
+            const float q0 = q_t[lane], q1 = q_t[lane + 32];
             const float pos = __int_as_float((127 - BITS * ((lane & 7) % SUB)) << 23);
             for (int h0 = warp; h0 < H; h0 += 2 * (SCORE_TPB / 32)) {     // two heads per pass: eight loads in flight
                 float sc[2][2], zz[2][2];
@@ -226,13 +226,13 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
 // rows (4 KB) of one head, a thread one 128-byte row at a time with the next one already in flight.
 template <typename T>
 __global__ void __launch_bounds__(SCORE_TPB) score_raw_kernel(LayerView lv, int H, int T_first, int T_c,
-                                                              const float* __restrict__ qpart, float qnorm,
+                                                              const float* __restrict__ qpart, int n_part, float qnorm,
                                                               float* __restrict__ scores) {
     xsv_dep_release();
     xsv_dep_sync();
     __shared__ __align__(16) float qt[64];
     __shared__ float part[4][64];
-    if (threadIdx.x < 64) qt[threadIdx.x] = qpart[threadIdx.x] * qnorm;
+    qtilde_sum(qpart, n_part, qnorm, part, qt);
     const int tok = threadIdx.x & 63, slice = threadIdx.x >> 6;
     const int j = blockIdx.x * 64 + tok;
     const int p = T_first + j;
@@ -1120,8 +1120,7 @@ cudaError_t xsv_launch_qtilde(const void* Q, int dtype, int H, int F, int n_spec
     dim3 grid(XSV_QCHUNKS, H);
     if (dtype == 0) xsv_launch_dep(qtilde_partial_kernel<__half>, grid, dim3(256), 0, st, (const __half*)Q, F, n_special, g, qpart);
     else xsv_launch_dep(qtilde_partial_kernel<__nv_bfloat16>, grid, dim3(256), 0, st, (const __nv_bfloat16*)Q, F, n_special, g, qpart);
-    xsv_launch_dep(qtilde_final_kernel, dim3(1), dim3(1024), 0, st, qpart, H * XSV_QCHUNKS);
-    xsv_count_launch(2);
+    xsv_count_launch(1);
     return cudaGetLastError();
 }
 
@@ -1141,7 +1140,7 @@ cudaError_t xsv_launch_score(const LayerView& lv, int H, int T_first, int T_c, c
             if (e != cudaSuccess) return e;                                                                \
             attr_set.set(dev, (int)smem);                                                                  \
         }                                                                                                  \
-        xsv_launch_dep(score_kernel<B>, dim3(grid), dim3(SCORE_TPB), smem, st, lv, H, T_first, T_c, qpart, qnorm, scores); \
+        xsv_launch_dep(score_kernel<B>, dim3(grid), dim3(SCORE_TPB), smem, st, lv, H, T_first, T_c, qpart, H * XSV_QCHUNKS, qnorm, scores); \
     }
     switch (lv.bits) {
         case 2: XSV_SCORE(2) break;
@@ -1159,8 +1158,8 @@ cudaError_t xsv_launch_score_raw(const LayerView& lv, int dtype, int H, int T_fi
     const int n = T_c - T_first;
     if (n <= 0) return cudaSuccess;
     const int grid = (n + 63) / 64;
-    if (dtype == 0) xsv_launch_dep(score_raw_kernel<__half>, dim3(grid), dim3(SCORE_TPB), 0, st, lv, H, T_first, T_c, qpart, qnorm, scores);
-    else xsv_launch_dep(score_raw_kernel<__nv_bfloat16>, dim3(grid), dim3(SCORE_TPB), 0, st, lv, H, T_first, T_c, qpart, qnorm, scores);
+    if (dtype == 0) xsv_launch_dep(score_raw_kernel<__half>, dim3(grid), dim3(SCORE_TPB), 0, st, lv, H, T_first, T_c, qpart, H * XSV_QCHUNKS, qnorm, scores);
+    else xsv_launch_dep(score_raw_kernel<__nv_bfloat16>, dim3(grid), dim3(SCORE_TPB), 0, st, lv, H, T_first, T_c, qpart, H * XSV_QCHUNKS, qnorm, scores);
     xsv_count_launch();
     return cudaGetLastError();
 }
