@@ -206,7 +206,7 @@ def oracle_config_times(max_seconds=60.0):
             else:
                 ref.step(q, k, v)
             dt_s = (time.perf_counter() - t0) * (Hc / heads)
-            entry[threads + "_threads_s"] = dt_s
+            entry[("all_threads_s" if threads == "all" else "one_thread_s")] = dt_s
             if threads == "one":
                 entry["one_thread_sample"] = f"{heads} of {Hc} heads, scaled by {Hc // heads}"
         out[name] = entry

@@ -14,11 +14,17 @@
 //   warps 0-3, 4-7 : softmax of query tile A / B, one query row per thread
 //                    (tensor-memory lane == row), online softmax in float32 with
 //                    lazy rescaling of the accumulator;
-//   warps 8-14     : producers: unpack the packed codes of a kv tile, dequantise
-//                    in registers (Eq. 12) and write fp16 tiles to shared memory
-//                    in the 128-byte-swizzled layout the MMA descriptors expect;
-//   warp 15        : one thread issues S = Q K^T (operands in shared memory) and
-//                    O += P V (P read from tensor memory, V from shared memory).
+//   warps 8-13     : producers: load the packed rows of a kv tile (16-byte loads, one
+//                    slab ahead), unpack the codes, dequantise in registers (Eq. 12)
+//                    and write fp16 tiles to shared memory in the 128-byte-swizzled
+//                    layout the MMA descriptors expect.  The operands do not exist in
+//                    HBM in that form, so the tiles cannot be copied in; feeding the
+//                    packed rows through a bulk-copy staging slot per warp
+//                    (cp.async.bulk + mbarrier) was built and measured 12-22 % slower
+//                    than the loads into registers, and is not used;
+//   warps 14, 15   : one thread each issues, for query tile A / B, S = Q K^T
+//                    (operands in shared memory) and O += P V (P read from tensor
+//                    memory, V from shared memory).
 // Stages are handed over with mbarriers; every wait is bounded and on expiry
 // sets XSV_DEV_TIMEOUT in the status word, after which all waits fall through
 // and the kernel runs to its end (tensor memory is always released).
