@@ -261,9 +261,13 @@ xsv_status xsv_quantization_mse(const void* x, int heads, long long n_tokens, xs
  *
  *   Arguments: as xsv_importance_scores.
  *   Limit    : heads <= 64; more returns XSV_ERR_LIMIT and launches nothing.
- *   Set-up   : the first call on each device looks up the array's device
- *              address (cudaGetSymbolAddress, with that device current).  Make
- *              that first call outside any stream capture.
+ *   Set-up   : the first call on each device (and for each input type) is
+ *              set-up: it looks up the array's device address
+ *              (cudaGetSymbolAddress, with that device current) and, where the
+ *              CUDA runtime loads modules lazily, makes it load the library's
+ *              device code, which may allocate and synchronise.  Make that
+ *              first call at start-up, outside any stream capture; from the
+ *              second call on nothing is allocated.
  *   Sharing  : every call on a device uses the same array.  Contents left by an
  *              earlier call are never read (each call rewrites all it uses), but
  *              two calls that overlap on the GPU -- different streams, no
