@@ -62,7 +62,12 @@ constexpr uint32_t OFF_KV = 2 * TILE_BYTES;                    // NSTAGE x (K ti
 constexpr uint32_t OFF_META = OFF_KV + NSTAGE * 2 * TILE_BYTES;   // key parameters as halves: [producer warp][scale | offset][64]
 constexpr uint32_t OFF_BAR = OFF_META + 3072;
 constexpr uint32_t BAR_BYTES = 512;
-constexpr uint32_t SMEM_BYTES = OFF_BAR + BAR_BYTES + 1024;    // + alignment slack
+constexpr uint32_t OFF_STAGE = OFF_BAR + BAR_BYTES;            // raw caches only: per producer warp one slab of 32 raw rows
+constexpr uint32_t STAGE_BYTES = 32 * 128;
+template <int BITS> constexpr uint32_t smem_bytes() {          // + alignment slack
+    return OFF_STAGE + (BITS == 16 ? NPROD * STAGE_BYTES : 0u) + 1024;
+}
+static_assert(smem_bytes<16>() <= 227 * 1024, "shared memory");
 
 // barrier slots (8 bytes each) inside the barrier block
 enum { B_KFULL = 0, B_VFULL = NSTAGE, B_EMPTY = 2 * NSTAGE, B_SFULL = 3 * NSTAGE, B_PREADY = B_SFULL + 2 * NBUF,
@@ -248,6 +253,12 @@ __device__ __forceinline__ uint32_t pack_h2(float a, float b) {
     asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));
     return r;
 }
+// 16-byte asynchronous copy global -> shared; src_bytes == 0 writes zeros and reads nothing
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t src_bytes) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ uint32_t hfma2_u(uint32_t a, uint32_t b, uint32_t c) {
     uint32_t d;
     asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
@@ -299,6 +310,26 @@ template <> __device__ __forceinline__ uint32_t beyond_h2<__nv_bfloat16>(uint32_
 // One row of 64 16-bit values (global) -> fp16, permuted, one swizzled 128-byte
 // row of a shared-memory tile.  grow == nullptr writes zeros.  Returns nonzero if a
 // value lay beyond the fp16 range (bf16 inputs only).
+// 16 channels (8 input words: block blk of a row) -> fp16, permuted, two 16-byte chunks of the tile's row.  Returns
+// nonzero if a value lay beyond the fp16 range (bf16 inputs only).
+template <typename T, int W>
+__device__ __forceinline__ uint32_t block16_to_tile(const uint32_t (&in)[8], uint8_t* tile, int row, int blk) {
+    uint32_t beyond = 0u;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) beyond |= beyond_h2<T>(in[i]);
+    uint32_t o[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        const int a = perm<W>(2 * q), b = perm<W>(2 * q + 1);   // local channels (W <= 16 keeps them in this block)
+        const uint32_t wa = in[a >> 1], wb = in[b >> 1];
+        const uint32_t lo = (a & 1) ? (wa >> 16) : (wa & 0xFFFFu);
+        const uint32_t hi = (b & 1) ? (wb & 0xFFFF0000u) : (wb << 16);
+        o[q] = to_h2<T>(lo | hi);
+    }
+    *reinterpret_cast<uint4*>(tile + swz(row, 2 * blk)) = make_uint4(o[0], o[1], o[2], o[3]);
+    *reinterpret_cast<uint4*>(tile + swz(row, 2 * blk + 1)) = make_uint4(o[4], o[5], o[6], o[7]);
+    return beyond;
+}
 template <typename T, int W>
 __device__ __forceinline__ uint32_t row16_to_tile(const T* grow, uint8_t* tile, int row) {
     uint32_t beyond = 0u;
@@ -312,19 +343,19 @@ __device__ __forceinline__ uint32_t row16_to_tile(const T* grow, uint8_t* tile, 
 #pragma unroll
             for (int i = 0; i < 8; ++i) in[i] = 0u;
         }
+        beyond |= block16_to_tile<T, W>(in, tile, row, blk);
+    }
+    return beyond;
+}
+// The same for a row already in registers (its eight 16-byte pieces in order)
+template <typename T, int W>
+__device__ __forceinline__ uint32_t row_regs_to_tile(const uint4 (&rw)[8], uint8_t* tile, int row) {
+    uint32_t beyond = 0u;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) beyond |= beyond_h2<T>(in[i]);
-        uint32_t o[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int a = perm<W>(2 * q), b = perm<W>(2 * q + 1);   // local channels (W <= 16 keeps them in this block)
-            const uint32_t wa = in[a >> 1], wb = in[b >> 1];
-            const uint32_t lo = (a & 1) ? (wa >> 16) : (wa & 0xFFFFu);
-            const uint32_t hi = (b & 1) ? (wb & 0xFFFF0000u) : (wb << 16);
-            o[q] = to_h2<T>(lo | hi);
-        }
-        *reinterpret_cast<uint4*>(tile + swz(row, 2 * blk)) = make_uint4(o[0], o[1], o[2], o[3]);
-        *reinterpret_cast<uint4*>(tile + swz(row, 2 * blk + 1)) = make_uint4(o[4], o[5], o[6], o[7]);
+    for (int blk = 0; blk < 4; ++blk) {
+        const uint32_t in[8] = {rw[2 * blk].x, rw[2 * blk].y, rw[2 * blk].z, rw[2 * blk].w,
+                                rw[2 * blk + 1].x, rw[2 * blk + 1].y, rw[2 * blk + 1].z, rw[2 * blk + 1].w};
+        beyond |= block16_to_tile<T, W>(in, tile, row, blk);
     }
     return beyond;
 }
@@ -533,6 +564,29 @@ __device__ __noinline__ void producer_loop(const Params& p, const Cta c) {
         }
     };
 
+    // A cache kept unquantised (BITS == 16): the slab's 32 raw rows (4 KB, contiguous in memory) are copied
+    // asynchronously into this warp's staging slot one slab ahead -- lane l moves bytes [512 k + 16 l, + 16), k < 8, so a
+    // copy instruction covers 512 consecutive bytes -- with the 16-byte piece p of row r at position p ^ (r & 7) of the
+    // row, so that the copies in (8 lanes per row) and the reads out (one row per lane) are free of bank conflicts.
+    // Rows past the end are filled with zeros (source size 0).
+    uint8_t* const slot = smem + OFF_STAGE + (uint32_t)pw * STAGE_BYTES;
+    auto stage = [&](const TileIter& ti, int sl) {
+        if (ti.valid) {
+            const bool cached = ti.kv < n_ct;
+            const int t0 = (cached ? ti.kv : ti.kv - n_ct) * BN + (sl & 3) * 32, lim = cached ? T_c : F;
+            const uint8_t* base = cached ? (sl < 4 ? lv.kcodes : lv.vcodes) + (size_t)ti.h * lv.cap * (XSV_D * 2)
+                                         : reinterpret_cast<const uint8_t*>(sl < 4 ? Kg : Vg) + (size_t)ti.h * F * (XSV_D * 2);
+            const uint32_t dst0 = smem_u32(slot);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int r = 4 * k + (lane >> 3), pc = lane & 7;
+                const bool ok = t0 + r < lim;
+                cp_async16(dst0 + swz(r, pc), base + (ok ? (size_t)(t0 + r) * (XSV_D * 2) + 16 * pc : 0), ok ? 16u : 0u);
+            }
+        }
+        cp_async_commit();
+    };
+
     uint32_t beyond = 0u;                           // a raw 16-bit input outside the fp16 range was seen
     TileIter cur{c.u_first, 0, 0, 0, false}, nxt;
     tile_iter_settle(p, b, u_last, cur);
@@ -546,7 +600,8 @@ __device__ __noinline__ void producer_loop(const Params& p, const Cta c) {
     };
     seek(cur, it, g >> 3);
     SlabRegs<NW> rc{}, rn{};
-    fetch(cur, (int)(g & 7u), rc);
+    if (BITS == 16) stage(cur, (int)(g & 7u));
+    else fetch(cur, (int)(g & 7u), rc);
     while (cur.valid) {
         const int sl = (int)(g & 7u);
         // the next slab of this warp: start its loads now
@@ -554,7 +609,18 @@ __device__ __noinline__ void producer_loop(const Params& p, const Cta c) {
         nxt = cur;
         uint32_t itn = it;
         seek(nxt, itn, gn >> 3);
-        fetch(nxt, (int)(gn & 7u), rn);
+        uint4 rw[8];
+        if (BITS == 16) {
+            // this slab's row out of the staging slot, then the slot is free for the next slab's copies
+            cp_async_wait_all();
+            __syncwarp();
+#pragma unroll
+            for (int pc = 0; pc < 8; ++pc) rw[pc] = *reinterpret_cast<const uint4*>(slot + swz(lane, pc));
+            __syncwarp();
+            stage(nxt, (int)(gn & 7u));
+        } else {
+            fetch(nxt, (int)(gn & 7u), rn);
+        }
 
         const uint32_t st = it % NSTAGE;
         uint8_t* tile = smem + OFF_KV + st * 2 * TILE_BYTES + (sl < 4 ? 0u : TILE_BYTES);
@@ -601,8 +667,10 @@ __device__ __noinline__ void producer_loop(const Params& p, const Cta c) {
 #pragma unroll
                 for (int ck = 0; ck < 8; ++ck) *reinterpret_cast<uint4*>(tile + swz(row, ck)) = make_uint4(0u, 0u, 0u, 0u);
             }
+        } else if (BITS == 16) {
+            beyond |= row_regs_to_tile<T, W>(rw, tile, row);     // rows past the end were staged as zeros
         } else {
-            // raw 16-bit rows: the fresh frame, or a cache kept unquantised (bits == 16)
+            // raw 16-bit rows of the fresh frame
             const T* src = nullptr;
             if (cached) {
                 const int tok = cur.kv * BN + row;
@@ -1100,11 +1168,11 @@ cudaError_t launch(const BatchParams& bp, bool merge_only, cudaStream_t st) {
     static XsvPerDeviceInt attr_set;      // the opt-in to large dynamic shared memory holds per device
     const int dev = xsv_current_device();
     if (!attr_set.get(dev)) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc5_kernel<T, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+        cudaError_t e = cudaFuncSetAttribute(attn_tc5_kernel<T, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes<BITS>());
         if (e != cudaSuccess) return e;
         attr_set.set(dev, 1);
     }
-    xsv_launch_dep(attn_tc5_kernel<T, BITS>, dim3(bp.cta_base[bp.n]), dim3(NTHREADS), SMEM_BYTES, st, bp);
+    xsv_launch_dep(attn_tc5_kernel<T, BITS>, dim3(bp.cta_base[bp.n]), dim3(NTHREADS), smem_bytes<BITS>(), st, bp);
     xsv_count_launch(1);
     return cudaGetLastError();
 }
