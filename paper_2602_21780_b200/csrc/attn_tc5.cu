@@ -21,7 +21,9 @@
 //                    HBM in that form, so the tiles cannot be copied in; feeding the
 //                    packed rows through a bulk-copy staging slot per warp
 //                    (cp.async.bulk + mbarrier) was built and measured 12-22 % slower
-//                    than the loads into registers, and is not used;
+//                    than the loads into registers, and is not used.  Only a cache kept
+//                    unquantised, whose rows are too wide to prefetch into registers, stages
+//                    its raw slabs in shared memory (16-byte asynchronous copies);
 //   warps 14, 15   : one thread each issues, for query tile A / B, S = Q K^T
 //                    (operands in shared memory) and O += P V (P read from tensor
 //                    memory, V from shared memory).
