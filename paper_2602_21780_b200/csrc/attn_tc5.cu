@@ -47,7 +47,7 @@ constexpr int BM = 128;            // query rows per tile
 constexpr int BN = 128;            // keys per kv tile
 constexpr int SUB = 64;            // keys per S sub-tile: a kv tile is consumed as two halves
 constexpr int NBUF = 3;            // S sub-tile buffers per query tile in tensor memory
-constexpr int NSTAGE = 5;          // kv stages in shared memory
+constexpr int NSTAGE = 4;          // kv stages in shared memory
 constexpr int NPROD = 6;              // producer warps
 constexpr int NTHREADS = (8 + NPROD + 2) * 32;   // 8 softmax warps, the producers, one MMA issuer per query tile
 constexpr uint32_t TILE_BYTES = 128u * 128u;   // 128 rows x 64 fp16
