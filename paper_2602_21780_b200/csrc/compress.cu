@@ -146,14 +146,9 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
             }
         }
         if (hb == 0) {
-            xsv_dep_sync();
-            qtilde_sum(qpart, n_part, qnorm, q_red, q_t);
-            // weights and bias: one warp per head at a time, lane l takes channels l and l + 32 (same position in
-            // their sub-words)
-            const float q0 = q_t[lane], q1 = q_t[lane + 32];
-            const float pos = __int_as_float((127 - BITS * ((lane & 7) % SUB)) << 23);
-            for (int h0 = warp; h0 < H; h0 += 2 * (SCORE_TPB / 32)) {     // two heads per pass: eight loads in flight
-                float sc[2][2], zz[2][2];
+            // the group's parameters of the first two heads of this warp: loaded, like the rows, before the wait
+            float sc[2][2], zz[2][2];
+            auto load_params = [&](int h0) {
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     const int h = h0 + t * (SCORE_TPB / 32);
@@ -161,6 +156,16 @@ __global__ void __launch_bounds__(SCORE_TPB) score_kernel(LayerView lv, int H, i
                     sc[t][0] = lv.kscale[m + lane]; sc[t][1] = lv.kscale[m + lane + 32];
                     zz[t][0] = lv.kzero[m + lane]; zz[t][1] = lv.kzero[m + lane + 32];
                 }
+            };
+            load_params(warp);
+            xsv_dep_sync();
+            qtilde_sum(qpart, n_part, qnorm, q_red, q_t);
+            // weights and bias: one warp per head at a time, lane l takes channels l and l + 32 (same position in
+            // their sub-words)
+            const float q0 = q_t[lane], q1 = q_t[lane + 32];
+            const float pos = __int_as_float((127 - BITS * ((lane & 7) % SUB)) << 23);
+            for (int h0 = warp; h0 < H; h0 += 2 * (SCORE_TPB / 32)) {     // two heads per pass: eight loads in flight
+                if (h0 != warp) load_params(h0);
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
                     const int h = h0 + t * (SCORE_TPB / 32);
