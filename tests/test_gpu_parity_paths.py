@@ -62,6 +62,15 @@ def test_paper_shape_two_and_eight_bits(bits):
     assert w["pruned_steps"] == 1
 
 
+@pytest.mark.parametrize("dtype,L_max", [("bf16", 2 * F_PAPER + 700), ("fp16", 0)])
+def test_paper_shape_unquantised_cache(dtype, L_max):
+    # bits = 16: raw rows staged through shared memory by the attention kernel's producers; paper-sized frames (a ragged
+    # last tile of 94 rows in the frame, ragged cache ends after pruning), pruning on (bf16) and off (fp16)
+    st = synth.Stream(H=4, d=64, F=F_PAPER, dtype=dtype, layer=41)
+    w = run_stream(st, 4, L_max, 16, max_cache_tokens=-1 if L_max else 4 * F_PAPER)
+    assert w["checked"] == 4 and w["pruned_steps"] == (2 if L_max else 0)
+
+
 @pytest.mark.parametrize("bits", [2, 4])
 def test_frames_of_alternating_size(bits):
     # frame sizes differ from step to step (inputs resized to a maximum edge have varying token counts):
