@@ -145,9 +145,12 @@ xsv_status xsv_step(xsv_cache* c, int layer, const void* Q, const void* K, const
  * two frames).  caches[i] is stepped on layer `layer` with the frame
  * Q[i], K[i], V[i] of n_tokens[i] tokens and writes out[i]; each call argument
  * is a HOST array of n entries (device pointers for Q, K, V, out), n at most
- * XSV_MAX_BATCH.  The attention of all n streams is ONE kernel launch (plus one
- * merge launch) whose CTAs are dealt to the streams in proportion to their
- * work; scores, selection and quantisation run per stream, the selection and
+ * XSV_MAX_BATCH.  The attention of the n streams is one kernel launch (plus one
+ * merge launch) per group of streams, a launch's CTAs dealt to its streams in
+ * proportion to their work; the library picks the grouping (all n, or
+ * consecutive groups of 4, 2 or 1) that its cost model estimates fastest, since
+ * CTAs do not span streams and 148 of them fit e.g. eight long streams badly.
+ * Scores, selection and quantisation run per stream, the selection and
  * quantisation on each cache's own streams side by side.  Results and cache
  * states are those of n xsv_step calls.  The caches must be distinct, on one
  * device, with equal heads and bit width (XSV_ERR_SHAPE otherwise) and use the

@@ -37,6 +37,7 @@
 // The channel order inside shared memory is permuted (the order in which the
 // codes fall out of a packed 32-bit word); Q and fresh K rows are permuted the
 // same way, and the output columns are un-permuted in the epilogue.
+#include <algorithm>
 #include <type_traits>
 
 #include "xsv_kernels.h"
@@ -1276,14 +1277,43 @@ cudaError_t xsv_launch_attn_tc5_batch(int n, const LayerView* lvs, const int* T_
                                       const void* const* Ks, const void* const* Vs, void* const* outs, int dtype, int H,
                                       const int* Fs, float* workspace, int* const* statuses, cudaStream_t st) {
     if (!workspace || n < 1 || n > XSV_MAX_BATCH) return cudaErrorInvalidValue;
-    BatchParams bp{};
-    bp.n = n;
+    Params ps[XSV_MAX_BATCH];
     for (int i = 0; i < n; ++i) {
         if (lvs[i].bits != lvs[0].bits) return cudaErrorInvalidValue;
-        fill_params(bp.p[i], lvs[i], T_cs[i], Qs[i], Ks[i], Vs[i], outs[i], H, Fs[i], statuses[i]);
+        fill_params(ps[i], lvs[i], T_cs[i], Qs[i], Ks[i], Vs[i], outs[i], H, Fs[i], statuses[i]);
     }
-    deal_ctas(bp, workspace, xsv_sm_count());
-    cudaError_t e = launch_tc5(bp, dtype, lvs[0].bits, false, st);
-    if (e != cudaSuccess) return e;
-    return launch_tc5(bp, dtype, lvs[0].bits, true, st);
+    // CTAs do not span streams, so a launch takes as long as its slowest stream: max over the streams of ticks per
+    // CTA.  With many streams the whole numbers of CTAs fit the work badly (eight equal streams get 18 or 19 of 148
+    // CTAs each); the streams are therefore launched in consecutive groups of g, with the g among n, 4, 2, 1 whose
+    // estimated time -- the groups' slowest streams, plus a fixed cost per launch -- is the smallest.
+    const int sms = xsv_sm_count();
+    constexpr long long LAUNCH_TICKS = 100;         // ramp and tail of a launch, in the ticks of the cost model
+    auto build = [&](int first, int count, BatchParams& bp) {
+        bp = BatchParams{};
+        bp.n = count;
+        for (int i = 0; i < count; ++i) bp.p[i] = ps[first + i];
+        deal_ctas(bp, workspace, sms);
+        long long worst = 0;
+        for (int i = 0; i < count; ++i) worst = std::max(worst, (bp.p[i].total + bp.p[i].G - 1) / bp.p[i].G);
+        return worst + LAUNCH_TICKS;
+    };
+    int best_g = n;
+    long long best = -1;
+    const int cand[4] = {n, 4, 2, 1};
+    BatchParams bp;
+    for (int c = 0; c < 4; ++c) {
+        const int g = cand[c];
+        if (g > n || (c > 0 && g >= cand[0])) continue;
+        long long t = 0;
+        for (int first = 0; first < n; first += g) t += build(first, std::min(g, n - first), bp);
+        if (best < 0 || t < best) { best = t; best_g = g; }
+    }
+    for (int first = 0; first < n; first += best_g) {
+        build(first, std::min(best_g, n - first), bp);
+        cudaError_t e = launch_tc5(bp, dtype, lvs[0].bits, false, st);
+        if (e != cudaSuccess) return e;
+        e = launch_tc5(bp, dtype, lvs[0].bits, true, st);     // the merge reads the workspace the next group reuses
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }

@@ -229,6 +229,14 @@ def test_two_streams_at_paper_shape_and_two_bits():
     assert w["pruned_steps"] >= 3
 
 
+def test_eight_long_streams_are_launched_in_groups():
+    # eight streams whose caches are long enough that the library splits the call into two attention launches of four
+    # streams each (148 CTAs do not divide evenly by eight); the last step is compared with each stream's oracle
+    streams = [synth.Stream(H=4, d=64, F=F_PAPER, dtype="bf16", layer=80 + i) for i in range(8)]
+    w = run_batch(streams, 18, 16 * F_PAPER, 4, check_steps={17}, deferred_join=True)
+    assert w["checked"] == 8 and w["pruned_steps"] == 8
+
+
 def test_batch_rejects_mismatched_caches_before_launching():
     a, b = binding.Cache(1, 4, 64, 500, 4), binding.Cache(1, 4, 64, 500, 2)
     Q = torch.zeros(4, 100, 64, device="cuda", dtype=torch.float16)
