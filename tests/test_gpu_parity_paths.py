@@ -62,6 +62,14 @@ def test_paper_shape_two_and_eight_bits(bits):
     assert w["pruned_steps"] == 1
 
 
+def test_paper_shape_fp16_inputs():
+    # float16 inputs at the paper's frame size (the other paper-shape cases feed bfloat16): no conversion on the way
+    # into the attention kernel, float16 rounding of the frame's rows in the quantiser's input
+    st = synth.Stream(H=4, d=64, F=F_PAPER, dtype="fp16", layer=40)
+    w = run_stream(st, 5, 3 * F_PAPER, 4)
+    assert w["checked"] == 5 and w["pruned_steps"] == 2
+
+
 @pytest.mark.parametrize("dtype,L_max", [("bf16", 2 * F_PAPER + 700), ("fp16", 0)])
 def test_paper_shape_unquantised_cache(dtype, L_max):
     # bits = 16: raw rows staged through shared memory by the attention kernel's producers; paper-sized frames (a ragged
