@@ -393,6 +393,20 @@ xsv_status xsv_selftest_bounded_wait(void* stream);
  */
 int xsv_selftest_device_table(void);
 
+/*
+ * How xsv_step_batch would group n streams into attention launches: the number
+ * of consecutive streams per launch (n, 4, 2 or 1) that the library's cost
+ * model estimates fastest for streams with cache_tokens[i] cached tokens and
+ * frames of frame_tokens[i] tokens (HOST arrays of n entries), `heads` heads,
+ * on a device with `multiprocessors` multiprocessors.  CTAs do not span
+ * streams, so e.g. eight long streams on 148 multiprocessors go out as two
+ * launches of four (37 CTAs each) rather than one of eight (18 or 19 each).
+ * Host arithmetic only: needs no GPU and touches no cache.  Returns -1 for bad
+ * arguments (n outside 1..XSV_MAX_BATCH, a null array, a negative length).
+ * (The paper has no counterpart.)
+ */
+int xsv_plan_batch_groups(int n, const int* cache_tokens, const int* frame_tokens, int heads, int multiprocessors);
+
 /* Kernels launched by this library in the calling process since load (the paper has no counterpart). */
 long long xsv_kernel_launches(void);
 

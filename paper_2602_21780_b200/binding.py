@@ -48,6 +48,7 @@ SYMBOLS = {
     "xsv_cache_profile_read": (_i, [_vp, C.POINTER(C.c_double), C.POINTER(_ll), _i]),
     "xsv_selftest_bounded_wait": (_i, [_vp]),
     "xsv_selftest_device_table": (_i, []),
+    "xsv_plan_batch_groups": (_i, [_i, C.POINTER(_i), C.POINTER(_i), _i, _i]),
     "xsv_kernel_launches": (_ll, []),
     "xsv_strerror": (C.c_char_p, [_i]),
     "xsv_last_cuda_error": (C.c_char_p, []),
@@ -69,6 +70,15 @@ def load():
             fn.restype, fn.argtypes = res, args
         _lib = lib
     return _lib
+
+
+def plan_batch_groups(cache_tokens, frame_tokens, heads, multiprocessors=148):
+    """Streams per attention launch that step_batch would use for streams of these cache and frame lengths
+    (host arithmetic inside the library; needs no GPU)."""
+    n = len(cache_tokens)
+    a = (C.c_int * n)(*[int(x) for x in cache_tokens])
+    f = (C.c_int * n)(*[int(x) for x in frame_tokens])
+    return int(load().xsv_plan_batch_groups(n, a, f, int(heads), int(multiprocessors)))
 
 
 def step_batch(caches, layer, Qs, Ks, Vs, outs, stream=None):

@@ -1220,7 +1220,7 @@ void deal_ctas(BatchParams& bp, float* workspace, int sms) {
         if (g > MAX_PARTS) g = MAX_PARTS;
         if (g < 1) g = 1;
         p.G = (int)g;
-        p.part = workspace + (size_t)used * 2 * PART_STRIDE;
+        p.part = workspace ? workspace + (size_t)used * 2 * PART_STRIDE : nullptr;   // no workspace: a planning call
         bp.cta_base[i] = used;
         used += p.G;
     }
@@ -1273,6 +1273,45 @@ cudaError_t xsv_launch_attn_tc5_merge(const LayerView& lv, int T_c, const void* 
     return launch_one(lv, T_c, Q, K, V, out, dtype, H, F, workspace, status, spare_sms, true, st);
 }
 
+namespace {
+// CTAs do not span streams, so a launch takes as long as its slowest stream: max over the streams of ticks per CTA.
+// With many streams the whole numbers of CTAs fit the work badly (eight equal streams get 18 or 19 of 148 CTAs
+// each); the streams are therefore launched in consecutive groups of g, with the g among n, 4, 2, 1 whose estimated
+// time -- the groups' slowest streams, plus a fixed cost per launch -- is the smallest.  Host arithmetic only.
+constexpr long long LAUNCH_TICKS = 100;             // ramp and tail of a launch, in the ticks of the cost model
+long long build_group(const Params* ps, int first, int count, float* workspace, int sms, BatchParams& bp) {
+    bp = BatchParams{};
+    bp.n = count;
+    for (int i = 0; i < count; ++i) bp.p[i] = ps[first + i];
+    deal_ctas(bp, workspace, sms);
+    long long worst = 0;
+    for (int i = 0; i < count; ++i) worst = std::max(worst, (bp.p[i].total + bp.p[i].G - 1) / bp.p[i].G);
+    return worst + LAUNCH_TICKS;
+}
+int choose_group_size(const Params* ps, int n, int sms) {
+    int best_g = n;
+    long long best = -1;
+    const int cand[4] = {n, 4, 2, 1};
+    BatchParams bp;
+    for (int c = 0; c < 4; ++c) {
+        const int g = cand[c];
+        if (g > n || (c > 0 && g >= cand[0])) continue;
+        long long t = 0;
+        for (int first = 0; first < n; first += g) t += build_group(ps, first, std::min(g, n - first), nullptr, sms, bp);
+        if (best < 0 || t < best) { best = t; best_g = g; }
+    }
+    return best_g;
+}
+}  // namespace
+
+int xsv_attn_batch_group_size(int n, const int* T_cs, const int* Fs, int H, int sms) {
+    if (n < 1 || n > XSV_MAX_BATCH || sms < 1) return -1;
+    Params ps[XSV_MAX_BATCH];
+    const LayerView none{};
+    for (int i = 0; i < n; ++i) fill_params(ps[i], none, T_cs[i], nullptr, nullptr, nullptr, nullptr, H, Fs[i], nullptr);
+    return choose_group_size(ps, n, sms);
+}
+
 cudaError_t xsv_launch_attn_tc5_batch(int n, const LayerView* lvs, const int* T_cs, const void* const* Qs,
                                       const void* const* Ks, const void* const* Vs, void* const* outs, int dtype, int H,
                                       const int* Fs, float* workspace, int* const* statuses, cudaStream_t st) {
@@ -1282,34 +1321,11 @@ cudaError_t xsv_launch_attn_tc5_batch(int n, const LayerView* lvs, const int* T_
         if (lvs[i].bits != lvs[0].bits) return cudaErrorInvalidValue;
         fill_params(ps[i], lvs[i], T_cs[i], Qs[i], Ks[i], Vs[i], outs[i], H, Fs[i], statuses[i]);
     }
-    // CTAs do not span streams, so a launch takes as long as its slowest stream: max over the streams of ticks per
-    // CTA.  With many streams the whole numbers of CTAs fit the work badly (eight equal streams get 18 or 19 of 148
-    // CTAs each); the streams are therefore launched in consecutive groups of g, with the g among n, 4, 2, 1 whose
-    // estimated time -- the groups' slowest streams, plus a fixed cost per launch -- is the smallest.
     const int sms = xsv_sm_count();
-    constexpr long long LAUNCH_TICKS = 100;         // ramp and tail of a launch, in the ticks of the cost model
-    auto build = [&](int first, int count, BatchParams& bp) {
-        bp = BatchParams{};
-        bp.n = count;
-        for (int i = 0; i < count; ++i) bp.p[i] = ps[first + i];
-        deal_ctas(bp, workspace, sms);
-        long long worst = 0;
-        for (int i = 0; i < count; ++i) worst = std::max(worst, (bp.p[i].total + bp.p[i].G - 1) / bp.p[i].G);
-        return worst + LAUNCH_TICKS;
-    };
-    int best_g = n;
-    long long best = -1;
-    const int cand[4] = {n, 4, 2, 1};
+    const int g = choose_group_size(ps, n, sms);
     BatchParams bp;
-    for (int c = 0; c < 4; ++c) {
-        const int g = cand[c];
-        if (g > n || (c > 0 && g >= cand[0])) continue;
-        long long t = 0;
-        for (int first = 0; first < n; first += g) t += build(first, std::min(g, n - first), bp);
-        if (best < 0 || t < best) { best = t; best_g = g; }
-    }
-    for (int first = 0; first < n; first += best_g) {
-        build(first, std::min(best_g, n - first), bp);
+    for (int first = 0; first < n; first += g) {
+        build_group(ps, first, std::min(g, n - first), workspace, sms, bp);
         cudaError_t e = launch_tc5(bp, dtype, lvs[0].bits, false, st);
         if (e != cudaSuccess) return e;
         e = launch_tc5(bp, dtype, lvs[0].bits, true, st);     // the merge reads the workspace the next group reuses

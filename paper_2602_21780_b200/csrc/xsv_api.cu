@@ -750,6 +750,13 @@ xsv_status xsv_importance_scores(const void* Q, const void* keys, int heads, int
     return e == cudaSuccess ? XSV_OK : cuda_fail(e);
 }
 
+int xsv_plan_batch_groups(int n, const int* cache_tokens, const int* frame_tokens, int heads, int multiprocessors) {
+    if (!cache_tokens || !frame_tokens || heads < 1) return -1;
+    for (int i = 0; i < n && i < XSV_MAX_BATCH; ++i)
+        if (cache_tokens[i] < 0 || frame_tokens[i] < 1) return -1;
+    return xsv_attn_batch_group_size(n, cache_tokens, frame_tokens, heads, multiprocessors);
+}
+
 int xsv_selftest_device_table(void) {
     // host-only: the per-device slots are independent, survive other slots' updates, and ignore devices
     // beyond the table (which then are configured on every launch instead of once)

@@ -76,6 +76,9 @@ cudaError_t xsv_launch_attn_tc5_merge(const LayerView& lv, int T_c, const void* 
 cudaError_t xsv_launch_attn_tc5_batch(int n, const LayerView* lvs, const int* T_cs, const void* const* Qs,
                                       const void* const* Ks, const void* const* Vs, void* const* outs, int dtype, int H,
                                       const int* Fs, float* workspace, int* const* statuses, cudaStream_t st);
+// Streams per attention launch that xsv_launch_attn_tc5_batch would choose for these cache and frame lengths on a
+// device with `sms` multiprocessors (host arithmetic only); -1 for bad arguments.
+int xsv_attn_batch_group_size(int n, const int* T_cs, const int* Fs, int H, int sms);
 
 // One small kernel whose only wait can never be satisfied: it must come back after the
 // attention kernel's wait limit with XSV_DEV_TIMEOUT set in *status (device int).

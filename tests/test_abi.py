@@ -43,3 +43,19 @@ def test_per_device_table_keeps_devices_apart():
     # kernel attributes are per CUDA device; the table that remembers them must not let one device's
     # entry stand for another's (host-only self-test inside the library)
     assert binding.load().xsv_selftest_device_table() == 0
+
+
+def test_batched_streams_are_grouped_so_that_ctas_fit():
+    # CTAs do not span streams: eight long streams on 148 multiprocessors go out as two launches of four (37 CTAs
+    # each) rather than one of eight (18 or 19 each); four go out together; short streams stay in one launch, where
+    # a second launch would cost more than the uneven split; other counts fall back to the best of n, 4, 2, 1
+    F = 1374
+    assert binding.plan_batch_groups([21984] * 8, [F] * 8, 16) == 4
+    assert binding.plan_batch_groups([21984] * 4, [F] * 4, 16) == 4
+    assert binding.plan_batch_groups([21984] * 2, [F] * 2, 16) == 2
+    assert binding.plan_batch_groups([21984], [F], 16) == 1
+    assert binding.plan_batch_groups([600] * 8, [200] * 8, 4) == 8
+    assert binding.plan_batch_groups([21984] * 6, [F] * 6, 16) in (6, 4, 2)
+    assert binding.plan_batch_groups([21984] * 8, [F] * 8, 16, multiprocessors=160) == 8      # 20 CTAs each: even
+    assert binding.plan_batch_groups([], [], 16) == -1
+    assert binding.plan_batch_groups([-1], [F], 16) == -1
