@@ -55,7 +55,8 @@ def test_batched_streams_are_grouped_so_that_ctas_fit():
     assert binding.plan_batch_groups([21984] * 2, [F] * 2, 16) == 2
     assert binding.plan_batch_groups([21984], [F], 16) == 1
     assert binding.plan_batch_groups([600] * 8, [200] * 8, 4) == 8
-    assert binding.plan_batch_groups([21984] * 6, [F] * 6, 16) in (6, 4, 2)
+    assert binding.plan_batch_groups([21984] * 6, [F] * 6, 16) == 4                          # 37 x 4, then 74 x 2
+    assert binding.plan_batch_groups([21984] * 7, [F] * 7, 16) == 7                          # 21 each: 147 of 148
     assert binding.plan_batch_groups([21984] * 8, [F] * 8, 16, multiprocessors=160) == 8      # 20 CTAs each: even
     assert binding.plan_batch_groups([], [], 16) == -1
     assert binding.plan_batch_groups([-1], [F], 16) == -1
