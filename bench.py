@@ -33,6 +33,7 @@ if ROOT not in sys.path:
 
 H, D, F, LAYERS, L_MAX, BITS = 16, 64, 1374, 24, 21984, 4
 PREFILL = 16                 # frames that fill the cache to the budget (untimed set-up)
+TORCH_DTYPE = "bfloat16"     # input type of the generated frames; "float16" only in sweep cases (--dtype fp16)
 POOL = 4                     # distinct frames per layer, cycled
 METRIC = "frames/s of compressed-KV causal attention step (24 layers)"
 WORKLOAD = ("config2: 24 layers x (16 heads x 64), 1374 tokens/frame, budget 21984 tokens/layer, 4-bit KV, bf16, "
@@ -125,9 +126,10 @@ def gen_frames(torch, dev, layers, pool, seed):
             m[h, 0, idx] = 10.0
         per = []
         for p in range(pool):
-            q = torch.randn(H, F, D, device=dev, generator=g).to(torch.bfloat16)
-            k = ((torch.randn(H, F, D, device=dev, generator=g) + mu) * m).to(torch.bfloat16)
-            v = torch.randn(H, F, D, device=dev, generator=g).to(torch.bfloat16)
+            dt = getattr(torch, TORCH_DTYPE)
+            q = torch.randn(H, F, D, device=dev, generator=g).to(dt)
+            k = ((torch.randn(H, F, D, device=dev, generator=g) + mu) * m).to(dt)
+            v = torch.randn(H, F, D, device=dev, generator=g).to(dt)
             per.append((q.contiguous(), k.contiguous(), v.contiguous()))
         frames.append(per)
     return frames
@@ -484,7 +486,7 @@ def run_batch_bench(args, torch, binding, dev, stream):
 
 
 def main():
-    global LAYERS, WORKLOAD, L_MAX, BITS, PREFILL
+    global LAYERS, WORKLOAD, L_MAX, BITS, PREFILL, TORCH_DTYPE
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=40)
@@ -499,6 +501,8 @@ def main():
                     help="cache budget in frames (default 16 = the benchmark; other values: the cache-length sweep)")
     ap.add_argument("--bits", type=int, default=BITS, choices=[2, 4, 8, 16],
                     help="bits per cached element (default 4 = the benchmark; 16 = quantisation off, pruning only)")
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16"],
+                    help="input type (default bf16 = the benchmark; fp16: a sweep case, e.g. with --bits 16 the copy-engine feed)")
     ap.add_argument("--config", type=int, default=2, choices=[2, 3, 4],
                     help="2: the benchmark (default); 3: the long-horizon run; 4: the one-layer sweep and the uncompressed cache")
     ap.add_argument("--frames", type=int, default=0, help="--config 3: frames to stream (default 1000)")
@@ -515,13 +519,15 @@ def main():
     if args.layers != LAYERS:
         WORKLOAD = WORKLOAD.replace("24 layers", f"{args.layers} layers (profiling case, not the benchmark)")
         LAYERS = args.layers
-    sweep = args.budget_frames * F != L_MAX or args.bits != BITS
+    sweep = args.budget_frames * F != L_MAX or args.bits != BITS or args.dtype != "bf16"
+    if args.dtype == "fp16":
+        TORCH_DTYPE = "float16"
     if sweep:
         if args.budget_frames < 3:
             ap.error("--budget-frames must be at least 3")
         WORKLOAD = (WORKLOAD.replace("config2:", "sweep case (not the benchmark), config2 with")
                     .replace(f"budget {L_MAX} tokens/layer", f"budget {args.budget_frames * F} tokens/layer")
-                    .replace(f"{BITS}-bit KV", f"{args.bits}-bit KV")
+                    .replace(f"{BITS}-bit KV", f"{args.bits}-bit KV").replace("-bit KV, bf16,", f"-bit KV, {args.dtype},")
                     .replace(f"{PREFILL}-frame prefill", f"{args.budget_frames}-frame prefill"))
         L_MAX, BITS, PREFILL = args.budget_frames * F, args.bits, args.budget_frames
         args.no_cpu_baseline = True
@@ -545,7 +551,8 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     frames = gen_frames(torch, dev, LAYERS, POOL, seed=replica_seed(20260221, rank))
-    out = torch.empty(H, F, D, device=dev, dtype=torch.bfloat16)
+    out = torch.empty(H, F, D, device=dev, dtype=getattr(torch, TORCH_DTYPE))
+    xsv_dtype = binding.BF16 if TORCH_DTYPE == "bfloat16" else binding.F16
     stream = torch.cuda.current_stream()
     sp = stream.cuda_stream
     impl = {"auto": binding.ATTN_AUTO, "mma": binding.ATTN_MMA, "tc5": binding.ATTN_TC5}[args.attn]
@@ -564,7 +571,7 @@ def main():
     def frame_step(cache, f):
         for l in range(LAYERS):
             q, k, v = ptrs[l][f % POOL]
-            rc = cache.step_raw(l, q, k, v, F, binding.BF16, optr, sp)
+            rc = cache.step_raw(l, q, k, v, F, xsv_dtype, optr, sp)
             if rc != 0:
                 raise RuntimeError(f"xsv_step failed: status {rc}")
 
@@ -669,7 +676,7 @@ def main():
     e2e = None
     if not args.no_e2e:
         hq = [[tuple(t.cpu().pin_memory() for t in fr) for fr in per[:2]] for per in frames]
-        houts = [torch.empty(H, F, D, dtype=torch.bfloat16).pin_memory() for _ in range(LAYERS)]
+        houts = [torch.empty(H, F, D, dtype=getattr(torch, TORCH_DTYPE)).pin_memory() for _ in range(LAYERS)]
         c2 = make_cache()
         c2.set_host_pipelining(True)          # results travel back while the next layer computes
         for f in range(PREFILL + 3):
@@ -713,7 +720,7 @@ def main():
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": "frames/s", "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                "vs_baseline": None, "dtype": "bf16" if TORCH_DTYPE == "bfloat16" else "fp16", "data": "synthetic",
                 "config": {"workload": WORKLOAD, "prefill_frames": PREFILL, "attn_impl": args.attn, "deferred_join": True,
                            "l2": "each step touches 203 MB of fresh inputs + 675 MB of cache (> 126 MB L2); no flush",
                            "multi_gpu": "replicas only"},

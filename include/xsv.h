@@ -30,7 +30,12 @@
  *    without rounding for magnitudes in [2^-14, 65504], smaller ones are
  *    held with an absolute error of at most 2^-25, and a bf16 magnitude of
  *    2^16 or more saturates and sets XSV_ERR_RANGE in the status word (the
- *    default attention kernel reports it; see xsv_cache_status).
+ *    default attention kernel reports it; see xsv_cache_status).  One case
+ *    differs: a cache kept unquantised (bits = 16) is attended in the inputs'
+ *    own type where the copy engine can fetch its tiles (pointers aligned as
+ *    required above) -- fp16 as above; bf16 inputs then stay bf16, with no
+ *    range limit and the probabilities rounded to bf16 (8-bit significand)
+ *    before they multiply V.
  *  - xsv_step only enqueues work on `stream`; it does not synchronise and,
  *    after the call that allocates, creates nothing: all device memory, the
  *    cache's own streams and its events come from xsv_cache_set_options with

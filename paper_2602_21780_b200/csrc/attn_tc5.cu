@@ -21,9 +21,13 @@
 //                    HBM in that form, so the tiles cannot be copied in; feeding the
 //                    packed rows through a bulk-copy staging slot per warp
 //                    (cp.async.bulk + mbarrier) was built and measured 12-22 % slower
-//                    than the loads into registers, and is not used.  Only a cache kept
-//                    unquantised, whose rows are too wide to prefetch into registers, stages
-//                    its raw slabs in shared memory (16-byte asynchronous copies);
+//                    than the loads into registers, and is not used.  A cache kept unquantised
+//                    does hold its operands in MMA form: its K and V tiles, and the frame's,
+//                    are fetched by tensor-map bulk copies issued by one producer lane
+//                    (cp.async.bulk.tensor, 128-byte swizzle, no multicast), fp16 or -- with
+//                    bf16 operands in the MMAs -- bf16; where no tensor map can be made (an
+//                    unaligned pointer) its producers stage raw slabs in shared memory by
+//                    16-byte asynchronous copies and convert bf16 to fp16;
 //   warps 14, 15   : one thread each issues, for query tile A / B, S = Q K^T
 //                    (operands in shared memory) and O += P V (P read from tensor
 //                    memory, V from shared memory).
@@ -37,7 +41,10 @@
 // The channel order inside shared memory is permuted (the order in which the
 // codes fall out of a packed 32-bit word); Q and fresh K rows are permuted the
 // same way, and the output columns are un-permuted in the epilogue.
+#include <cuda.h>
+
 #include <algorithm>
+#include <cstdlib>
 #include <type_traits>
 
 #include "xsv_kernels.h"
@@ -103,11 +110,17 @@ constexpr int PART_STRIDE = 256 * 66;   // floats per (CTA, slot)
 // Several independent streams (caches) in one launch: stream s owns the CTAs [cta_base[s], cta_base[s + 1]) and the
 // units [unit_base[s], unit_base[s + 1]) of the merge grid; each stream's Params carries its own CTA count G, its
 // slice of the workspace and its own status word, so inside a CTA everything is as for a launch of that stream alone.
+// Tensor maps of one stream for the copy-engine feed of an unquantised fp16 cache: cached keys, cached values, the
+// frame's keys, the frame's values, each a [heads][rows][64] tensor read in boxes of 128 rows.
+struct alignas(64) StreamMaps { CUtensorMap m[4]; };
+
 struct BatchParams {
     int n;
+    int use_tma;         // every stream's K / V tiles are fetched by tensor-map bulk copies (bits == 16)
     int cta_base[XSV_MAX_BATCH + 1];
     int unit_base[XSV_MAX_BATCH + 1];
     Params p[XSV_MAX_BATCH];
+    StreamMaps tm[XSV_MAX_BATCH];
 };
 
 // ------------------------------------------------------------------ work split
@@ -197,6 +210,16 @@ __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sy
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// One arrival that also announces `bytes` of asynchronous copies to come
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// Box (x, y, z) of a rank-3 tensor map -> shared memory; the bytes complete on the mbarrier.  No multicast.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z) {
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                 ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
+                 : "memory");
+}
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
     asm volatile(
@@ -262,6 +285,15 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+// two probabilities -> the packed pair the P V MMA reads: fp16, or bf16 when the operands are bf16 (BF)
+template <bool BF> __device__ __forceinline__ uint32_t pack_p(float a, float b) {
+    if (BF) {
+        uint32_t r;
+        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));
+        return r;
+    }
+    return pack_h2(a, b);
+}
 __device__ __forceinline__ uint32_t hfma2_u(uint32_t a, uint32_t b, uint32_t c) {
     uint32_t d;
     asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
@@ -425,6 +457,7 @@ __device__ __forceinline__ unsigned long long f2_add(unsigned long long a, unsig
 
 // 32 logits of one row -> 32 probabilities 2^(s * sc - m) packed as fp16 pairs; their sum is added to the two
 // lanes of ls2.  Whole sub-tiles only.  The scaling and the sum run as packed float32 pairs (half the issue slots).
+template <bool BF>
 __device__ __forceinline__ void softmax32_fast(const uint32_t (&v)[32], unsigned long long sc2, unsigned long long nm2,
                                                unsigned long long& ls2, uint32_t (&pk)[16]) {
 #pragma unroll
@@ -433,11 +466,11 @@ __device__ __forceinline__ void softmax32_fast(const uint32_t (&v)[32], unsigned
         f2_unpack(f2_fma(f2_pack(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), sc2, nm2), x0, x1);
         const float p0 = ex2(x0), p1 = ex2(x1);
         ls2 = f2_add(ls2, f2_pack(p0, p1));
-        pk[i >> 1] = pack_h2(p0, p1);
+        pk[i >> 1] = pack_p<BF>(p0, p1);
     }
 }
 // The same with a mask: columns at or beyond `valid` (a ragged last tile) give probability 0.
-template <bool MASK>
+template <bool MASK, bool BF>
 __device__ __forceinline__ void softmax32(const uint32_t (&v)[32], float sc, float nm, int valid, float& ls, uint32_t (&pk)[16]) {
 #pragma unroll
     for (int i = 0; i < 32; i += 2) {
@@ -447,7 +480,7 @@ __device__ __forceinline__ void softmax32(const uint32_t (&v)[32], float sc, flo
             if (i + 1 >= valid) p1 = 0.f;
         }
         ls += p0 + p1;
-        pk[i >> 1] = pack_h2(p0, p1);
+        pk[i >> 1] = pack_p<BF>(p0, p1);
     }
 }
 // running maximum of 32 raw logits (the first `valid` of them)
@@ -696,8 +729,42 @@ __device__ __noinline__ void producer_loop(const Params& p, const Cta c) {
     if (beyond) atomicOr(status, XSV_DEV_RANGE);
 }
 
-// Softmax warpgroups (warps 0-3: query tile A, warps 4-7: tile B) and the epilogue.
-template <typename T, int BITS>
+// Copy-engine feed for a cache kept unquantised with fp16 inputs: the operands exist in HBM in the form the MMA reads
+// (rows of 64 fp16, no conversion, identity channel order), so one lane asks the copy engine for whole K and V tiles
+// -- boxes of 128 rows x 128 bytes of a [heads][rows][64] tensor map, written in the 128-byte-swizzled layout of the MMA
+// descriptors; rows past the end of the cache or of the frame arrive as zeros -- and the other producer lanes have
+// nothing to do.  The byte counts complete the stage's KFULL / VFULL barriers (one announcing arrival each).
+__device__ __noinline__ void producer_tma_loop(const Params& p, const Cta c, const StreamMaps& maps) {
+    if (threadIdx.x != 8 * 32) return;              // lane 0 of the first producer warp
+    auto BAR = [&](int i) { return c.bar_base + 8u * (uint32_t)i; };
+    volatile int* const abort_flag = c.abort_flag;
+    const int n_ct = p.n_ct;
+    TileIter cur{c.u_first, 0, 0, 0, false};
+    tile_iter_settle(p, c.b, c.u_last, cur);
+    for (uint32_t it = 0; cur.valid; ++it, tile_iter_next(p, c.b, c.u_last, cur)) {
+        const uint32_t st = it % NSTAGE;
+        if (it >= NSTAGE) mbar_wait(BAR(B_EMPTY + st), ((it / NSTAGE) - 1u) & 1u, abort_flag, p.status, XSV_DEV_SITE_STAGE);
+        const bool cached = cur.kv < n_ct;
+        const int row0 = (cached ? cur.kv : cur.kv - n_ct) * BN;
+        const uint32_t kdst = c.smem_base + OFF_KV + st * 2 * TILE_BYTES, vdst = kdst + TILE_BYTES;
+        mbar_expect_tx(BAR(B_KFULL + (int)st), TILE_BYTES);
+        tma_load_3d(kdst, &maps.m[cached ? 0 : 2], BAR(B_KFULL + (int)st), 0, row0, cur.h);
+        mbar_expect_tx(BAR(B_VFULL + (int)st), TILE_BYTES);
+        tma_load_3d(vdst, &maps.m[cached ? 1 : 3], BAR(B_VFULL + (int)st), 0, row0, cur.h);
+    }
+}
+
+// One row of 64 16-bit values copied as it is (identity channel order) into a swizzled row of a tile; zeros for null.
+__device__ __forceinline__ void row16_raw_to_tile(const void* grow, uint8_t* tile, int row) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        *reinterpret_cast<uint4*>(tile + swz(row, i)) = grow ? reinterpret_cast<const uint4*>(grow)[i] : make_uint4(0u, 0u, 0u, 0u);
+}
+
+// Softmax warpgroups (warps 0-3: query tile A, warps 4-7: tile B) and the epilogue.  BF: the MMA operands are bf16
+// (an unquantised bf16 cache fed by the copy engine): the queries go in unconverted and the probabilities are packed
+// as bf16 pairs.
+template <typename T, int BITS, bool BF>
 __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
     constexpr int W = BITS == 16 ? 2 : 32 / BITS;
     uint8_t* const smem = cta.smem;
@@ -736,7 +803,8 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
             const int grow = q0 + row;
             // ---- this unit's queries -> shared memory (all MMAs reading the previous unit's tile are complete:
             //      the last S of that unit has been received)
-            if (row16_to_tile<T, W>(grow < F ? Qg + ((size_t)h * F + grow) * XSV_D : nullptr, sQ, row)) atomicOr(status, XSV_DEV_RANGE);
+            if (BF) row16_raw_to_tile(grow < F ? Qg + ((size_t)h * F + grow) * XSV_D : nullptr, sQ, row);
+            else if (row16_to_tile<T, W>(grow < F ? Qg + ((size_t)h * F + grow) * XSV_D : nullptr, sQ, row)) atomicOr(status, XSV_DEV_RANGE);
             fence_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(BAR(B_QFULL + X));
@@ -770,9 +838,9 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
                     if (!careful) {
                         const unsigned long long sc2 = f2_pack(SC, SC), nm2 = f2_pack(-m_used, -m_used);
                         unsigned long long ls2 = f2_pack(0.f, 0.f);
-                        softmax32_fast(va, sc2, nm2, ls2, pk);
+                        softmax32_fast<BF>(va, sc2, nm2, ls2, pk);
                         tmem_st16(tSb, pk);
-                        softmax32_fast(vb, sc2, nm2, ls2, pk);
+                        softmax32_fast<BF>(vb, sc2, nm2, ls2, pk);
                         tmem_st16(tSb + 16u, pk);
                         float l0, l1;
                         f2_unpack(ls2, l0, l1);
@@ -809,14 +877,14 @@ __device__ __noinline__ void softmax_loop(const Params& p, const Cta cta) {
                         const float nm = -m_used;
                         ls = 0.f;
                         if (valid >= SUB) {
-                            softmax32<false>(va, SC, nm, 32, ls, pk);
+                            softmax32<false, BF>(va, SC, nm, 32, ls, pk);
                             tmem_st16(tSb, pk);
-                            softmax32<false>(vb, SC, nm, 32, ls, pk);
+                            softmax32<false, BF>(vb, SC, nm, 32, ls, pk);
                             tmem_st16(tSb + 16u, pk);
                         } else {
-                            softmax32<true>(va, SC, nm, valid, ls, pk);
+                            softmax32<true, BF>(va, SC, nm, valid, ls, pk);
                             tmem_st16(tSb, pk);
-                            softmax32<true>(vb, SC, nm, valid - 32, ls, pk);
+                            softmax32<true, BF>(vb, SC, nm, valid - 32, ls, pk);
                             tmem_st16(tSb + 16u, pk);
                         }
                     }
@@ -893,7 +961,8 @@ __device__ __forceinline__ bool elect_one() {
 // the operands of the tcgen05 instructions (descriptors, tensor-memory addresses, barrier addresses) uniform.
 // What sets the pace of this loop is the chain of waits, fences and elections around each group of four MMAs,
 // not the MMAs themselves (which execute in 35-52 clocks each), hence one such loop per query tile.
-__device__ __noinline__ void mma_loop(const Params& p, const Cta c, const int x) {
+constexpr uint32_t IDESC_BF16 = (1u << 7) | (1u << 10);     // A and B are bf16 instead of fp16
+__device__ __noinline__ void mma_loop(const Params& p, const Cta c, const int x, const uint32_t fmt) {
     const uint32_t smem_base = c.smem_base, tmem_base = c.tmem_base;
     volatile int* const abort_flag = c.abort_flag;
     const int b = c.b, u_first = c.u_first, u_last = c.u_last;
@@ -915,7 +984,7 @@ __device__ __noinline__ void mma_loop(const Params& p, const Cta c, const int x)
         if (elect_one()) {
 #pragma unroll
             for (int k = 0; k < 4; ++k)            // 16 channels = 32 bytes inside the swizzled row
-                mma_ss(tS + buf * SUB, qd + 2u * k, kd + 2u * k, IDESC_QK, k > 0);
+                mma_ss(tS + buf * SUB, qd + 2u * k, kd + 2u * k, IDESC_QK | fmt, k > 0);
             tc_commit(BAR(B_SFULL + x * NBUF + (int)buf));
         }
         __syncwarp();
@@ -964,7 +1033,7 @@ __device__ __noinline__ void mma_loop(const Params& p, const Cta c, const int x)
                 if (elect_one()) {
 #pragma unroll
                     for (int k = 0; k < SUB / 16; ++k)     // 16 tokens: 8 columns of P, 2048 bytes of V
-                        mma_ts(tO, tS + buf * SUB + 8u * k, vd + 128u * k, IDESC_PV, k > 0 ? 1u : acc0);
+                        mma_ts(tO, tS + buf * SUB + 8u * k, vd + 128u * k, IDESC_PV | fmt, k > 0 ? 1u : acc0);
                     tc_commit(BAR(B_PVDONE + x * NBUF + (int)buf));
                     if (release) {
                         tc_commit(BAR(B_EMPTY + (int)st));
@@ -986,7 +1055,7 @@ __device__ __noinline__ void mma_loop(const Params& p, const Cta c, const int x)
 }
 
 // ------------------------------------------------------------------ the kernel
-template <typename T, int BITS>
+template <typename T, int BITS, bool BF>
 __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_constant__ BatchParams bp) {
     int s_idx = 0;
     while (s_idx + 1 < bp.n && (int)blockIdx.x >= bp.cta_base[s_idx + 1]) ++s_idx;    // uniform: this CTA's stream
@@ -1010,8 +1079,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_cons
 
     if (tid == 0) {
         for (int i = 0; i < NSTAGE; ++i) {
-            mbar_init(BAR(B_KFULL + i), 4);     // one arrival per producer warp
-            mbar_init(BAR(B_VFULL + i), 4);
+            mbar_init(BAR(B_KFULL + i), bp.use_tma ? 1 : 4);     // one arrival per slab of 32 rows, or the one that announces the copy
+            mbar_init(BAR(B_VFULL + i), bp.use_tma ? 1 : 4);
             mbar_init(BAR(B_EMPTY + i), 2);     // one commit per query tile
         }
         for (int x = 0; x < 2; ++x) {
@@ -1037,9 +1106,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) attn_tc5_kernel(const __grid_cons
     const Cta cta{smem, smem_base, bar_base, tmem_base, abort_flag, b, u_first, u_last};
 
     xsv_dep_sync();      // everything above is set-up that touches no global memory
-    if (warp < 8) softmax_loop<T, BITS>(p, cta);
-    else if (warp < 8 + NPROD) producer_loop<T, BITS>(p, cta);
-    else mma_loop(p, cta, warp - (8 + NPROD));
+    if (warp < 8) softmax_loop<T, BITS, BF>(p, cta);
+    else if (warp < 8 + NPROD) {
+        if (bp.use_tma) producer_tma_loop(p, cta, bp.tm[s_idx]);
+        else producer_loop<T, BITS>(p, cta);
+    }
+    else mma_loop(p, cta, warp - (8 + NPROD), BF ? IDESC_BF16 : 0u);
     tc_fence_before();
     __syncthreads();
     // Only now may the next kernel be scheduled: released at the start, its blocks would sit through this whole kernel
@@ -1161,7 +1233,7 @@ __global__ void wait_selftest_kernel(int* status) {
     mbar_wait(smem_u32(&bar), 0u, &abort_flag, status, XSV_DEV_SITE_SELFTEST);
 }
 
-template <typename T, int BITS>
+template <typename T, int BITS, bool BF = false>
 cudaError_t launch(const BatchParams& bp, bool merge_only, cudaStream_t st) {
     if (merge_only) {
         xsv_launch_dep(attn_combine_kernel<T>, dim3(16, bp.unit_base[bp.n]), dim3(256), 0, st, bp);
@@ -1171,11 +1243,11 @@ cudaError_t launch(const BatchParams& bp, bool merge_only, cudaStream_t st) {
     static XsvPerDeviceInt attr_set;      // the opt-in to large dynamic shared memory holds per device
     const int dev = xsv_current_device();
     if (!attr_set.get(dev)) {
-        cudaError_t e = cudaFuncSetAttribute(attn_tc5_kernel<T, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes<BITS>());
+        cudaError_t e = cudaFuncSetAttribute(attn_tc5_kernel<T, BITS, BF>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes<BITS>());
         if (e != cudaSuccess) return e;
         attr_set.set(dev, 1);
     }
-    xsv_launch_dep(attn_tc5_kernel<T, BITS>, dim3(bp.cta_base[bp.n]), dim3(NTHREADS), smem_bytes<BITS>(), st, bp);
+    xsv_launch_dep(attn_tc5_kernel<T, BITS, BF>, dim3(bp.cta_base[bp.n]), dim3(NTHREADS), smem_bytes<BITS>(), st, bp);
     xsv_count_launch(1);
     return cudaGetLastError();
 }
@@ -1202,6 +1274,48 @@ void fill_params(Params& p, const LayerView& lv, int T_c, const void* Q, const v
     p.n_full = ((p.npair - 1) * 2 * BM + BM < F) ? p.npair : p.npair - 1;
     p.ticks_head = p.n_full * unit_len(p, true) + (p.npair - p.n_full) * unit_len(p, false);
     p.total = p.ticks_head * H;
+}
+
+// ---- tensor maps for the copy-engine feed (bits == 16: the cache holds the 16-bit inputs themselves)
+typedef CUresult (*XsvEncodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+XsvEncodeTiled encode_tiled_fn() {          // the driver's encoder, looked up once; null where there is no driver
+    static XsvEncodeTiled fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        return (XsvEncodeTiled)f;
+    }();
+    return fn;
+}
+// [heads][rows][64] fp16 with `head_stride_rows` rows between heads, read in boxes of 128 rows; rows at or beyond
+// `rows` read as zeros.  False if the tensor cannot be described (no encoder, an unaligned pointer).
+bool encode_rows_map(CUtensorMap* m, const void* base, long long rows, long long head_stride_rows, int H, int dtype) {
+    XsvEncodeTiled enc = encode_tiled_fn();
+    if (!enc || !base || (reinterpret_cast<uintptr_t>(base) & 15u) != 0) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)XSV_D, (cuuint64_t)(rows > 0 ? rows : 1), (cuuint64_t)H};
+    const cuuint64_t strides[2] = {(cuuint64_t)XSV_D * 2, (cuuint64_t)head_stride_rows * XSV_D * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)XSV_D, (cuuint32_t)BN, 1u};
+    const cuuint32_t estr[3] = {1u, 1u, 1u};
+    return enc(m, dtype == 0 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// The four maps of one stream; false leaves the launch on the producers' own loads.
+bool encode_stream_maps(StreamMaps& sm, const Params& p, int dtype) {
+    if (p.lv.bits != 16 || p.H < 1 || p.F < 1) return false;
+    return encode_rows_map(&sm.m[0], p.lv.kcodes, p.T_c, p.lv.cap, p.H, dtype) && encode_rows_map(&sm.m[1], p.lv.vcodes, p.T_c, p.lv.cap, p.H, dtype) &&
+           encode_rows_map(&sm.m[2], p.K, p.F, p.F, p.H, dtype) && encode_rows_map(&sm.m[3], p.V, p.F, p.F, p.H, dtype);
+}
+// Whether the launch described by bp (streams and CTAs already dealt) can be fed by the copy engine, and its maps.
+void prepare_tma(BatchParams& bp, int dtype) {
+    static const bool off = getenv("XSV_NO_TMA") != nullptr;      // for comparisons
+    bp.use_tma = 0;
+    if (off || (dtype != 0 && dtype != 1) || bp.n < 1 || bp.p[0].lv.bits != 16) return;
+    for (int i = 0; i < bp.n; ++i)
+        if (!encode_stream_maps(bp.tm[i], bp.p[i], dtype)) return;
+    bp.use_tma = 1;
 }
 
 // CTAs of the launch dealt to the streams in proportion to their work (at least one each, never more than a
@@ -1243,7 +1357,9 @@ cudaError_t launch_tc5(const BatchParams& bp, int dtype, int bits, bool merge_on
             case 2: XSV_TC5(__nv_bfloat16, 2);
             case 4: XSV_TC5(__nv_bfloat16, 4);
             case 8: XSV_TC5(__nv_bfloat16, 8);
-            case 16: XSV_TC5(__nv_bfloat16, 16);
+            case 16:
+                if (bp.use_tma && !merge_only) return launch<__nv_bfloat16, 16, true>(bp, merge_only, st);   // bf16 operands, copy-engine feed
+                XSV_TC5(__nv_bfloat16, 16);
         }
     }
 #undef XSV_TC5
@@ -1258,6 +1374,7 @@ cudaError_t launch_one(const LayerView& lv, int T_c, const void* Q, const void* 
     fill_params(bp.p[0], lv, T_c, Q, K, V, out, H, F, status);
     const int sms = xsv_sm_count() - spare_sms > 0 ? xsv_sm_count() - spare_sms : 1;   // multiprocessors left to another kernel
     deal_ctas(bp, workspace, sms);
+    if (!merge_only) prepare_tma(bp, dtype);
     return launch_tc5(bp, dtype, lv.bits, merge_only, st);
 }
 }  // namespace
@@ -1326,6 +1443,7 @@ cudaError_t xsv_launch_attn_tc5_batch(int n, const LayerView* lvs, const int* T_
     BatchParams bp;
     for (int first = 0; first < n; first += g) {
         build_group(ps, first, std::min(g, n - first), workspace, sms, bp);
+        prepare_tma(bp, dtype);
         cudaError_t e = launch_tc5(bp, dtype, lvs[0].bits, false, st);
         if (e != cudaSuccess) return e;
         e = launch_tc5(bp, dtype, lvs[0].bits, true, st);     // the merge reads the workspace the next group reuses

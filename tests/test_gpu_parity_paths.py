@@ -79,6 +79,18 @@ def test_paper_shape_unquantised_cache(dtype, L_max):
     assert w["checked"] == 4 and w["pruned_steps"] == (2 if L_max else 0)
 
 
+def test_unquantised_fp16_cache_fed_by_the_copy_engine():
+    # fp16 inputs with bits = 16: K and V tiles reach shared memory by tensor-map bulk copies (rows past the end of the
+    # cache or of the frame arrive as zeros).  Ragged sizes: 300-token frames (a 44-row last tile), a cache that ends
+    # inside a tile after pruning, several heads; every step checked.  Then two such streams in one launch.
+    st = synth.Stream(H=3, d=64, F=300, dtype="fp16", layer=43)
+    w = run_stream(st, 7, 1000, 16)
+    assert w["checked"] == 7 and w["pruned_steps"] >= 3
+    streams = [synth.Stream(H=3, d=64, F=300 - 40 * i, dtype="fp16", layer=44 + i) for i in range(2)]
+    w = run_batch(streams, 6, 900, 16, starts=[0, 1])
+    assert w["pruned_steps"] >= 4
+
+
 @pytest.mark.parametrize("bits", [2, 4])
 def test_frames_of_alternating_size(bits):
     # frame sizes differ from step to step (inputs resized to a maximum edge have varying token counts):
@@ -186,12 +198,16 @@ def test_bf16_inputs_at_the_edges_of_the_fp16_range():
 
     w = run_stream(st, 6, 0, 16, frame_fn=frame, max_cache_tokens=1024)           # raw 16-bit cache: the inputs themselves
     assert w["checked"] == 6
-    c = binding.Cache(1, H, 64, 0, 16)
     q, k, v = frame(0)
     v[0, 0, 0] = 65536.0
     out = torch.empty(H, F, 64, device="cuda", dtype=torch.bfloat16)
+    c = binding.Cache(1, H, 64, 1000, 4)              # a quantised cache attends over fp16 operands: out of range
     c.step(0, to_dev(q, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), out)
     assert c.status() == 7                                                         # XSV_ERR_RANGE
+    c.destroy()
+    c = binding.Cache(1, H, 64, 0, 16)                # an unquantised bf16 cache attends over bf16 operands: no such limit
+    c.step(0, to_dev(q, "bf16"), to_dev(k, "bf16"), to_dev(v, "bf16"), out)
+    assert c.status() == 0 and bool(torch.isfinite(out.float()).all())
     c.destroy()
 
 
